@@ -1,0 +1,366 @@
+"""Pins for the CPU oracle: each test checks oracle/ckv_oracle.py against something
+other than itself -- brute force written with plain loops, closed forms, invariants
+that follow from the paper's equations, or a textbook routine."""
+import itertools
+import json
+import math
+import os
+
+import numpy as np
+import pytest
+from scipy.special import softmax
+
+from oracle import ckv_oracle as O
+
+GOLDEN = os.path.join(os.path.dirname(__file__), "golden")
+
+
+def rand_cache(rng, L, H, s, d, ar=0.0):
+    K = rng.standard_normal((L, H, s, d))
+    if ar > 0:
+        for t in range(1, s):
+            K[:, :, t] = ar * K[:, :, t - 1] + K[:, :, t]
+    V = rng.standard_normal((L, H, s, d))
+    return K, V
+
+
+# ----------------------------------------------------------------------------- P1: brute force on tiny chunks
+
+def brute_round(K, V, deg, n_sink, n_recent, c, M):
+    """One round written with plain loops: full cosine matrix, exhaustive choice of
+    the M edges with the largest total similarity, explicit member lists (Sec. 5.2, 5.3, Eq. 2, Eq. 5)."""
+    s, d = len(K), len(K[0])
+    lo, hi = n_sink, s - n_recent
+
+    def cos(i, j):
+        dot = sum(K[i][x] * K[j][x] for x in range(d))
+        ni = math.sqrt(sum(K[i][x] ** 2 for x in range(d)))
+        nj = math.sqrt(sum(K[j][x] ** 2 for x in range(d)))
+        return dot / (ni * nj)
+
+    edges = []  # (a, b, sim)
+    start = lo
+    while start < hi and hi - lo >= 2:
+        end = min(start + c, hi)
+        odd_1idx = [p for p in range(start, end) if (p - start + 1) % 2 == 1]   # 1-indexed odd = set A
+        even_1idx = [p for p in range(start, end) if (p - start + 1) % 2 == 0]  # set B
+        for a in odd_1idx:
+            best, best_s = None, None
+            for b in even_1idx:
+                sc = cos(a, b)
+                if best is None or sc > best_s:
+                    best, best_s = b, sc
+            if best is not None:
+                edges.append((a, best, best_s))
+        start = end
+    best_subset, best_total = (), -1e300
+    for sub in itertools.combinations(range(len(edges)), M):
+        tot = sum(edges[i][2] for i in sub)
+        if tot > best_total + 1e-15:
+            best_subset, best_total = sub, tot
+    clusters = {}
+    gone = set()
+    for i in best_subset:
+        a, b, _ = edges[i]
+        clusters.setdefault(b, [b]).append(a)
+        gone.add(a)
+    Ko, Vo, do = [], [], []
+    for p in range(s):
+        if p in gone:
+            continue
+        mem = clusters.get(p, [p])
+        n = sum(deg[m] for m in mem)
+        Ko.append([sum(deg[m] * K[m][x] for m in mem) / n for x in range(d)])
+        Vo.append([sum(deg[m] * V[m][x] for m in mem) / n for x in range(d)])
+        do.append(n)
+    return np.array(Ko), np.array(Vo), np.array(do), len(edges)
+
+
+@pytest.mark.parametrize("c", [4, 6, 8])
+@pytest.mark.parametrize("r", [1.0, 0.5, 0.34])
+@pytest.mark.parametrize("sink,recent,s", [(0, 0, 16), (1, 2, 19), (3, 0, 12)])
+def test_p1_brute_force_rounds(c, r, sink, recent, s):
+    rng = np.random.default_rng(100 * c + s)
+    K, V = rand_cache(rng, 1, 1, s, 5, ar=0.7)
+    deg = np.ones((1, 1, s), dtype=np.int64)
+    p = O.Params(chunk=c, n_sink=sink, n_recent=recent, select=O.SELECT_GLOBAL, budget=0)
+    for _ in range(3):  # three rounds: degrees > 1 enter the later ones
+        Ko, Vo, do, _, log = O.csm_round(K, V, deg, p, r)
+        n_edges = len(log.edges[0].a_pos)
+        M = int(math.floor(r * n_edges + 1e-9))
+        Kb, Vb, db, n_edges_b = brute_round(K[0, 0].tolist(), V[0, 0].tolist(), deg[0, 0].tolist(), sink, recent, c, M)
+        assert n_edges == n_edges_b
+        assert Ko.shape[2] == Kb.shape[0] == K.shape[2] - M
+        np.testing.assert_allclose(Ko[0, 0], Kb, rtol=1e-12, atol=1e-12)
+        np.testing.assert_allclose(Vo[0, 0], Vb, rtol=1e-12, atol=1e-12)
+        np.testing.assert_array_equal(do[0, 0], db)
+        K, V, deg = Ko, Vo, do
+
+
+def test_p1_chunk_mode_is_per_chunk_top_m():
+    rng = np.random.default_rng(7)
+    s, c = 24, 8
+    K, V = rand_cache(rng, 1, 1, s, 4, ar=0.5)
+    deg = np.ones((1, 1, s), dtype=np.int64)
+    p = O.Params(chunk=c, n_sink=0, n_recent=0, select=O.SELECT_CHUNK)
+    Ko, Vo, do, _, _ = O.csm_round(K, V, deg, p, 0.5)
+    outs = []
+    for i in range(s // c):  # each chunk on its own, brute force, M = floor(0.5 * 4) = 2
+        sl = slice(i * c, (i + 1) * c)
+        Kb, Vb, db, _ = brute_round(K[0, 0, sl].tolist(), V[0, 0, sl].tolist(), [1] * c, 0, 0, c, 2)
+        outs.append((Kb, Vb, db))
+    np.testing.assert_allclose(Ko[0, 0], np.concatenate([o[0] for o in outs]), rtol=1e-12)
+    np.testing.assert_allclose(Vo[0, 0], np.concatenate([o[1] for o in outs]), rtol=1e-12)
+    np.testing.assert_array_equal(do[0, 0], np.concatenate([o[2] for o in outs]))
+
+
+def test_hand_worked_example():
+    """A four-token chunk small enough to do on paper (Eq. 2, Eq. 5); numbers in tests/golden/hand_example.json."""
+    g = json.load(open(os.path.join(GOLDEN, "hand_example.json")))
+    K = np.array(g["K"], dtype=np.float64)[None, None]
+    V = np.array(g["V"], dtype=np.float64)[None, None]
+    deg = np.array(g["deg"], dtype=np.int64)[None, None]
+    p = O.Params(chunk=4, n_sink=0, n_recent=0)
+    Ko, Vo, do, asg, log = O.csm_round(K, V, deg, p, 1.0)
+    np.testing.assert_array_equal(log.edges[0].b_pos, g["edge_b"])
+    np.testing.assert_allclose(log.edges[0].sim, g["edge_sim"], rtol=1e-6)
+    np.testing.assert_allclose(Ko[0, 0], g["K_out"], rtol=1e-12)
+    np.testing.assert_allclose(Vo[0, 0], g["V_out"], rtol=1e-12)
+    np.testing.assert_array_equal(do[0, 0], g["deg_out"])
+    np.testing.assert_array_equal(asg[0, 0], g["assign"])
+    # top-1 of two edges (r = 0.5): only the better edge (token 2 -> 3, cos = 1) is merged
+    Ko, Vo, do, asg, _ = O.csm_round(K, V, deg, p, 0.5)
+    np.testing.assert_array_equal(do[0, 0], g["deg_out_half"])
+    np.testing.assert_array_equal(asg[0, 0], g["assign_half"])
+
+
+# ----------------------------------------------------------------------------- P2-P5, P12: fixed points and invariants
+
+def test_p2_ratio_zero_is_identity():
+    rng = np.random.default_rng(1)
+    K, V = rand_cache(rng, 2, 2, 50, 8, ar=0.8)
+    p = O.Params(chunk=8, n_sink=3, n_recent=5, r_init=0.0, r_decay=0.0, r_min=0.0, n_rounds_max=3, budget=0)
+    Ko, Vo, do, asg, logs = O.compress_prefill(K, V, None, p)
+    assert len(logs) == 3
+    np.testing.assert_array_equal(Ko, K)
+    np.testing.assert_array_equal(Vo, V)
+    np.testing.assert_array_equal(do, np.ones((2, 2, 50)))
+    np.testing.assert_array_equal(asg[0, 0], np.arange(50))
+
+
+def test_p3_identical_keys_merge_to_exact_mean():
+    rng = np.random.default_rng(2)
+    s, c, d = 32, 8, 6
+    K = np.repeat(rng.standard_normal((1, 1, s // c, 1, d)), c, axis=3).reshape(1, 1, s, d)  # one key per chunk
+    V = rng.standard_normal((1, 1, s, d))
+    deg = rng.integers(1, 5, size=(1, 1, s))
+    p = O.Params(chunk=c, n_sink=0, n_recent=0)
+    Ko, Vo, do, asg, _ = O.csm_round(K, V, deg, p, 1.0)
+    for t in range(Ko.shape[2]):
+        mem = np.nonzero(asg[0, 0] == t)[0]
+        np.testing.assert_allclose(Ko[0, 0, t], K[0, 0, mem[0]], rtol=1e-15, atol=0)
+        w = deg[0, 0, mem]
+        np.testing.assert_allclose(Vo[0, 0, t], (w[:, None] * V[0, 0, mem]).sum(0) / w.sum(), rtol=1e-13)
+        assert do[0, 0, t] == w.sum()
+    # all cosines are 1, so every A token ties over all B tokens and must take the first one
+    e = O.match_head(K[0, 0], 0, 0, c)
+    np.testing.assert_array_equal(e.b_pos, (e.a_pos // c) * c + 1)
+
+
+@pytest.mark.parametrize("select", [O.SELECT_GLOBAL, O.SELECT_CHUNK])
+def test_p4_p5_degree_and_first_moment_conservation(select):
+    rng = np.random.default_rng(3)
+    L, H, s, d = 2, 3, 203, 8
+    K, V = rand_cache(rng, L, H, s, d, ar=0.9)
+    p = O.Params(chunk=16, n_sink=4, n_recent=7, r_init=0.8, r_decay=0.2, r_min=0.2, budget=s // 4, select=select,
+                 n_rounds_max=40)
+    Ko, Vo, do, asg, logs = O.compress_prefill(K, V, None, p)
+    assert len(logs) >= 2
+    if select == O.SELECT_GLOBAL:
+        assert Ko.shape[2] == s // 4           # the last round is trimmed onto the budget
+    else:
+        assert Ko.shape[2] <= s // 4
+    np.testing.assert_array_equal(do.sum(axis=2), np.full((L, H), s))
+    np.testing.assert_allclose((do[..., None] * Ko).sum(axis=2), K.sum(axis=2), rtol=1e-10, atol=1e-10)
+    np.testing.assert_allclose((do[..., None] * Vo).sum(axis=2), V.sum(axis=2), rtol=1e-10, atol=1e-10)
+    # assign really is the cluster map: degree = member count, centroid = member mean (all original degrees are 1)
+    for t in range(0, Ko.shape[2], 7):
+        mem = np.nonzero(asg[1, 2] == t)[0]
+        assert do[1, 2, t] == len(mem)
+        np.testing.assert_allclose(Ko[1, 2, t], K[1, 2, mem].mean(axis=0), rtol=1e-10, atol=1e-12)
+
+
+def test_p4_append_keeps_degree_sum_and_triggers_per_chunk():
+    rng = np.random.default_rng(4)
+    L, H, s, d, c = 1, 2, 40, 4, 8
+    K, V = rand_cache(rng, L, H, s, d, ar=0.8)
+    deg = np.ones((L, H, s), dtype=np.int64)
+    p = O.Params(chunk=c, r_init=1.0, r_decay=0.0, r_min=1.0, n_rounds_max=2, budget=0)
+    kn, vn = rand_cache(rng, L, H, 21, d, ar=0.8)
+    Ka, Va, da, pend = O.compress_append(K, V, deg, 0, kn, vn, p)
+    # 21 new tokens = two full windows (8 -> 4 -> 2 each) + 5 pending
+    assert pend == 5 and Ka.shape[2] == s + 2 + 2 + 5
+    np.testing.assert_array_equal(da.sum(axis=2), np.full((L, H), s + 21))
+    np.testing.assert_array_equal(Ka[:, :, :s], K)                 # the old cache is not touched
+    np.testing.assert_array_equal(Ka[:, :, -5:], kn[:, :, -5:])    # pending tokens are stored verbatim
+    np.testing.assert_allclose((da[..., None] * Va).sum(axis=2), V.sum(axis=2) + vn.sum(axis=2), rtol=1e-10)
+
+
+def test_p12_at_most_half_and_borders_untouched():
+    rng = np.random.default_rng(5)
+    s, n1, n2 = 101, 6, 9
+    K, V = rand_cache(rng, 1, 2, s, 8, ar=0.9)
+    deg = rng.integers(1, 4, size=(1, 2, s))
+    p = O.Params(chunk=10, n_sink=n1, n_recent=n2)
+    Ko, Vo, do, _, log = O.csm_round(K, V, deg, p, 1.0)
+    m = s - n1 - n2
+    assert log.s_out >= s - m // 2
+    assert log.s_out == s - sum(len(range(0, min(10, m - b), 2)) if min(10, m - b) >= 2 else 0 for b in range(0, m, 10))
+    np.testing.assert_array_equal(Ko[:, :, :n1], K[:, :, :n1])
+    np.testing.assert_array_equal(Vo[:, :, -n2:], V[:, :, -n2:])
+    np.testing.assert_array_equal(do[:, :, :n1], deg[:, :, :n1])
+    np.testing.assert_array_equal(do[:, :, -n2:], deg[:, :, -n2:])
+
+
+def test_odd_and_single_token_chunks():
+    rng = np.random.default_rng(6)
+    # middle of 9 tokens with c = 4: chunks of 4, 4 and 1 -> the lone token passes through and draws no edge
+    K, V = rand_cache(rng, 1, 1, 9, 4)
+    e = O.match_head(K[0, 0], 0, 0, 4)
+    assert len(e.a_pos) == 4 and 8 not in e.a_pos
+    # middle of 7 with c = 4: last chunk has 3 tokens: A = {4, 6}, B = {5}
+    e = O.match_head(K[0, 0, :7], 0, 0, 4)
+    np.testing.assert_array_equal(e.a_pos, [0, 2, 4, 6])
+    np.testing.assert_array_equal(e.b_pos[2:], [5, 5])
+
+
+def test_zero_norm_key_has_zero_similarity():
+    K = np.array([[0.0, 0.0], [1.0, 0.0], [1.0, 1.0], [0.0, 2.0]])
+    e = O.match_head(K, 0, 0, 4)
+    assert e.sim[0] == 0.0 and e.b_pos[0] == 1     # all-zero row: every candidate scores 0, first one wins
+
+
+def test_ranking_ties_go_to_lower_position():
+    # two chunks with identical content: equal similarities; M = 1 must take the edge at the lower position
+    base = np.array([[1.0, 0.2], [1.0, 0.0], [0.0, 1.0], [0.3, 1.0]])
+    K = np.concatenate([base, base])[None, None]
+    V = np.zeros_like(K)
+    deg = np.ones((1, 1, 8), dtype=np.int64)
+    e = O.match_head(K[0, 0], 0, 0, 4)
+    sel, _ = O.select_edges(e, 0.25, 8, 0, O.SELECT_GLOBAL)
+    assert sel.sum() == 1 and e.a_pos[sel][0] == int(e.a_pos[np.argmax(e.sim)])
+    assert e.a_pos[sel][0] < 4
+
+
+def test_schedule_eq4_with_floor():
+    p = O.Params(r_init=0.8, r_decay=0.2, r_min=0.2)
+    np.testing.assert_allclose([O.ratio_for_round(p, j) for j in range(6)], [0.8, 0.6, 0.4, 0.2, 0.2, 0.2], atol=1e-12)
+    assert O.merges_from_ratio(0.6, 10) == 6 and O.merges_from_ratio(0.8, 7) == 5 and O.merges_from_ratio(0.2, 4) == 0
+
+
+# ----------------------------------------------------------------------------- P6-P9: attention
+
+def textbook_attention(q, K, V, scale):
+    return softmax((q @ K.T) * scale, axis=-1) @ V
+
+
+def test_p6_unit_degrees_give_softmax_attention():
+    rng = np.random.default_rng(10)
+    H, G, s, d = 2, 3, 37, 16
+    q = rng.standard_normal((H * G, d))
+    K, V = rng.standard_normal((H, s, d)), rng.standard_normal((H, s, d))
+    out = O.app_attn(q, K, V, np.ones((H, s), dtype=np.int64), 1 / math.sqrt(d))
+    for j in range(H * G):
+        np.testing.assert_allclose(out[j], textbook_attention(q[j], K[j // G], V[j // G], 1 / math.sqrt(d)), rtol=1e-12)
+    np.testing.assert_allclose(O.attn(q, K, V, 1 / math.sqrt(d)), out, rtol=1e-14)
+
+
+def test_p7_zero_query_returns_mean_of_original_values():
+    rng = np.random.default_rng(11)
+    K, V = rand_cache(rng, 1, 2, 96, 8, ar=0.9)
+    p = O.Params(chunk=16, n_sink=2, n_recent=3, r_init=0.8, r_decay=0.2, r_min=0.2, budget=30)
+    Ko, Vo, do, _, _ = O.compress_prefill(K, V, None, p)
+    out = O.app_attn(np.zeros((2, 8)), Ko[0], Vo[0], do[0], 0.3)
+    np.testing.assert_allclose(out, V[0].mean(axis=1), rtol=1e-11, atol=1e-12)
+
+
+def test_p8_replication_identity():
+    rng = np.random.default_rng(12)
+    H, s, d = 2, 11, 8
+    q = rng.standard_normal((H * 2, d))
+    K, V = rng.standard_normal((H, s, d)), rng.standard_normal((H, s, d))
+    deg = rng.integers(1, 6, size=(H, s))
+    out = O.app_attn(q, K, V, deg, 0.4)
+    for j in range(H * 2):
+        h = j // 2
+        Kr, Vr = np.repeat(K[h], deg[h], axis=0), np.repeat(V[h], deg[h], axis=0)
+        np.testing.assert_allclose(out[j], textbook_attention(q[j], Kr, Vr, 0.4), rtol=1e-12)
+
+
+def test_p9_duplicated_keys_make_the_approximation_exact():
+    rng = np.random.default_rng(13)
+    s, d, c = 64, 8, 16
+    K = rng.standard_normal((1, 1, s, d))
+    K[:, :, 0::2] = K[:, :, 1::2]                       # every A token carries its right neighbour's key
+    V = rng.standard_normal((1, 1, s, d))
+    p = O.Params(chunk=c, n_sink=0, n_recent=0, r_init=1.0, r_decay=0, r_min=1.0, n_rounds_max=1)
+    Ko, Vo, do, asg, _ = O.compress_prefill(K, V, None, p)
+    np.testing.assert_array_equal(asg[0, 0], np.arange(s) // 2)
+    np.testing.assert_allclose(Ko[0, 0], K[0, 0, 1::2], rtol=1e-15)
+    q = rng.standard_normal((1, d))
+    np.testing.assert_allclose(O.app_attn(q, Ko[0], Vo[0], do[0], 0.35), textbook_attention(q[0], K[0, 0], V[0, 0], 0.35)[None],
+                               rtol=1e-12)
+
+
+# ----------------------------------------------------------------------------- P10: Theorem A.1
+
+def c_closed_form(n, l):
+    """c_{2n,l} as printed in the proof of Theorem A.1."""
+    if l % 2 == 0:
+        return -l ** 3 / 12 + (2 * n - 1) / 4 * l ** 2 + (6 * n - 1) / 6 * l
+    return -l ** 3 / 12 + (2 * n - 1) / 4 * l ** 2 + (12 * n - 5) / 12 * l + (2 * n - 1) / 4
+
+
+@pytest.mark.parametrize("n", [1, 2, 3, 4, 5])
+def test_p10_alternating_partition_is_optimal(n):
+    rng = np.random.default_rng(20 + n)
+    A0, B0 = O.alternating_partition(2 * n)
+    np.testing.assert_array_equal(A0 + 1, np.arange(1, 2 * n, 2))   # {1, 3, ...} in the theorem's 1-indexed notation
+    np.testing.assert_array_equal(B0 + 1, np.arange(2, 2 * n + 1, 2))
+    for _ in range(5):
+        steps = np.sort(rng.random(2 * n - 1))[::-1]                # decreasing, non-negative differences => convex decreasing f
+        fvals = np.concatenate([[0.0], -np.cumsum(steps)])           # fvals[dist - 1]
+        f = lambda dist: fvals[dist - 1]
+        best = max(O.partition_objective(A, [x for x in range(2 * n) if x not in A], f)
+                   for A in itertools.combinations(range(2 * n), n))
+        assert O.partition_objective(A0, B0, f) >= best - 1e-12
+
+
+@pytest.mark.parametrize("n", [2, 3, 5, 7])
+def test_p10_closed_form_counts(n):
+    A0, B0 = O.alternating_partition(2 * n)
+    dist = [abs(int(a) - int(b)) for a in A0 for b in B0]
+    for i in range(1, n + 1):
+        assert dist.count(2 * i - 1) == 2 * n - 2 * i + 1             # |D_{A0,B0,2i-1}|
+    for l in range(1, 2 * n - 1):
+        lhs = sum((l + 1 - i) * dist.count(i) for i in range(1, l + 1))
+        assert abs(lhs - c_closed_form(n, l)) < 1e-9                  # equality case of the proof's bound
+
+
+# ----------------------------------------------------------------------------- P11, P13
+
+def test_p11_table1_multiply_add_count():
+    g = json.load(open(os.path.join(GOLDEN, "table1_macs.json")))
+    for case in g["cases"]:
+        n, c, d = case["n"], case["c"], case["d"]
+        K = np.random.default_rng(0).standard_normal((n, d))
+        assert O.match_head(K, 0, 0, c).macs == case["macs"] == n * c * d // 4
+
+
+def test_p13_ar1_edges_join_neighbours():
+    import torch
+    from paper_2506_11418_b200 import synth
+    K = synth.ar1_keys(1, 1, 2048, 128, (0.9, 0.9), 0.0, seed=0).double().numpy()
+    e = O.match_head(K[0, 0], 0, 0, 64)
+    assert np.mean(np.abs(e.a_pos - e.b_pos) == 1) > 0.9
+    assert 0.8 < float(np.mean(e.sim)) < 0.97   # E[cos] at distance 1 is about rho = 0.9
