@@ -1,0 +1,136 @@
+/*
+ * ckv -- CentroidKV hot path for NVIDIA B200 (sm_100a): Chunked Soft Matching KV-cache
+ * clustering, degree-weighted centroid merge, online append, and decode attention over
+ * the compressed cache.  C ABI; no C++ or framework types cross this boundary.
+ *
+ * Conventions
+ *  - Every pointer is a DEVICE pointer owned by the caller unless its comment says "host".
+ *    The library allocates and frees nothing and keeps no global state.
+ *  - All work is enqueued on `cuda_stream` (a cudaStream_t passed as void*; NULL = the
+ *    default stream) and the calls return without synchronising.
+ *  - The return value is a ckv_status.  Argument errors are found on the host before any
+ *    launch and leave every output untouched.
+ *  - Tensors are row-major.  K and V of one sequence: [L, H, cap, D] (layers, KV heads,
+ *    token capacity, head_dim) of which the first `len` tokens of every (layer, head)
+ *    are valid; deg and logdeg: [L, H, cap].  K and V must be 16-byte aligned.
+ *  - Thread safety: calls on distinct streams with distinct workspaces and outputs do
+ *    not interfere.
+ *  - This version supports D = 128 and even chunk sizes 2..256; anything else returns
+ *    CKV_ERR_UNSUPPORTED.
+ */
+#ifndef CKV_H_
+#define CKV_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum { CKV_F32 = 0, CKV_BF16 = 1 } ckv_dtype;
+
+typedef enum {
+  CKV_SELECT_GLOBAL = 0, /* rank the edges of all chunks of a (layer, head) together (Sec. 5.2 last paragraph, Sec. 5.3) */
+  CKV_SELECT_CHUNK = 1   /* rank the edges inside each chunk */
+} ckv_select;
+
+typedef enum {
+  CKV_OK = 0,
+  CKV_ERR_INVALID_ARG = 1, /* null pointer, negative size, odd chunk, overlapping src/dst ... */
+  CKV_ERR_ALIGNMENT = 2,   /* K, V, q or out not 16-byte aligned */
+  CKV_ERR_CAPACITY = 3,    /* a destination cache is too small for what would be written */
+  CKV_ERR_WORKSPACE = 4,   /* workspace NULL or smaller than ckv_*_workspace_bytes says */
+  CKV_ERR_NO_PROGRESS = 5, /* the ratio schedule merges nothing although the budget is not met */
+  CKV_ERR_UNSUPPORTED = 6, /* head_dim, chunk size or group size outside this version's range */
+  CKV_ERR_CUDA = 7         /* a CUDA runtime call failed (launch configuration, invalid stream ...) */
+} ckv_status;
+
+/* One sequence's KV cache over all layers and KV heads, with the cluster degrees N of Sec. 3
+ * (n_t = number of original tokens merged into slot t). */
+typedef struct ckv_cache {
+  void* k;         /* [L, H, cap, D] */
+  void* v;         /* [L, H, cap, D] */
+  int32_t* deg;    /* [L, H, cap] cluster degree n_t >= 1.  As a source: NULL means all ones.  As a destination: required. */
+  float* logdeg;   /* [L, H, cap] natural log of deg, kept for Eq. 3's bias.  As a destination: NULL = not maintained. */
+  int32_t L, H, D; /* layers, KV heads, head_dim */
+  int32_t dtype;   /* ckv_dtype of k and v */
+  int64_t cap;     /* capacity in tokens of every (layer, head) slab */
+  int64_t len;     /* valid tokens; the same for every (layer, head), since the merge count depends on shapes only */
+  int64_t pending; /* appended tokens at the tail that have not yet formed a full chunk (append path) */
+} ckv_cache;
+
+/* Algorithm 1's inputs and Eq. 4's schedule. */
+typedef struct ckv_params {
+  int32_t chunk;        /* c: chunk size, even */
+  int32_t n_sink;       /* n1: leading tokens never merged */
+  int32_t n_recent;     /* n2: trailing tokens never merged */
+  int32_t n_rounds_max; /* upper bound on clustering rounds per call */
+  float r_init;         /* Eq. 4: ratio of round 0 = fraction of the matched edges that are merged */
+  float r_decay;        /* Eq. 4: delta_r */
+  float r_min;          /* floor: r_j = max(r_init - j * r_decay, r_min) */
+  int32_t select;       /* ckv_select */
+  int64_t budget;       /* B: target cache length, sinks and recent tokens included.  0 = run exactly n_rounds_max rounds.
+                           ckv_compress_append applies it to each completed window of `chunk` appended tokens. */
+} ckv_params;
+
+/* Host-only: what a ckv_compress_prefill call with this source length would do (Algorithm 1's
+ * `while s > B` loop with Eq. 4): the final length, the number of rounds, the capacity the
+ * destination needs.  Any output pointer (host) may be NULL.  No GPU is touched. */
+int ckv_compress_plan(int64_t len, const ckv_params* params, int64_t* out_len, int64_t* rounds,
+                      int64_t* dst_cap_needed);
+
+/* Host-only: bytes of workspace ckv_compress_prefill / ckv_compress_append need for a cache of
+ * this shape (k, v, deg pointers are not read).  Returns 0 for invalid arguments. */
+size_t ckv_workspace_bytes(const ckv_cache* shape, const ckv_params* params);
+
+/* Algorithm 1, pre-filling branch; one round is Sec. 5.2 (chunks, alternating split, cosine
+ * similarity of Eq. 2, one edge per A token), Sec. 5.3 (merge the top fraction r of the ranked
+ * edges, Eq. 4) and Eq. 5 (degree-weighted centroids of K and V, degrees summed).
+ * Compresses src (len tokens) into dst: sinks, then the survivors of the middle in their
+ * original order with each centroid at its B token's place, then the recent tokens.
+ * dst must not overlap src or the workspace; dst->cap must be at least what ckv_compress_plan
+ * reports.  On return dst->len (host field) is the new length, dst->pending is 0.
+ * assign: optional [L, H, src->len] int32, receives for each source token the dst slot that
+ * holds it (its cluster).  rounds_done: optional host pointer. */
+int ckv_compress_prefill(const ckv_cache* src, ckv_cache* dst, const ckv_params* params, int32_t* assign,
+                         void* workspace, size_t workspace_bytes, void* cuda_stream, int64_t* rounds_done);
+
+/* Algorithm 1, decoding branch, `K = [K, k], V = [V, v], N = [N, 1]`: appends t_new tokens
+ * (k_new, v_new: [L, H, t_new, D], cache dtype) with degree 1.  Whenever the appended tail
+ * reaches `chunk` tokens that window alone is clustered as a stand-alone sequence (no sinks
+ * or recent tokens inside it) with Eq. 4's schedule until it is no longer than params->budget
+ * (0: exactly n_rounds_max rounds), and the result replaces the window.
+ * cache->len and cache->pending (host fields) are updated; CKV_ERR_CAPACITY if the cache
+ * cannot hold the tokens. */
+int ckv_compress_append(ckv_cache* cache, const void* k_new, const void* v_new, int32_t t_new,
+                        const ckv_params* params, void* workspace, size_t workspace_bytes, void* cuda_stream);
+
+/* One layer of one sequence for decode attention: k, v: [H, cap, D]; logdeg: [H, cap] or NULL
+ * (all degrees one: Eq. 1). */
+typedef struct ckv_layer_view {
+  const void* k;
+  const void* v;
+  const float* logdeg;
+  int64_t len;
+  int64_t cap;
+} ckv_layer_view;
+
+/* Host-only: workspace bytes of ckv_decode_attn (split partials). */
+size_t ckv_decode_workspace_bytes(int32_t Bz, int32_t H, int32_t G, int32_t D, int64_t max_len);
+
+/* Eq. 3 / Algorithm 1 decoding branch: out = softmax(q K^T * scale + log N) V for one layer and
+ * a batch of Bz sequences.  views_dev: device array [Bz]; q, out: [Bz, H*G, D] in `dtype`;
+ * query head j reads KV head j / G; G <= 8.  max_len (host): an upper bound on every
+ * views_dev[b].len, used to size the grid.  A sequence with len 0 gets zeros. */
+int ckv_decode_attn(const ckv_layer_view* views_dev, int32_t Bz, int32_t H, int32_t G, int32_t D, int32_t dtype,
+                    const void* q, void* out, float scale, int64_t max_len, void* workspace,
+                    size_t workspace_bytes, void* cuda_stream);
+
+/* Host-only: a static string for a ckv_status. */
+const char* ckv_status_string(int status);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* CKV_H_ */

@@ -1,0 +1,194 @@
+"""ctypes binding of the ckv C ABI (include/ckv.h): argument marshalling only.
+
+Every function takes torch tensors that live on the GPU, passes their pointers to the
+library and returns; all arithmetic runs in the CUDA kernels.  There is no CPU fallback:
+if libckv.so is missing or cannot be loaded the import of this module fails.
+"""
+from __future__ import annotations
+
+import ctypes as C
+import os
+from dataclasses import dataclass
+
+import torch
+
+from . import build as _build
+
+F32, BF16 = 0, 1
+SELECT_GLOBAL, SELECT_CHUNK = 0, 1
+OK = 0
+
+EXPORTS = ["ckv_compress_plan", "ckv_workspace_bytes", "ckv_compress_prefill", "ckv_compress_append",
+           "ckv_decode_workspace_bytes", "ckv_decode_attn", "ckv_status_string"]
+
+
+class CkvCache(C.Structure):
+    _fields_ = [("k", C.c_void_p), ("v", C.c_void_p), ("deg", C.c_void_p), ("logdeg", C.c_void_p),
+                ("L", C.c_int32), ("H", C.c_int32), ("D", C.c_int32), ("dtype", C.c_int32),
+                ("cap", C.c_int64), ("len", C.c_int64), ("pending", C.c_int64)]
+
+
+class CkvParams(C.Structure):
+    _fields_ = [("chunk", C.c_int32), ("n_sink", C.c_int32), ("n_recent", C.c_int32), ("n_rounds_max", C.c_int32),
+                ("r_init", C.c_float), ("r_decay", C.c_float), ("r_min", C.c_float), ("select", C.c_int32),
+                ("budget", C.c_int64)]
+
+
+class CkvLayerView(C.Structure):
+    _fields_ = [("k", C.c_void_p), ("v", C.c_void_p), ("logdeg", C.c_void_p), ("len", C.c_int64), ("cap", C.c_int64)]
+
+
+def _load():
+    path = _build.LIB
+    if not os.path.exists(path):
+        path = _build.build()
+    lib = C.CDLL(path)
+    lib.ckv_status_string.restype = C.c_char_p
+    lib.ckv_status_string.argtypes = [C.c_int]
+    lib.ckv_compress_plan.restype = C.c_int
+    lib.ckv_compress_plan.argtypes = [C.c_int64, C.POINTER(CkvParams), C.POINTER(C.c_int64), C.POINTER(C.c_int64),
+                                      C.POINTER(C.c_int64)]
+    lib.ckv_workspace_bytes.restype = C.c_size_t
+    lib.ckv_workspace_bytes.argtypes = [C.POINTER(CkvCache), C.POINTER(CkvParams)]
+    lib.ckv_compress_prefill.restype = C.c_int
+    lib.ckv_compress_prefill.argtypes = [C.POINTER(CkvCache), C.POINTER(CkvCache), C.POINTER(CkvParams), C.c_void_p,
+                                         C.c_void_p, C.c_size_t, C.c_void_p, C.POINTER(C.c_int64)]
+    lib.ckv_compress_append.restype = C.c_int
+    lib.ckv_compress_append.argtypes = [C.POINTER(CkvCache), C.c_void_p, C.c_void_p, C.c_int32, C.POINTER(CkvParams),
+                                        C.c_void_p, C.c_size_t, C.c_void_p]
+    lib.ckv_decode_workspace_bytes.restype = C.c_size_t
+    lib.ckv_decode_workspace_bytes.argtypes = [C.c_int32, C.c_int32, C.c_int32, C.c_int32, C.c_int64]
+    lib.ckv_decode_attn.restype = C.c_int
+    lib.ckv_decode_attn.argtypes = [C.c_void_p, C.c_int32, C.c_int32, C.c_int32, C.c_int32, C.c_int32, C.c_void_p,
+                                    C.c_void_p, C.c_float, C.c_int64, C.c_void_p, C.c_size_t, C.c_void_p]
+    return lib
+
+
+lib = _load()
+
+
+class CkvError(RuntimeError):
+    def __init__(self, status: int):
+        self.status = status
+        super().__init__(f"ckv status {status}: {lib.ckv_status_string(status).decode()}")
+
+
+def _check(status: int):
+    if status != OK:
+        raise CkvError(status)
+
+
+def dtype_code(t: torch.dtype) -> int:
+    return {torch.float32: F32, torch.bfloat16: BF16}[t]
+
+
+@dataclass
+class Params:
+    """Mirror of ckv_params.  Ratios are stored as float32, like the C struct."""
+    chunk: int = 256
+    n_sink: int = 16
+    n_recent: int = 64
+    n_rounds_max: int = 8
+    r_init: float = 0.8
+    r_decay: float = 0.2
+    r_min: float = 0.2
+    select: int = SELECT_GLOBAL
+    budget: int = 0
+
+    def c(self) -> CkvParams:
+        return CkvParams(self.chunk, self.n_sink, self.n_recent, self.n_rounds_max, self.r_init, self.r_decay,
+                         self.r_min, self.select, self.budget)
+
+    def as_float32(self):
+        """(r_init, r_decay, r_min) as the float32 values the library sees."""
+        p = self.c()
+        return float(p.r_init), float(p.r_decay), float(p.r_min)
+
+
+def compress_plan(length: int, params: Params):
+    """ckv_compress_plan: (final length, rounds, destination capacity needed).  Host only."""
+    out_len, rounds, cap = C.c_int64(), C.c_int64(), C.c_int64()
+    _check(lib.ckv_compress_plan(length, C.byref(params.c()), C.byref(out_len), C.byref(rounds), C.byref(cap)))
+    return out_len.value, rounds.value, cap.value
+
+
+class Cache:
+    """One sequence's cache on the GPU: k, v [L, H, cap, D]; deg int32 and logdeg fp32 [L, H, cap]."""
+
+    def __init__(self, k: torch.Tensor, v: torch.Tensor, deg: torch.Tensor | None, logdeg: torch.Tensor | None,
+                 length: int, pending: int = 0):
+        assert k.is_contiguous() and v.is_contiguous() and k.shape == v.shape and k.dim() == 4
+        self.k, self.v, self.deg, self.logdeg = k, v, deg, logdeg
+        self.len, self.pending = length, pending
+
+    @classmethod
+    def empty(cls, L, H, cap, D, dtype, device="cuda", with_logdeg=True):
+        k = torch.empty((L, H, cap, D), dtype=dtype, device=device)
+        v = torch.empty_like(k)
+        deg = torch.zeros((L, H, cap), dtype=torch.int32, device=device)
+        logdeg = torch.zeros((L, H, cap), dtype=torch.float32, device=device) if with_logdeg else None
+        return cls(k, v, deg, logdeg, 0)
+
+    @property
+    def cap(self):
+        return self.k.shape[2]
+
+    def c(self) -> CkvCache:
+        L, H, cap, D = self.k.shape
+        return CkvCache(self.k.data_ptr(), self.v.data_ptr(),
+                        self.deg.data_ptr() if self.deg is not None else None,
+                        self.logdeg.data_ptr() if self.logdeg is not None else None,
+                        L, H, D, dtype_code(self.k.dtype), cap, self.len, self.pending)
+
+
+def _stream_ptr():
+    return C.c_void_p(torch.cuda.current_stream().cuda_stream)
+
+
+def workspace_bytes(cache: Cache, params: Params) -> int:
+    return lib.ckv_workspace_bytes(C.byref(cache.c()), C.byref(params.c()))
+
+
+def compress_prefill(src: Cache, dst: Cache, params: Params, workspace: torch.Tensor, assign: torch.Tensor | None = None):
+    """ckv_compress_prefill on the current stream.  Returns the number of rounds; dst.len is updated."""
+    cs, cd, rounds = src.c(), dst.c(), C.c_int64()
+    _check(lib.ckv_compress_prefill(C.byref(cs), C.byref(cd), C.byref(params.c()),
+                                    assign.data_ptr() if assign is not None else None,
+                                    workspace.data_ptr(), workspace.numel() * workspace.element_size(), _stream_ptr(),
+                                    C.byref(rounds)))
+    dst.len, dst.pending = cd.len, cd.pending
+    return rounds.value
+
+
+def compress_append(cache: Cache, k_new: torch.Tensor, v_new: torch.Tensor, params: Params, workspace: torch.Tensor):
+    """ckv_compress_append on the current stream; cache.len / cache.pending are updated."""
+    assert k_new.is_contiguous() and v_new.is_contiguous() and k_new.shape == v_new.shape
+    cc = cache.c()
+    _check(lib.ckv_compress_append(C.byref(cc), k_new.data_ptr(), v_new.data_ptr(), k_new.shape[2], C.byref(params.c()),
+                                   workspace.data_ptr(), workspace.numel() * workspace.element_size(), _stream_ptr()))
+    cache.len, cache.pending = cc.len, cc.pending
+
+
+def layer_views(caches, layer: int, device="cuda") -> torch.Tensor:
+    """Device array of ckv_layer_view for one layer of a batch of caches (as an int64 tensor of 5 words each)."""
+    rows = []
+    for c in caches:
+        L, H, cap, D = c.k.shape
+        es = c.k.element_size()
+        off = layer * H * cap
+        rows.append([c.k.data_ptr() + off * D * es, c.v.data_ptr() + off * D * es,
+                     (c.logdeg.data_ptr() + off * 4) if c.logdeg is not None else 0, c.len, cap])
+    return torch.tensor(rows, dtype=torch.int64).to(device)
+
+
+def decode_workspace_bytes(Bz, H, G, D, max_len) -> int:
+    return lib.ckv_decode_workspace_bytes(Bz, H, G, D, max_len)
+
+
+def decode_attn(views: torch.Tensor, H: int, G: int, q: torch.Tensor, out: torch.Tensor, scale: float, max_len: int,
+                workspace: torch.Tensor):
+    """ckv_decode_attn on the current stream.  views: layer_views(...); q, out: [Bz, H*G, D]."""
+    Bz, HG, D = q.shape
+    assert HG == H * G and q.is_contiguous() and out.is_contiguous()
+    _check(lib.ckv_decode_attn(views.data_ptr(), Bz, H, G, D, dtype_code(q.dtype), q.data_ptr(), out.data_ptr(), scale,
+                               max_len, workspace.data_ptr(), workspace.numel() * workspace.element_size(), _stream_ptr()))

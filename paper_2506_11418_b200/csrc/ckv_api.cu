@@ -1,0 +1,432 @@
+// Host side of the C ABI: argument checks, the round schedule of Algorithm 1 / Eq. 4, workspace
+// layout, and the launch sequences.  No device memory is allocated here.
+#include <cmath>
+#include <cstring>
+#include <vector>
+
+#include "../../include/ckv.h"
+#include "ckv_internal.h"
+
+namespace ckv {
+namespace {
+
+struct RoundPlan {
+  int64_t s_in, s_out, lo, hi;
+  int32_t n_chunks;
+  int64_t n_edges;  // A tokens that have a B candidate
+  int64_t M;        // merges per (layer, head)
+  int32_t m_full, m_tail;
+  int32_t mode;     // RoundMode, or -1: nothing merges (verbatim copy)
+};
+
+inline size_t align_up(size_t x, size_t a = 256) { return (x + a - 1) / a * a; }
+
+int check_params(const ckv_params* p) {
+  if (!p) return CKV_ERR_INVALID_ARG;
+  if (p->chunk < 2 || (p->chunk & 1)) return CKV_ERR_INVALID_ARG;
+  if (p->n_sink < 0 || p->n_recent < 0 || p->n_rounds_max < 0 || p->budget < 0) return CKV_ERR_INVALID_ARG;
+  if (!(p->r_init >= 0.f && p->r_init <= 1.f) || !(p->r_decay >= 0.f) || !(p->r_min >= 0.f && p->r_min <= 1.f))
+    return CKV_ERR_INVALID_ARG;
+  if (p->select != CKV_SELECT_GLOBAL && p->select != CKV_SELECT_CHUNK) return CKV_ERR_INVALID_ARG;
+  if (p->chunk > 256) return CKV_ERR_UNSUPPORTED;
+  return CKV_OK;
+}
+
+inline int64_t floor_ratio(double r, int64_t n) { return (int64_t)std::floor(r * (double)n + 1e-9); }
+
+// Algorithm 1's `while s > B` loop with Eq. 4: everything a round does is a function of lengths.
+int plan_rounds(int64_t len, const ckv_params& p, std::vector<RoundPlan>& plan) {
+  plan.clear();
+  int64_t s = len;
+  for (int j = 0; j < p.n_rounds_max && (p.budget == 0 || s > p.budget); ++j) {
+    const double r = std::fmax((double)p.r_init - (double)j * (double)p.r_decay, (double)p.r_min);
+    RoundPlan rp{};
+    rp.s_in = s;
+    rp.lo = std::min<int64_t>(p.n_sink, s);
+    rp.hi = std::max<int64_t>(rp.lo, s - p.n_recent);
+    const int64_t mid = rp.hi - rp.lo;
+    const int c = p.chunk;
+    const int64_t n_full = mid >= 2 ? mid / c : 0;
+    const int tail = mid >= 2 ? (int)(mid % c) : 0;
+    rp.n_chunks = (int32_t)(n_full + (tail > 0 ? 1 : 0));
+    const int64_t tail_edges = tail >= 2 ? (tail + 1) / 2 : 0;
+    rp.n_edges = n_full * (c / 2) + tail_edges;
+    if (p.select == CKV_SELECT_GLOBAL) {
+      rp.M = floor_ratio(r, rp.n_edges);
+      if (p.budget > 0) rp.M = std::min<int64_t>(rp.M, s - p.budget);
+      rp.mode = rp.M == 0 ? -1 : (rp.M == rp.n_edges ? kModeAll : kModeExternal);
+      rp.m_full = c / 2;
+      rp.m_tail = (int32_t)tail_edges;
+    } else {
+      rp.m_full = (int32_t)floor_ratio(r, c / 2);
+      rp.m_tail = (int32_t)floor_ratio(r, tail_edges);
+      rp.M = n_full * rp.m_full + rp.m_tail;
+      rp.mode = rp.M == 0 ? -1 : ((rp.m_full == c / 2 && rp.m_tail == tail_edges) ? kModeAll : kModeChunkTopM);
+    }
+    rp.s_out = s - rp.M;
+    if (rp.M == 0 && p.budget > 0) return CKV_ERR_NO_PROGRESS;
+    plan.push_back(rp);
+    s = rp.s_out;
+  }
+  return CKV_OK;
+}
+
+// Which buffer each round writes: the last one lands in dst, the others alternate with tmp.
+inline bool round_targets_dst(size_t j, size_t R) { return ((R - 1 - j) & 1) == 0; }
+
+struct Workspace {
+  size_t tmp_k, tmp_v, tmp_deg, tmp_logdeg;  // offsets; tmp cache [LH, tmp_cap, D]
+  int64_t tmp_cap;
+  size_t edge_sim, edge_b, sel, chunk_off;
+  int64_t edge_stride;
+  size_t assign_step;
+  int64_t assign_stride;
+  size_t total;
+};
+
+Workspace layout_workspace(int64_t LH, int D, int esize, int chunk, const std::vector<RoundPlan>& plan,
+                           bool want_assign) {
+  Workspace w{};
+  const size_t R = plan.size();
+  int64_t max_chunks = 0, max_sin = 0;
+  for (size_t j = 0; j < R; ++j) {
+    if (!round_targets_dst(j, R)) w.tmp_cap = std::max(w.tmp_cap, plan[j].s_out);
+    if (plan[j].mode == kModeExternal) max_chunks = std::max<int64_t>(max_chunks, plan[j].n_chunks);
+    max_sin = std::max(max_sin, plan[j].s_in);
+  }
+  size_t off = 0;
+  auto take = [&off](size_t bytes) {
+    const size_t at = off;
+    off += align_up(bytes);
+    return at;
+  };
+  w.tmp_k = take((size_t)LH * w.tmp_cap * D * esize);
+  w.tmp_v = take((size_t)LH * w.tmp_cap * D * esize);
+  w.tmp_deg = take((size_t)LH * w.tmp_cap * 4);
+  w.tmp_logdeg = take((size_t)LH * w.tmp_cap * 4);
+  w.edge_stride = max_chunks * (chunk / 2);
+  w.edge_sim = take((size_t)LH * w.edge_stride * 4);
+  w.edge_b = take((size_t)LH * w.edge_stride * 4);
+  w.sel = take((size_t)LH * w.edge_stride);
+  w.chunk_off = take((size_t)LH * max_chunks * 4);
+  w.assign_stride = (want_assign && R >= 2) ? max_sin : 0;
+  w.assign_step = take((size_t)LH * w.assign_stride * 4);
+  w.total = off + 256;
+  return w;
+}
+
+inline int esize_of(int dtype) { return dtype == CKV_F32 ? 4 : 2; }
+
+int check_cache_shape(const ckv_cache* c, bool with_len = true) {
+  if (!c) return CKV_ERR_INVALID_ARG;
+  if (c->L <= 0 || c->H <= 0 || c->D <= 0 || c->cap < 0) return CKV_ERR_INVALID_ARG;
+  if (with_len && (c->len < 0 || c->len > c->cap || c->pending < 0 || c->pending > c->len)) return CKV_ERR_INVALID_ARG;
+  if (c->dtype != CKV_F32 && c->dtype != CKV_BF16) return CKV_ERR_INVALID_ARG;
+  if ((int64_t)c->L * c->H > 65535) return CKV_ERR_UNSUPPORTED;
+  if (c->D != 128) return CKV_ERR_UNSUPPORTED;
+  return CKV_OK;
+}
+
+inline bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+
+inline bool overlaps(const void* a, size_t an, const void* b, size_t bn) {
+  const uintptr_t x = reinterpret_cast<uintptr_t>(a), y = reinterpret_cast<uintptr_t>(b);
+  return an && bn && x < y + bn && y < x + an;
+}
+
+struct Buf {  // one cache buffer a round reads or writes
+  void* k;
+  void* v;
+  int32_t* deg;
+  float* logdeg;
+  int64_t cap;
+};
+
+// One clustering round src -> dst (Sec. 5.2, Sec. 5.3, Eq. 5), sinks and recent tokens copied verbatim.
+cudaError_t run_round(const RoundPlan& rp, const Buf& src, const Buf& dst, int LH, int D, int dtype, int chunk,
+                      int32_t* assign, int64_t assign_stride, const Workspace& w, unsigned char* ws, cudaStream_t st) {
+  cudaError_t e;
+  CopyArgs c{};
+  c.k_src = src.k; c.v_src = src.v; c.deg_src = src.deg;
+  c.k_dst = dst.k; c.v_dst = dst.v; c.deg_dst = dst.deg; c.logdeg_dst = dst.logdeg;
+  c.assign = assign; c.assign_stride = assign_stride;
+  c.src_cap = src.cap; c.dst_cap = dst.cap; c.LH = LH;
+  if (rp.mode < 0) {  // nothing merges: the round is the identity
+    c.src_off = 0; c.dst_off = 0; c.count = rp.s_in;
+    return launch_copy(c, dtype, D, st);
+  }
+  c.src_off = 0; c.dst_off = 0; c.count = rp.lo;
+  if ((e = launch_copy(c, dtype, D, st)) != cudaSuccess) return e;
+  c.src_off = rp.hi; c.dst_off = rp.hi - rp.M; c.count = rp.s_in - rp.hi;
+  if ((e = launch_copy(c, dtype, D, st)) != cudaSuccess) return e;
+
+  RoundArgs a{};
+  a.k_src = src.k; a.v_src = src.v; a.deg_src = src.deg;
+  a.k_dst = dst.k; a.v_dst = dst.v; a.deg_dst = dst.deg; a.logdeg_dst = dst.logdeg;
+  a.assign = assign; a.assign_stride = assign_stride;
+  a.src_cap = src.cap; a.dst_cap = dst.cap;
+  a.lo = rp.lo; a.hi = rp.hi;
+  a.chunk = chunk; a.n_chunks = rp.n_chunks;
+  a.m_full = rp.m_full; a.m_tail = rp.m_tail;
+  a.out_stride = chunk - rp.m_full;
+  a.LH = LH;
+  a.edge_stride = (int64_t)rp.n_chunks * (chunk / 2);
+  if (rp.mode == kModeExternal) {
+    a.edge_sim = reinterpret_cast<float*>(ws + w.edge_sim);
+    a.edge_b = reinterpret_cast<int32_t*>(ws + w.edge_b);
+    a.sel = ws + w.sel;
+    a.chunk_out_off = reinterpret_cast<int32_t*>(ws + w.chunk_off);
+    a.mode = kModeMatchOnly;
+    if ((e = launch_round(a, dtype, D, st)) != cudaSuccess) return e;
+    SelectArgs s{};
+    s.edge_sim = a.edge_sim; s.sel = a.sel; s.chunk_out_off = a.chunk_out_off;
+    s.edge_stride = a.edge_stride; s.M = rp.M; s.lo = rp.lo; s.chunk = chunk; s.n_chunks = rp.n_chunks; s.LH = LH;
+    if ((e = launch_select(s, st)) != cudaSuccess) return e;
+  }
+  a.mode = rp.mode;
+  return launch_round(a, dtype, D, st);
+}
+
+// Runs the planned rounds from `src` into `dst` (ping-pong through the workspace's tmp cache).
+int run_plan(const std::vector<RoundPlan>& plan, const Buf& src, const Buf& dst, int64_t src_len, int LH, int D,
+             int dtype, int chunk, int32_t* assign, Workspace& w, unsigned char* ws, cudaStream_t st) {
+  const size_t R = plan.size();
+  cudaError_t e;
+  if (R == 0) {
+    RoundPlan id{};
+    id.s_in = src_len;
+    id.mode = -1;
+    e = run_round(id, src, dst, LH, D, dtype, chunk, assign, src_len, w, ws, st);
+    return e == cudaSuccess ? CKV_OK : CKV_ERR_CUDA;
+  }
+  Buf tmp{ws + w.tmp_k, ws + w.tmp_v, reinterpret_cast<int32_t*>(ws + w.tmp_deg),
+          reinterpret_cast<float*>(ws + w.tmp_logdeg), w.tmp_cap};
+  Buf cur = src;
+  for (size_t j = 0; j < R; ++j) {
+    const Buf& target = round_targets_dst(j, R) ? dst : tmp;
+    int32_t* step = nullptr;
+    int64_t step_stride = 0;
+    if (assign) {
+      if (j == 0) {
+        step = assign;
+        step_stride = src_len;
+      } else {
+        step = reinterpret_cast<int32_t*>(ws + w.assign_step);
+        step_stride = w.assign_stride;
+      }
+    }
+    e = run_round(plan[j], cur, target, LH, D, dtype, chunk, step, step_stride, w, ws, st);
+    if (e != cudaSuccess) return CKV_ERR_CUDA;
+    if (assign && j > 0) {
+      e = launch_compose_assign(assign, step, src_len, step_stride, LH, st);
+      if (e != cudaSuccess) return CKV_ERR_CUDA;
+    }
+    cur = target;
+  }
+  return CKV_OK;
+}
+
+// Capacity dst needs: everything a round writes into it.
+int64_t dst_cap_needed(const std::vector<RoundPlan>& plan, int64_t len) {
+  const size_t R = plan.size();
+  if (R == 0) return len;
+  int64_t need = 0;
+  for (size_t j = 0; j < R; ++j)
+    if (round_targets_dst(j, R)) need = std::max(need, plan[j].s_out);
+  return need;
+}
+
+ckv_params window_params(const ckv_params& p) {
+  ckv_params wp = p;
+  wp.n_sink = 0;
+  wp.n_recent = 0;
+  return wp;
+}
+
+}  // namespace
+}  // namespace ckv
+
+using namespace ckv;
+
+extern "C" {
+
+const char* ckv_status_string(int status) {
+  switch (status) {
+    case CKV_OK: return "ok";
+    case CKV_ERR_INVALID_ARG: return "invalid argument";
+    case CKV_ERR_ALIGNMENT: return "pointer not 16-byte aligned";
+    case CKV_ERR_CAPACITY: return "destination capacity too small";
+    case CKV_ERR_WORKSPACE: return "workspace missing or too small";
+    case CKV_ERR_NO_PROGRESS: return "ratio schedule merges nothing but the budget is not met";
+    case CKV_ERR_UNSUPPORTED: return "unsupported shape or size";
+    case CKV_ERR_CUDA: return "CUDA runtime error";
+    default: return "unknown status";
+  }
+}
+
+int ckv_compress_plan(int64_t len, const ckv_params* params, int64_t* out_len, int64_t* rounds,
+                      int64_t* dst_cap) {
+  int st = check_params(params);
+  if (st != CKV_OK) return st;
+  if (len < 0) return CKV_ERR_INVALID_ARG;
+  std::vector<RoundPlan> plan;
+  if ((st = plan_rounds(len, *params, plan)) != CKV_OK) return st;
+  if (out_len) *out_len = plan.empty() ? len : plan.back().s_out;
+  if (rounds) *rounds = (int64_t)plan.size();
+  if (dst_cap) *dst_cap = dst_cap_needed(plan, len);
+  return CKV_OK;
+}
+
+size_t ckv_workspace_bytes(const ckv_cache* shape, const ckv_params* params) {
+  if (check_params(params) != CKV_OK || check_cache_shape(shape) != CKV_OK) return 0;
+  const int64_t LH = (int64_t)shape->L * shape->H;
+  const int es = esize_of(shape->dtype);
+  std::vector<RoundPlan> plan;
+  size_t need = 256;
+  // prefill over the current length (an unreachable budget is reported by the call itself)
+  if (plan_rounds(shape->len, *params, plan) == CKV_OK) {
+    need = std::max(need, layout_workspace(LH, shape->D, es, params->chunk, plan, true).total);
+  }
+  // append: one window of `chunk` tokens, with a tmp window for odd round counts
+  const ckv_params wp = window_params(*params);
+  if (plan_rounds(params->chunk, wp, plan) == CKV_OK) {
+    const size_t win = align_up((size_t)LH * params->chunk * shape->D * es) * 2 + align_up((size_t)LH * params->chunk * 4) * 2;
+    need = std::max(need, layout_workspace(LH, shape->D, es, params->chunk, plan, false).total + win);
+  }
+  return need;
+}
+
+int ckv_compress_prefill(const ckv_cache* src, ckv_cache* dst, const ckv_params* params, int32_t* assign,
+                         void* workspace, size_t workspace_bytes, void* cuda_stream, int64_t* rounds_done) {
+  int st;
+  if ((st = check_params(params)) != CKV_OK) return st;
+  if ((st = check_cache_shape(src)) != CKV_OK) return st;
+  if ((st = check_cache_shape(dst, false)) != CKV_OK) return st;
+  if (src->L != dst->L || src->H != dst->H || src->D != dst->D || src->dtype != dst->dtype) return CKV_ERR_INVALID_ARG;
+  if (!src->k || !src->v || !dst->k || !dst->v || !dst->deg) return CKV_ERR_INVALID_ARG;
+  if (!aligned16(src->k) || !aligned16(src->v) || !aligned16(dst->k) || !aligned16(dst->v)) return CKV_ERR_ALIGNMENT;
+  const int64_t LH = (int64_t)src->L * src->H;
+  const int es = esize_of(src->dtype);
+  const size_t src_bytes = (size_t)LH * src->cap * src->D * es, dst_bytes = (size_t)LH * dst->cap * dst->D * es;
+  if (overlaps(src->k, src_bytes, dst->k, dst_bytes) || overlaps(src->v, src_bytes, dst->v, dst_bytes) ||
+      overlaps(src->k, src_bytes, dst->v, dst_bytes) || overlaps(src->v, src_bytes, dst->k, dst_bytes))
+    return CKV_ERR_INVALID_ARG;
+  std::vector<RoundPlan> plan;
+  if ((st = plan_rounds(src->len, *params, plan)) != CKV_OK) return st;
+  if (dst->cap < dst_cap_needed(plan, src->len)) return CKV_ERR_CAPACITY;
+  Workspace w = layout_workspace(LH, src->D, es, params->chunk, plan, assign != nullptr);
+  const size_t need = w.total;
+  if (!workspace || workspace_bytes < need || !aligned16(workspace)) return CKV_ERR_WORKSPACE;
+  if (overlaps(workspace, need, dst->k, dst_bytes) || overlaps(workspace, need, dst->v, dst_bytes) ||
+      overlaps(workspace, need, src->k, src_bytes) || overlaps(workspace, need, src->v, src_bytes))
+    return CKV_ERR_INVALID_ARG;
+
+  const Buf s{src->k, src->v, src->deg, src->logdeg, src->cap};
+  const Buf d{dst->k, dst->v, dst->deg, dst->logdeg, dst->cap};
+  st = run_plan(plan, s, d, src->len, (int)LH, src->D, src->dtype, params->chunk, assign, w,
+                static_cast<unsigned char*>(workspace), static_cast<cudaStream_t>(cuda_stream));
+  if (st != CKV_OK) return st;
+  dst->len = plan.empty() ? src->len : plan.back().s_out;
+  dst->pending = 0;
+  if (rounds_done) *rounds_done = (int64_t)plan.size();
+  return CKV_OK;
+}
+
+int ckv_compress_append(ckv_cache* cache, const void* k_new, const void* v_new, int32_t t_new,
+                        const ckv_params* params, void* workspace, size_t workspace_bytes, void* cuda_stream) {
+  int st;
+  if ((st = check_params(params)) != CKV_OK) return st;
+  if ((st = check_cache_shape(cache)) != CKV_OK) return st;
+  if (t_new < 0 || (t_new > 0 && (!k_new || !v_new))) return CKV_ERR_INVALID_ARG;
+  if (!cache->k || !cache->v || !cache->deg) return CKV_ERR_INVALID_ARG;
+  if (!aligned16(cache->k) || !aligned16(cache->v) || !aligned16(k_new) || !aligned16(v_new)) return CKV_ERR_ALIGNMENT;
+  if (cache->pending >= params->chunk) return CKV_ERR_INVALID_ARG;
+  const int64_t LH = (int64_t)cache->L * cache->H;
+  const int D = cache->D, es = esize_of(cache->dtype), c = params->chunk;
+  const ckv_params wp = window_params(*params);
+  std::vector<RoundPlan> plan;
+  if ((st = plan_rounds(c, wp, plan)) != CKV_OK) return st;
+  const int64_t win_out = plan.empty() ? c : plan.back().s_out;
+
+  // host-side walk first: capacity must hold every intermediate state
+  {
+    int64_t len = cache->len, pend = cache->pending, peak = len;
+    for (int32_t done = 0; done < t_new;) {
+      const int32_t take = (int32_t)std::min<int64_t>(t_new - done, c - pend);
+      len += take; pend += take; done += take;
+      peak = std::max(peak, len);
+      if (pend == c) { len -= c - win_out; pend = 0; }
+    }
+    if (peak > cache->cap) return CKV_ERR_CAPACITY;
+  }
+  Workspace w = layout_workspace(LH, D, es, c, plan, false);
+  const size_t base = w.total;
+  const size_t win_kv = align_up((size_t)LH * c * D * es), win_dg = align_up((size_t)LH * c * 4);
+  if (!workspace || workspace_bytes < base + 2 * win_kv + 2 * win_dg || !aligned16(workspace)) return CKV_ERR_WORKSPACE;
+  unsigned char* ws = static_cast<unsigned char*>(workspace);
+  const Buf stage{ws + base, ws + base + win_kv, reinterpret_cast<int32_t*>(ws + base + 2 * win_kv),
+                  reinterpret_cast<float*>(ws + base + 2 * win_kv + win_dg), c};
+  cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
+
+  for (int32_t done = 0; done < t_new;) {
+    const int32_t take = (int32_t)std::min<int64_t>(t_new - done, c - cache->pending);
+    CopyArgs cp{};  // K = [K, k], V = [V, v], N = [N, 1]
+    cp.k_src = k_new; cp.v_src = v_new; cp.deg_src = nullptr;
+    cp.k_dst = cache->k; cp.v_dst = cache->v; cp.deg_dst = cache->deg; cp.logdeg_dst = cache->logdeg;
+    cp.src_cap = t_new; cp.dst_cap = cache->cap; cp.src_off = done; cp.dst_off = cache->len; cp.count = take;
+    cp.LH = (int)LH;
+    if (launch_copy(cp, cache->dtype, D, stream) != cudaSuccess) return CKV_ERR_CUDA;
+    cache->len += take;
+    cache->pending += take;
+    done += take;
+    if (cache->pending == c && !plan.empty()) {
+      // cluster the completed window: copy it aside, then run the rounds back into its place
+      const int64_t w0 = cache->len - c;
+      CopyArgs out{};
+      out.k_src = cache->k; out.v_src = cache->v; out.deg_src = cache->deg;
+      out.k_dst = stage.k; out.v_dst = stage.v; out.deg_dst = stage.deg; out.logdeg_dst = stage.logdeg;
+      out.src_cap = cache->cap; out.dst_cap = c; out.src_off = w0; out.dst_off = 0; out.count = c; out.LH = (int)LH;
+      if (launch_copy(out, cache->dtype, D, stream) != cudaSuccess) return CKV_ERR_CUDA;
+      // the window's destination is a view of the cache that starts at w0
+      const Buf dstw{static_cast<unsigned char*>(cache->k) + (size_t)w0 * D * es,
+                     static_cast<unsigned char*>(cache->v) + (size_t)w0 * D * es, cache->deg + w0,
+                     cache->logdeg ? cache->logdeg + w0 : nullptr, cache->cap};
+      st = run_plan(plan, stage, dstw, c, (int)LH, D, cache->dtype, c, nullptr, w, ws, stream);
+      if (st != CKV_OK) return st;
+      cache->len = w0 + win_out;
+    }
+    if (cache->pending == c) cache->pending = 0;
+  }
+  return CKV_OK;
+}
+
+size_t ckv_decode_workspace_bytes(int32_t Bz, int32_t H, int32_t G, int32_t D, int64_t max_len) {
+  if (Bz <= 0 || H <= 0 || G <= 0 || D <= 0 || max_len < 0) return 0;
+  const int64_t max_splits = std::max<int64_t>(1, (max_len + 127) / 128);
+  const int64_t want = (4 * 148 + (int64_t)Bz * H - 1) / ((int64_t)Bz * H);
+  const int64_t n_splits = std::max<int64_t>(1, std::min(want, max_splits));
+  return align_up((size_t)Bz * H * G * n_splits * (D + 4) * 4) + 256;
+}
+
+int ckv_decode_attn(const ckv_layer_view* views_dev, int32_t Bz, int32_t H, int32_t G, int32_t D, int32_t dtype,
+                    const void* q, void* out, float scale, int64_t max_len, void* workspace, size_t workspace_bytes,
+                    void* cuda_stream) {
+  if (!views_dev || !q || !out || Bz <= 0 || H <= 0 || G <= 0 || max_len < 0) return CKV_ERR_INVALID_ARG;
+  if (dtype != CKV_F32 && dtype != CKV_BF16) return CKV_ERR_INVALID_ARG;
+  if (D != 128 || G > 8 || H > 65535 || Bz > 65535) return CKV_ERR_UNSUPPORTED;
+  if (!aligned16(q) || !aligned16(out)) return CKV_ERR_ALIGNMENT;
+  const size_t need = ckv_decode_workspace_bytes(Bz, H, G, D, max_len);
+  if (!workspace || workspace_bytes < need || !aligned16(workspace)) return CKV_ERR_WORKSPACE;
+  const int64_t max_splits = std::max<int64_t>(1, (max_len + 127) / 128);
+  const int64_t want = (4 * 148 + (int64_t)Bz * H - 1) / ((int64_t)Bz * H);
+  DecodeArgs a{};
+  a.views = views_dev; a.q = q; a.out = out;
+  a.partial = static_cast<float*>(workspace);
+  a.Bz = Bz; a.H = H; a.G = G;
+  a.n_splits = (int32_t)std::max<int64_t>(1, std::min(want, max_splits));
+  a.span = std::max<int64_t>(128, ((max_len + a.n_splits - 1) / a.n_splits + 127) / 128 * 128);
+  a.scale = scale;
+  return launch_decode(a, dtype, D, static_cast<cudaStream_t>(cuda_stream)) == cudaSuccess ? CKV_OK : CKV_ERR_CUDA;
+}
+
+}  // extern "C"

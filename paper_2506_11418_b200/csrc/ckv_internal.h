@@ -1,0 +1,87 @@
+// Internal interfaces between the host driver (ckv_api.cu) and the kernel files.
+#pragma once
+
+#include <cuda_runtime.h>
+#include <stddef.h>
+#include <stdint.h>
+
+namespace ckv {
+
+enum RoundMode : int32_t {
+  kModeAll = 0,       // every edge is merged (ratio 1)
+  kModeChunkTopM = 1, // the best m edges of each chunk are merged
+  kModeExternal = 2,  // edge targets, selection flags and output offsets come from global memory
+  kModeMatchOnly = 3  // write each A token's edge (similarity, target) and stop
+};
+
+// One clustering round over the middle region [lo, hi) of every (layer, head) slab.
+struct RoundArgs {
+  const void* k_src;
+  const void* v_src;
+  const int32_t* deg_src;  // may be null: all ones
+  void* k_dst;
+  void* v_dst;
+  int32_t* deg_dst;
+  float* logdeg_dst;       // may be null
+  int32_t* assign;         // may be null; [LH, assign_stride] slot of each source token, this round
+  int64_t assign_stride;
+  int64_t src_cap, dst_cap;
+  int64_t lo, hi;
+  int32_t chunk, n_chunks;
+  int32_t mode;
+  int32_t m_full, m_tail;  // kModeChunkTopM: merges in a full chunk / in the shorter last chunk
+  int64_t out_stride;      // kModeAll, kModeChunkTopM: survivors of a full chunk
+  float* edge_sim;         // [LH, edge_stride]   kModeMatchOnly writes, select kernel reads
+  int32_t* edge_b;         // [LH, edge_stride]   local offset of the edge's B token, -1 = no candidate
+  uint8_t* sel;            // [LH, edge_stride]   kModeExternal: 1 = merge this edge
+  int32_t* chunk_out_off;  // [LH, n_chunks]      kModeExternal: dst position of the chunk's first survivor
+  int64_t edge_stride;     // n_chunks * chunk / 2
+  int32_t LH;
+};
+
+// Copy `count` token rows (K, V, degree) of every slab from src_off to dst_off.
+struct CopyArgs {
+  const void* k_src;
+  const void* v_src;
+  const int32_t* deg_src;  // may be null: ones
+  void* k_dst;
+  void* v_dst;
+  int32_t* deg_dst;
+  float* logdeg_dst;       // may be null
+  int32_t* assign;         // may be null
+  int64_t assign_stride;
+  int64_t src_cap, dst_cap, src_off, dst_off, count;
+  int32_t LH;
+};
+
+struct SelectArgs {
+  const float* edge_sim;
+  uint8_t* sel;
+  int32_t* chunk_out_off;
+  int64_t edge_stride;
+  int64_t M;       // edges to merge per (layer, head)
+  int64_t lo;
+  int32_t chunk, n_chunks;
+  int32_t LH;
+};
+
+struct DecodeArgs {
+  const void* views;  // const ckv_layer_view*
+  const void* q;
+  void* out;
+  float* partial;     // [Bz, H*G, n_splits, D + 4]: out[D], max, sum, pad
+  int32_t Bz, H, G;
+  int32_t n_splits;
+  int64_t span;       // tokens per split
+  float scale;
+};
+
+cudaError_t launch_round(const RoundArgs& a, int dtype, int D, cudaStream_t st);
+cudaError_t launch_copy(const CopyArgs& a, int dtype, int D, cudaStream_t st);
+cudaError_t launch_select(const SelectArgs& a, cudaStream_t st);
+cudaError_t launch_compose_assign(int32_t* total, const int32_t* step, int64_t n_src, int64_t step_stride, int32_t LH,
+                                  cudaStream_t st);
+cudaError_t launch_decode(const DecodeArgs& a, int dtype, int D, cudaStream_t st);
+size_t round_smem_bytes(int chunk, int D);
+
+}  // namespace ckv
