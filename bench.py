@@ -1,0 +1,384 @@
+"""Benchmark of the CentroidKV hot path on B200.
+
+A step is one pass of the whole path over the Llama-3-8B-shaped prefill workload
+(32 layers, 8 KV heads, head_dim 128, 32768 tokens, bf16, chunk 64, retain 50 %):
+  1. ckv_compress_prefill  -- Chunked Soft Matching + centroid merge of the whole cache
+  2. ckv_compress_append   -- one chunk of 64 generated tokens, which triggers the window clustering
+  3. ckv_decode_attn x 32  -- one decode step over the compressed cache, all layers (32 query heads)
+`value` is the number of prefill tokens compressed per second of whole-step time, summed over ranks.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--impl reference]
+
+Under torchrun every rank runs the same per-GPU workload (weak scaling, no collective on the data
+path); time is the maximum over ranks.  `--impl reference` times the CPU oracle on a bounded sample.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import math
+import os
+import statistics
+import subprocess
+import sys
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+WORKLOAD = "llama8b_32k"
+METRIC = "compressed KV tokens/s"
+UNIT = "tokens/s"
+
+
+def measured_peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        with open(path) as f:
+            return json.load(f), "measured"
+    return {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0}, "fallback"
+
+
+# --------------------------------------------------------------------------- algorithmic bytes
+
+def compress_bytes(L, H, s, D, es, keep):
+    """Per token-vector: K and V read, the kept fraction of K and V written, degrees in (4 B) and
+    degree + log-degree out (8 B per kept slot)."""
+    per_vec = 2 * D * es + keep * 2 * D * es + 4 + keep * 8
+    return L * H * s * per_vec
+
+
+def decode_bytes(rows, D, es):
+    """Per cached token-vector: K and V rows plus the fp32 log-degree."""
+    return rows * (2 * D * es + 4)
+
+
+# --------------------------------------------------------------------------- clocks
+
+class ClockSampler:
+    FIELDS = "clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown," \
+             "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap"
+
+    def __init__(self, index: int):
+        self.proc = None
+        try:
+            self.proc = subprocess.Popen(["nvidia-smi", "-i", str(index), f"--query-gpu={self.FIELDS}",
+                                          "--format=csv,noheader,nounits", "-lms", "100"],
+                                         stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+        except OSError:
+            self.proc = None
+
+    def stop(self):
+        if self.proc is None:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+        self.proc.terminate()
+        try:
+            out, _ = self.proc.communicate(timeout=5)
+        except subprocess.TimeoutExpired:
+            self.proc.kill()
+            out, _ = self.proc.communicate()
+        sm, smax, reasons = [], None, set()
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        for line in out.strip().splitlines():
+            f = [x.strip() for x in line.split(",")]
+            if len(f) < 7:
+                continue
+            try:
+                sm.append(float(f[0]))
+                smax = float(f[1])
+            except ValueError:
+                continue
+            for n, v in zip(names, f[3:7]):
+                if v.lower().startswith("active"):
+                    reasons.add(n)
+        return {"sm_mhz": statistics.median(sm) if sm else None, "sm_max_mhz": smax, "reasons": sorted(reasons),
+                "samples": len(sm)}
+
+
+# --------------------------------------------------------------------------- CPU oracle leg
+
+def oracle_inputs(n_heads: int, seed: int = 0):
+    """`n_heads` (layer, head) slabs of the workload as fp64 arrays holding bf16-rounded values."""
+    from paper_2506_11418_b200 import synth
+
+    cfg = synth.CONFIGS[WORKLOAD]
+    s, D, c, G = cfg["s"], cfg["d"], cfg["chunk"], cfg["G"]
+    f64 = lambda t: t.float().double().numpy()
+    return dict(
+        K=f64(synth.ar1_keys(1, n_heads, s, D, cfg["rho"], cfg["mean_std"], seed=seed, dtype="bf16")),
+        V=f64(synth.normal_values(1, n_heads, s, D, seed=seed, dtype="bf16")),
+        kn=f64(synth.ar1_keys(1, n_heads, c, D, cfg["rho"], cfg["mean_std"], seed=seed + 1, dtype="bf16")),
+        vn=f64(synth.normal_values(1, n_heads, c, D, seed=seed + 1, dtype="bf16")),
+        q=f64(synth.queries(1, n_heads * G, D, seed=seed + 2, dtype="bf16"))[0],
+        n_heads=n_heads, tokens=s * n_heads / (cfg["L"] * cfg["H"]), chunk=c, D=D,
+        desc=f"{n_heads} of {cfg['L'] * cfg['H']} (layer, head) slabs of {WORKLOAD}: compress + append 64 + 1 decode step")
+
+
+def oracle_pass(x) -> float:
+    """The oracle, as it stands, over one sample: compress, append one chunk, one decode step.  Seconds."""
+    from threadpoolctl import threadpool_limits
+
+    from oracle import ckv_oracle as O
+
+    p = O.Params(chunk=x["chunk"], n_sink=0, n_recent=0, n_rounds_max=1, r_init=1.0, r_decay=0.0, r_min=1.0)
+    with threadpool_limits(limits=1):
+        t0 = time.perf_counter()
+        Ko, Vo, do, _, _ = O.compress_prefill(x["K"], x["V"], None, p, storage="bf16")
+        Ko, Vo, do, _ = O.compress_append(Ko, Vo, do, 0, x["kn"], x["vn"], p, storage="bf16")
+        O.app_attn(x["q"], Ko[0], Vo[0], do[0], 1.0 / math.sqrt(x["D"]))
+        return time.perf_counter() - t0
+
+
+def run_reference(args):
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    x = oracle_inputs(2)
+    for _ in range(min(args.warmup, 1)):
+        oracle_pass(x)
+    times = [oracle_pass(x) for _ in range(args.steps)]
+    total = sum(times)
+    value = x["tokens"] * len(times) / total
+    line = {"impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus, "steps": args.steps,
+            "warmup": args.warmup, "ms_per_step": 1e3 * total / len(times), "higher_is_better": True, "scaling": "weak",
+            "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+            "config": {"workload": WORKLOAD, "sample": x["desc"]},
+            "cpu_baseline": {"value": value, "unit": UNIT, "cores": 1, "kind": "oracle", "sample": x["desc"]},
+            "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0}}
+    print(json.dumps(line))
+
+
+# --------------------------------------------------------------------------- GPU leg
+
+def run_gpu(args):
+    import torch
+    import torch.distributed as dist
+
+    from paper_2506_11418_b200 import binding as b, synth
+
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    rank = int(os.environ.get("RANK", "0"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device; there is no CPU fallback")
+    torch.cuda.set_device(local)
+    dev = torch.device("cuda", local)
+    if world > 1:
+        dist.init_process_group("nccl", device_id=dev)
+
+    cfg = synth.CONFIGS[WORKLOAD]
+    L, H, G, s, D, c = cfg["L"], cfg["H"], cfg["G"], cfg["s"], cfg["d"], cfg["chunk"]
+    es = 2
+    seed = cfg["seed"] + 7919 * rank
+    K = synth.ar1_keys(L, H, s, D, cfg["rho"], cfg["mean_std"], seed=seed, dtype="bf16", device=dev)
+    V = synth.normal_values(L, H, s, D, seed=seed, dtype="bf16", device=dev)
+    kn = synth.ar1_keys(L, H, c, D, cfg["rho"], cfg["mean_std"], seed=seed + 1, dtype="bf16", device=dev)
+    vn = synth.normal_values(L, H, c, D, seed=seed + 1, dtype="bf16", device=dev)
+    q = synth.queries(L, H * G, D, seed=seed + 2, dtype="bf16", device=dev)  # one [1, H*G, D] query per layer
+    out = torch.empty_like(q)
+
+    p = b.Params(chunk=c, n_sink=0, n_recent=0, n_rounds_max=1, r_init=1.0, r_decay=0.0, r_min=1.0, select=b.SELECT_GLOBAL)
+    src = b.Cache(K, V, None, None, s)
+    out_len, rounds, cap = b.compress_plan(s, p)
+    dst = b.Cache.empty(L, H, cap + c, D, K.dtype, dev)
+    ws = torch.empty(max(b.workspace_bytes(src, p), b.workspace_bytes(dst, p)), dtype=torch.uint8, device=dev)
+    wsd = torch.empty(b.decode_workspace_bytes(1, H, G, D, cap + c), dtype=torch.uint8, device=dev)
+    scale = 1.0 / math.sqrt(D)
+    final_len = out_len + c // 2
+    # the lengths a step produces are a function of shapes only, so the decode views can be built once
+    dst.len = final_len
+    views = [b.layer_views([dst], l, dev) for l in range(L)]
+    launches_per_step = 1 + 3 + 2 * L
+
+    ev = lambda: torch.cuda.Event(enable_timing=True)
+    comp_ev, dec_ev = [], []
+
+    def step(record: bool):
+        e0, e1, e2, e3 = (ev(), ev(), ev(), ev()) if record else (None,) * 4
+        if record:
+            e0.record()
+        b.compress_prefill(src, dst, p, ws)
+        if record:
+            e1.record()
+        b.compress_append(dst, kn, vn, p, ws)
+        if record:
+            e2.record()
+        for l in range(L):
+            b.decode_attn(views[l], H, G, q[l:l + 1], out[l:l + 1], scale, final_len, wsd)
+        if record:
+            e3.record()
+            comp_ev.append((e0, e1))
+            dec_ev.append((e2, e3))
+        assert dst.len == final_len
+
+    def barrier():
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    for _ in range(max(args.warmup, 3)):
+        step(False)
+    barrier()
+    sampler = ClockSampler(local) if rank == 0 else None
+    t_start, t_end = ev(), ev()
+    t_start.record()
+    for _ in range(args.steps):
+        step(True)
+    t_end.record()
+    barrier()
+    clocks = sampler.stop() if sampler else None
+    elapsed_ms = t_start.elapsed_time(t_end)
+    if world > 1:
+        t = torch.tensor([elapsed_ms], device=dev)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        elapsed_ms = float(t.item())
+    ms_per_step = elapsed_ms / args.steps
+    value = world * s * args.steps / (elapsed_ms * 1e-3)
+
+    comp_ms = statistics.mean(a.elapsed_time(z) for a, z in comp_ev)
+    dec_ms = statistics.mean(a.elapsed_time(z) for a, z in dec_ev)
+    peaks, peak_kind = measured_peaks()
+    cbytes = compress_bytes(L, H, s, D, es, out_len / s)
+    achieved = cbytes / (comp_ms * 1e-3) / 1e9
+    roofline = {"bound": "hbm", "kernel": "compress round kernel (one launch per ckv_compress_prefill)", "achieved": achieved,
+                "peak": peaks["hbm_gbs"], "peak_kind": peak_kind, "unit": "GB/s", "frac": achieved / peaks["hbm_gbs"],
+                "traffic": None, "bytes_per_launch": cbytes, "ms_per_launch": comp_ms}
+    dbytes = decode_bytes(H * final_len, D, es)
+    dec_achieved = dbytes * L / (dec_ms * 1e-3) / 1e9
+    extra = {"compress_ms": comp_ms, "compress_tokens_per_s": s / (comp_ms * 1e-3), "decode_ms_all_layers": dec_ms,
+             "decode_gbs_batch1": dec_achieved}
+
+    if rank == 0 and not args.skip_decode_cfg4:
+        extra["decode_cfg4"] = bench_decode_cfg4(b, synth, dev, peaks["hbm_gbs"])
+
+    # end to end: inputs start in pinned host memory, the compressed cache and the decode output end there
+    e2e = None
+    if not args.skip_e2e:
+        e2e = bench_e2e(b, torch, dev, K, V, kn, vn, q, step, dst, final_len, out, s, world, max(2, min(args.steps, 5)))
+        if world > 1:
+            t = torch.tensor([e2e["ms_per_step"]], device=dev)
+            dist.all_reduce(t, op=dist.ReduceOp.MAX)
+            e2e["ms_per_step"] = float(t.item())
+            e2e["value"] = world * s / (e2e["ms_per_step"] * 1e-3)
+
+    cpu = None
+    if rank == 0 and world == 1 and not args.skip_cpu:
+        x = oracle_inputs(16)
+        dt = oracle_pass(x)
+        cpu = {"value": x["tokens"] / dt, "unit": UNIT, "cores": 1, "kind": "oracle", "sample": x["desc"], "seconds": dt}
+
+    if rank == 0:
+        line = {"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": max(args.warmup, 3),
+                "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "bf16",
+                "data": "synthetic",
+                "config": {"workload": WORKLOAD, "layers": L, "kv_heads": H, "q_heads": H * G, "head_dim": D, "seq": s,
+                           "chunk": c, "retain": out_len / s, "step": "compress_prefill + append 64 + decode all layers",
+                           "l2": "inputs (4 GiB) exceed L2"},
+                "clocks": clocks, "e2e": e2e, "gpu_launches": launches_per_step * args.steps, "roofline": roofline,
+                "cpu_baseline": cpu, "detail": extra}
+        print(json.dumps(line))
+    if world > 1:
+        dist.destroy_process_group()
+
+
+def bench_e2e(b, torch, dev, K, V, kn, vn, q, step, dst, final_len, out, s, world, iters):
+    hK = torch.empty(K.shape, dtype=K.dtype, pin_memory=True)
+    hV = torch.empty(V.shape, dtype=V.dtype, pin_memory=True)
+    hK.copy_(K)
+    hV.copy_(V)
+    hkn, hvn, hq = kn.cpu().pin_memory(), vn.cpu().pin_memory(), q.cpu().pin_memory()
+    L, H, _, D = K.shape
+    hKo = torch.empty((L, H, final_len, D), dtype=K.dtype, pin_memory=True)
+    hVo = torch.empty_like(hKo).pin_memory()
+    hdeg = torch.empty((L, H, final_len), dtype=torch.int32, pin_memory=True)
+    hout = torch.empty(out.shape, dtype=out.dtype, pin_memory=True)
+    h2d = sum(t.numel() * t.element_size() for t in (hK, hV, hkn, hvn, hq))
+    d2h = sum(t.numel() * t.element_size() for t in (hKo, hVo, hdeg, hout))
+
+    def e2e_step():
+        K.copy_(hK, non_blocking=True)
+        V.copy_(hV, non_blocking=True)
+        kn.copy_(hkn, non_blocking=True)
+        vn.copy_(hvn, non_blocking=True)
+        q.copy_(hq, non_blocking=True)
+        step(False)
+        hKo.copy_(dst.k[:, :, :final_len], non_blocking=True)
+        hVo.copy_(dst.v[:, :, :final_len], non_blocking=True)
+        hdeg.copy_(dst.deg[:, :, :final_len], non_blocking=True)
+        hout.copy_(out, non_blocking=True)
+
+    e2e_step()
+    torch.cuda.synchronize()
+    t0, t1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    t0.record()
+    for _ in range(iters):
+        e2e_step()
+    t1.record()
+    torch.cuda.synchronize()
+    ms = t0.elapsed_time(t1) / iters
+    return {"value": world * s / (ms * 1e-3), "unit": UNIT, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
+            "ms_per_step": ms, "steps": iters}
+
+
+def bench_decode_cfg4(b, synth, dev, peak_gbs):
+    """Decode attention on the batch-32 shape: 8192 centroids (+256 appended) vs the uncompressed 32768-token cache."""
+    import torch
+    cfg = synth.CONFIGS["decode_b32"]
+    Bz, H, G, D = cfg["batch"], cfg["H"], cfg["G"], cfg["d"]
+    res = {}
+    for name, slots, with_deg in (("compressed", cfg["slots"], True), ("uncompressed", cfg["s"], False)):
+        cap = slots + 256
+        caches = []
+        for i in range(Bz):
+            k = torch.randn((1, H, cap, D), device=dev, dtype=torch.float32).to(torch.bfloat16)
+            v = torch.randn((1, H, cap, D), device=dev, dtype=torch.float32).to(torch.bfloat16)
+            deg = logdeg = None
+            if with_deg:
+                deg = torch.ones((1, H, cap), dtype=torch.int32)
+                deg[:, :, :slots] = synth.random_degrees((1, H), slots, cfg["s"], seed=i)
+                deg = deg.to(dev)
+                logdeg = torch.log(deg.float())
+            caches.append(b.Cache(k, v, deg, logdeg, slots))
+        q = synth.queries(Bz, H * G, D, seed=3, dtype="bf16", device=dev)
+        out = torch.empty_like(q)
+        ws = torch.empty(b.decode_workspace_bytes(Bz, H, G, D, cap), dtype=torch.uint8, device=dev)
+        views = b.layer_views(caches, 0, dev)
+        scale = 1.0 / math.sqrt(D)
+        for _ in range(5):
+            b.decode_attn(views, H, G, q, out, scale, slots, ws)
+        torch.cuda.synchronize()
+        iters = 50
+        t0, t1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        t0.record()
+        for _ in range(iters):
+            b.decode_attn(views, H, G, q, out, scale, slots, ws)
+        t1.record()
+        torch.cuda.synchronize()
+        us = 1e3 * t0.elapsed_time(t1) / iters
+        nbytes = decode_bytes(Bz * H * slots, D, 2) if with_deg else Bz * H * slots * 2 * D * 2
+        res[name] = {"slots": slots, "us_per_layer_step": us, "gbs": nbytes / (us * 1e-6) / 1e9,
+                     "frac_of_peak": nbytes / (us * 1e-6) / 1e9 / peak_gbs, "decode_tok_s_per_layer": Bz / (us * 1e-6)}
+        del caches
+    res["speedup"] = res["uncompressed"]["us_per_layer_step"] / res["compressed"]["us_per_layer_step"]
+    return res
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=20)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--impl", default="ckv", choices=["ckv", "reference"])
+    ap.add_argument("--skip-e2e", action="store_true")
+    ap.add_argument("--skip-cpu", action="store_true")
+    ap.add_argument("--skip-decode-cfg4", action="store_true")
+    args = ap.parse_args()
+    if args.impl == "reference":
+        run_reference(args)
+    else:
+        run_gpu(args)
+
+
+if __name__ == "__main__":
+    main()
