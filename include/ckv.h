@@ -106,6 +106,12 @@ int ckv_compress_prefill(const ckv_cache* src, ckv_cache* dst, const ckv_params*
 int ckv_compress_append(ckv_cache* cache, const void* k_new, const void* v_new, int32_t t_new,
                         const ckv_params* params, void* workspace, size_t workspace_bytes, void* cuda_stream);
 
+/* The kernels wait on asynchronous copies with a bounded number of polls; a wait that gives up sets a
+ * status word at the start of the workspace instead of hanging.  This call copies that word to
+ * *status_host (host pointer) and synchronises the stream: 0 = every wait completed, nonzero = some
+ * output of the last ckv_compress_* call on this workspace is incomplete.  The paper has no counterpart. */
+int ckv_workspace_status(const void* workspace, void* cuda_stream, int32_t* status_host);
+
 /* One layer of one sequence for decode attention: k, v: [H, cap, D]; logdeg: [H, cap] or NULL
  * (all degrees one: Eq. 1). */
 typedef struct ckv_layer_view {

@@ -19,7 +19,7 @@ SELECT_GLOBAL, SELECT_CHUNK = 0, 1
 OK = 0
 
 EXPORTS = ["ckv_compress_plan", "ckv_workspace_bytes", "ckv_compress_prefill", "ckv_compress_append",
-           "ckv_decode_workspace_bytes", "ckv_decode_attn", "ckv_status_string"]
+           "ckv_decode_workspace_bytes", "ckv_decode_attn", "ckv_status_string", "ckv_workspace_status"]
 
 
 class CkvCache(C.Structure):
@@ -56,6 +56,8 @@ def _load():
     lib.ckv_compress_append.restype = C.c_int
     lib.ckv_compress_append.argtypes = [C.POINTER(CkvCache), C.c_void_p, C.c_void_p, C.c_int32, C.POINTER(CkvParams),
                                         C.c_void_p, C.c_size_t, C.c_void_p]
+    lib.ckv_workspace_status.restype = C.c_int
+    lib.ckv_workspace_status.argtypes = [C.c_void_p, C.c_void_p, C.POINTER(C.c_int32)]
     lib.ckv_decode_workspace_bytes.restype = C.c_size_t
     lib.ckv_decode_workspace_bytes.argtypes = [C.c_int32, C.c_int32, C.c_int32, C.c_int32, C.c_int64]
     lib.ckv_decode_attn.restype = C.c_int
@@ -167,6 +169,13 @@ def compress_append(cache: Cache, k_new: torch.Tensor, v_new: torch.Tensor, para
     _check(lib.ckv_compress_append(C.byref(cc), k_new.data_ptr(), v_new.data_ptr(), k_new.shape[2], C.byref(params.c()),
                                    workspace.data_ptr(), workspace.numel() * workspace.element_size(), _stream_ptr()))
     cache.len, cache.pending = cc.len, cc.pending
+
+
+def workspace_status(workspace: torch.Tensor) -> int:
+    """ckv_workspace_status: synchronises the current stream and returns the device status word (0 = fine)."""
+    st = C.c_int32(-1)
+    _check(lib.ckv_workspace_status(workspace.data_ptr(), _stream_ptr(), C.byref(st)))
+    return st.value
 
 
 def layer_views(caches, layer: int, device="cuda") -> torch.Tensor:

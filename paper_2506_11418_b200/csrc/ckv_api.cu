@@ -94,7 +94,7 @@ Workspace layout_workspace(int64_t LH, int D, int esize, int chunk, const std::v
     if (plan[j].mode == kModeExternal) max_chunks = std::max<int64_t>(max_chunks, plan[j].n_chunks);
     max_sin = std::max(max_sin, plan[j].s_in);
   }
-  size_t off = 0;
+  size_t off = 256;  // the first 256 bytes hold the device status word
   auto take = [&off](size_t bytes) {
     const size_t at = off;
     off += align_up(bytes);
@@ -111,7 +111,7 @@ Workspace layout_workspace(int64_t LH, int D, int esize, int chunk, const std::v
   w.chunk_off = take((size_t)LH * max_chunks * 4);
   w.assign_stride = (want_assign && R >= 2) ? max_sin : 0;
   w.assign_step = take((size_t)LH * w.assign_stride * 4);
-  w.total = off + 256;
+  w.total = off;
   return w;
 }
 
@@ -169,7 +169,9 @@ cudaError_t run_round(const RoundPlan& rp, const Buf& src, const Buf& dst, int L
   a.chunk = chunk; a.n_chunks = rp.n_chunks;
   a.m_full = rp.m_full; a.m_tail = rp.m_tail;
   a.out_stride = chunk - rp.m_full;
+  a.out_lo = rp.lo;
   a.LH = LH;
+  a.status = reinterpret_cast<int32_t*>(ws);
   a.edge_stride = (int64_t)rp.n_chunks * (chunk / 2);
   if (rp.mode == kModeExternal) {
     a.edge_sim = reinterpret_cast<float*>(ws + w.edge_sim);
@@ -184,6 +186,16 @@ cudaError_t run_round(const RoundPlan& rp, const Buf& src, const Buf& dst, int L
     if ((e = launch_select(s, st)) != cudaSuccess) return e;
   }
   a.mode = rp.mode;
+  if (round_fast_supported(a, dtype, D)) {
+    // full chunks on the fast kernel, the shorter last chunk (if any) on the general one
+    const int64_t mid = rp.hi - rp.lo;
+    const int64_t n_full = mid / chunk;
+    if ((e = launch_round_fast(a, n_full, st)) != cudaSuccess) return e;
+    if (rp.n_chunks == n_full) return cudaSuccess;
+    a.lo = rp.lo + n_full * chunk;
+    a.out_lo = rp.lo + n_full * a.out_stride;
+    a.n_chunks = 1;
+  }
   return launch_round(a, dtype, D, st);
 }
 
@@ -321,6 +333,7 @@ int ckv_compress_prefill(const ckv_cache* src, ckv_cache* dst, const ckv_params*
       overlaps(workspace, need, src->k, src_bytes) || overlaps(workspace, need, src->v, src_bytes))
     return CKV_ERR_INVALID_ARG;
 
+  if (cudaMemsetAsync(workspace, 0, 256, static_cast<cudaStream_t>(cuda_stream)) != cudaSuccess) return CKV_ERR_CUDA;
   const Buf s{src->k, src->v, src->deg, src->logdeg, src->cap};
   const Buf d{dst->k, dst->v, dst->deg, dst->logdeg, dst->cap};
   st = run_plan(plan, s, d, src->len, (int)LH, src->D, src->dtype, params->chunk, assign, w,
@@ -367,6 +380,7 @@ int ckv_compress_append(ckv_cache* cache, const void* k_new, const void* v_new, 
   const Buf stage{ws + base, ws + base + win_kv, reinterpret_cast<int32_t*>(ws + base + 2 * win_kv),
                   reinterpret_cast<float*>(ws + base + 2 * win_kv + win_dg), c};
   cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
+  if (cudaMemsetAsync(workspace, 0, 256, stream) != cudaSuccess) return CKV_ERR_CUDA;
 
   for (int32_t done = 0; done < t_new;) {
     const int32_t take = (int32_t)std::min<int64_t>(t_new - done, c - cache->pending);
@@ -398,6 +412,13 @@ int ckv_compress_append(ckv_cache* cache, const void* k_new, const void* v_new, 
     if (cache->pending == c) cache->pending = 0;
   }
   return CKV_OK;
+}
+
+int ckv_workspace_status(const void* workspace, void* cuda_stream, int32_t* status_host) {
+  if (!workspace || !status_host) return CKV_ERR_INVALID_ARG;
+  cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+  if (cudaMemcpyAsync(status_host, workspace, sizeof(int32_t), cudaMemcpyDeviceToHost, st) != cudaSuccess) return CKV_ERR_CUDA;
+  return cudaStreamSynchronize(st) == cudaSuccess ? CKV_OK : CKV_ERR_CUDA;
 }
 
 size_t ckv_decode_workspace_bytes(int32_t Bz, int32_t H, int32_t G, int32_t D, int64_t max_len) {

@@ -184,7 +184,7 @@ __global__ void __launch_bounds__(kRoundThreads) round_kernel(const RoundArgs a)
   __syncthreads();
 
   const int64_t out_base = (a.mode == kModeExternal) ? (int64_t)a.chunk_out_off[(int64_t)lh * a.n_chunks + chunk_id]
-                                                     : a.lo + (int64_t)chunk_id * a.out_stride;
+                                                     : a.out_lo + (int64_t)chunk_id * a.out_stride;
   T* kdst = reinterpret_cast<T*>(a.k_dst) + ((int64_t)lh * a.dst_cap + out_base) * D;
   T* vdst = reinterpret_cast<T*>(a.v_dst) + ((int64_t)lh * a.dst_cap + out_base) * D;
 

@@ -1,0 +1,371 @@
+// Chunked Soft Matching round, fast path: bf16, chunk 64, head_dim 128, every edge merged (ratio 1).
+//
+// Persistent kernel, one CTA per SM.  Every warp is an independent worker that owns one shared-memory
+// stage (a chunk's K tile and V tile, 2 x 16 KiB): it fetches the two tiles with bulk async copies that
+// signal the warp's own mbarrier, and while one warp computes, the copies of the others are in flight.
+//   Sec. 5.2  the 32 x 32 A x B dot products on tensor cores (mma.sync m16n8k16, bf16 in, fp32
+//             accumulate); the squared norms of the B keys come from the same fragments (diagonal of
+//             B B^T); row argmax of dot / |b| (dividing a row by |a| > 0 does not change its argmax)
+//   Sec. 5.3  ratio 1: every A token merges into its best B token
+//   Eq. 5     degree-weighted sums of K and V rows in fp32 from the staged tiles, divided by the
+//             summed degree, rounded to bf16, written with coalesced 8-byte stores
+// Waits on the mbarrier are bounded: a warp that gives up records it in the status word and leaves.
+#include <algorithm>
+#include <cstdint>
+
+#include "ckv_common.cuh"
+#include "ckv_internal.h"
+
+namespace ckv {
+
+namespace {
+
+constexpr int kC = 64;            // chunk size
+constexpr int kD = 128;           // head_dim
+constexpr int kRowBytes = kD * 2; // one bf16 row
+constexpr int kTileBytes = kC * kRowBytes;
+constexpr int kStageBytes = 2 * kTileBytes;  // K tile then V tile
+constexpr int kExtraBytes = 400;             // per warp: degrees [64] int, best [32] int, mbarrier (8 B), pad
+constexpr uint32_t kSpinLimit = 1u << 22;
+
+__device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
+
+__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
+  asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count));
+}
+
+__device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes) {
+  asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
+}
+
+__device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
+  uint32_t ok;
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+      "selp.u32 %0, 1, 0, p;\n\t}"
+      : "=r"(ok)
+      : "r"(bar), "r"(parity)
+      : "memory");
+  return ok != 0;
+}
+
+// Bounded wait: false if the phase did not complete within the spin limit.
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity) {
+  for (uint32_t i = 0; i < kSpinLimit; ++i) {
+    if (mbar_try_wait(bar, parity)) return true;
+    if (i > 64) __nanosleep(64);
+  }
+  return false;
+}
+
+__device__ __forceinline__ void bulk_load(uint32_t dst, const void* src, uint32_t bytes, uint32_t bar) {
+  asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];" ::"r"(dst),
+               "l"(src), "r"(bytes), "r"(bar)
+               : "memory");
+}
+
+__device__ __forceinline__ void mma_bf16(float (&d)[4], uint32_t a0, uint32_t a1, uint32_t a2, uint32_t a3, uint32_t b0,
+                                         uint32_t b1) {
+  asm volatile(
+      "mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
+      : "+f"(d[0]), "+f"(d[1]), "+f"(d[2]), "+f"(d[3])
+      : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1));
+}
+
+__device__ __forceinline__ void unpack4(uint2 u, float (&f)[4]) {
+  f[0] = __uint_as_float(u.x << 16);
+  f[1] = __uint_as_float(u.x & 0xffff0000u);
+  f[2] = __uint_as_float(u.y << 16);
+  f[3] = __uint_as_float(u.y & 0xffff0000u);
+}
+
+struct FastArgs {
+  const __nv_bfloat16* k_src;
+  const __nv_bfloat16* v_src;
+  const int32_t* deg_src;  // may be null: all ones
+  __nv_bfloat16* k_dst;
+  __nv_bfloat16* v_dst;
+  int32_t* deg_dst;
+  float* logdeg_dst;  // may be null
+  int32_t* assign;    // may be null
+  int64_t assign_stride;
+  int64_t src_cap, dst_cap;
+  int64_t lo;       // first token of the middle region in src
+  int64_t out_lo;   // where the first chunk's survivors go in dst
+  int64_t n_full;   // full chunks per (layer, head)
+  int64_t n_items;  // n_full * LH
+  int32_t* status;  // device word: set to 1 if a wait gave up
+};
+
+template <int NW, bool HAS_DEG>
+__global__ void __launch_bounds__(NW * 32, 1) round_fast_kernel(const FastArgs a) {
+  extern __shared__ __align__(128) unsigned char smem[];
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+  const int g = lane >> 2, t = lane & 3;
+  unsigned char* stage = smem + (size_t)warp * kStageBytes;
+  unsigned char* extra = smem + (size_t)NW * kStageBytes + (size_t)warp * kExtraBytes;
+  int* degs = reinterpret_cast<int*>(extra);             // [64]
+  int* best = reinterpret_cast<int*>(extra + 256);       // [32] B index (0..31) chosen by A token i
+  const uint32_t bar = smem_u32(extra + 384);
+  const uint32_t k_s = smem_u32(stage), v_s = k_s + kTileBytes;
+
+  if (lane == 0) {
+    mbar_init(bar, 1);
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+  }
+  __syncwarp();
+
+  const int64_t stride = (int64_t)gridDim.x * NW;
+  int64_t item = (int64_t)blockIdx.x * NW + warp;
+  auto issue = [&](int64_t it) {
+    const int64_t lh = it / a.n_full, ch = it - lh * a.n_full;
+    const int64_t row0 = lh * a.src_cap + a.lo + ch * kC;
+    mbar_expect_tx(bar, kStageBytes);
+    bulk_load(k_s, a.k_src + row0 * kD, kTileBytes, bar);
+    bulk_load(v_s, a.v_src + row0 * kD, kTileBytes, bar);
+  };
+  if (item < a.n_items && lane == 0) issue(item);
+
+  uint32_t parity = 0;
+  for (; item < a.n_items; item += stride, parity ^= 1) {
+    const int64_t lh = item / a.n_full, ch = item - lh * a.n_full;
+    const int64_t src_row0 = lh * a.src_cap + a.lo + ch * kC;
+    const int64_t out_row0 = lh * a.dst_cap + a.out_lo + ch * (kC / 2);
+    if (HAS_DEG) {
+      degs[lane] = a.deg_src[src_row0 + lane];
+      degs[lane + 32] = a.deg_src[src_row0 + lane + 32];
+    }
+    if (!mbar_wait(bar, parity)) {
+      if (lane == 0) atomicExch(a.status, 1);
+      mbar_wait(bar, parity);  // the copies may still land: give them one more bounded wait before leaving
+      return;
+    }
+    __syncwarp();
+
+    // ---- A x B dot products and the B keys' squared norms on tensor cores
+    float acc[2][4][4];   // [m tile][n tile][c]: A token 16*mt + g (+8), B index 8*nt + 2t (+1)
+    float nacc[2][2][4];  // [pair of n tiles][which of the pair as column operand][c]
+#pragma unroll
+    for (int i = 0; i < 2; ++i)
+#pragma unroll
+      for (int j = 0; j < 4; ++j)
+#pragma unroll
+        for (int c = 0; c < 4; ++c) acc[i][j][c] = 0.f;
+#pragma unroll
+    for (int i = 0; i < 2; ++i)
+#pragma unroll
+      for (int j = 0; j < 2; ++j)
+#pragma unroll
+        for (int c = 0; c < 4; ++c) nacc[i][j][c] = 0.f;
+
+#pragma unroll
+    for (int kp = 0; kp < 4; ++kp) {
+      // each lane reads 16 contiguous bytes of a row: elements 32*kp + 8*t .. +7.  The same permutation of the
+      // contraction index is applied to both operands, so the dot products are unchanged.
+      uint4 ra[2][2], rb[4];
+      const uint32_t col = 64u * kp + 16u * t;
+#pragma unroll
+      for (int mt = 0; mt < 2; ++mt)
+#pragma unroll
+        for (int hi = 0; hi < 2; ++hi) {
+          const uint32_t tok = 2u * (16u * mt + 8u * hi + g);
+          asm volatile("ld.shared.v4.u32 {%0,%1,%2,%3}, [%4];"
+                       : "=r"(ra[mt][hi].x), "=r"(ra[mt][hi].y), "=r"(ra[mt][hi].z), "=r"(ra[mt][hi].w)
+                       : "r"(k_s + tok * kRowBytes + col));
+        }
+#pragma unroll
+      for (int nt = 0; nt < 4; ++nt) {
+        const uint32_t tok = 2u * (8u * nt + g) + 1u;
+        asm volatile("ld.shared.v4.u32 {%0,%1,%2,%3}, [%4];"
+                     : "=r"(rb[nt].x), "=r"(rb[nt].y), "=r"(rb[nt].z), "=r"(rb[nt].w)
+                     : "r"(k_s + tok * kRowBytes + col));
+      }
+#pragma unroll
+      for (int ks = 0; ks < 2; ++ks) {
+        uint32_t b0[4], b1[4];
+#pragma unroll
+        for (int nt = 0; nt < 4; ++nt) {
+          b0[nt] = ks ? rb[nt].z : rb[nt].x;
+          b1[nt] = ks ? rb[nt].w : rb[nt].y;
+        }
+#pragma unroll
+        for (int mt = 0; mt < 2; ++mt) {
+          const uint32_t a0 = ks ? ra[mt][0].z : ra[mt][0].x, a1 = ks ? ra[mt][1].z : ra[mt][1].x;
+          const uint32_t a2 = ks ? ra[mt][0].w : ra[mt][0].y, a3 = ks ? ra[mt][1].w : ra[mt][1].y;
+#pragma unroll
+          for (int nt = 0; nt < 4; ++nt) mma_bf16(acc[mt][nt], a0, a1, a2, a3, b0[nt], b1[nt]);
+        }
+        // B B^T on pairs of n tiles: rows = B indices 16p + g (+8), the diagonal holds the squared norms
+#pragma unroll
+        for (int p = 0; p < 2; ++p) {
+          mma_bf16(nacc[p][0], b0[2 * p], b0[2 * p + 1], b1[2 * p], b1[2 * p + 1], b0[2 * p], b1[2 * p]);
+          mma_bf16(nacc[p][1], b0[2 * p], b0[2 * p + 1], b1[2 * p], b1[2 * p + 1], b0[2 * p + 1], b1[2 * p + 1]);
+        }
+      }
+    }
+
+    // squared norm of B index 8*nt + g sits on the diagonal: lane (g, t = g / 2), register g & 1 (+2 for odd nt)
+    float inv0[4], inv1[4];
+#pragma unroll
+    for (int nt = 0; nt < 4; ++nt) {
+      const int p = nt >> 1, h = nt & 1;
+      const float ss = (g & 1) ? nacc[p][h][2 * h + 1] : nacc[p][h][2 * h];
+      const float inv = ss > 0.f ? rsqrtf(ss) : 0.f;
+      inv0[nt] = __shfl_sync(0xffffffffu, inv, 9 * t);      // B index 8*nt + 2t     lives in lane 4*(2t) + t
+      inv1[nt] = __shfl_sync(0xffffffffu, inv, 9 * t + 4);  // B index 8*nt + 2t + 1 lives in lane 4*(2t+1) + t
+    }
+
+    // ---- row argmax (lowest B index on ties)
+#pragma unroll
+    for (int mt = 0; mt < 2; ++mt)
+#pragma unroll
+      for (int hi = 0; hi < 2; ++hi) {
+        float bv = -INFINITY;
+        int bi = 0x7fffffff;
+#pragma unroll
+        for (int nt = 0; nt < 4; ++nt) {
+          float s0 = acc[mt][nt][2 * hi] * inv0[nt] + 0.f, s1 = acc[mt][nt][2 * hi + 1] * inv1[nt] + 0.f;
+          if (s0 > bv) { bv = s0; bi = 8 * nt + 2 * t; }
+          if (s1 > bv) { bv = s1; bi = 8 * nt + 2 * t + 1; }
+        }
+#pragma unroll
+        for (int o = 1; o <= 2; o <<= 1) {
+          const float ov = __shfl_xor_sync(0xffffffffu, bv, o);
+          const int oi = __shfl_xor_sync(0xffffffffu, bi, o);
+          if (ov > bv || (ov == bv && oi < bi)) { bv = ov; bi = oi; }
+        }
+        if (t == 0) best[16 * mt + 8 * hi + g] = bi;
+      }
+    __syncwarp();
+    const int my_best = best[lane];  // lane = A index
+
+    // ---- Eq. 5: one output row per B token, members gathered from the staged tiles
+    int my_deg = 0;
+    __nv_bfloat16* kdst = a.k_dst + out_row0 * kD + lane * 4;
+    __nv_bfloat16* vdst = a.v_dst + out_row0 * kD + lane * 4;
+#pragma unroll 2
+    for (int j = 0; j < 32; ++j) {
+      unsigned members = __ballot_sync(0xffffffffu, my_best == j);
+      const uint32_t brow = (2u * j + 1u) * kRowBytes + lane * 8u;
+      uint2 uk, uv;
+      asm volatile("ld.shared.v2.u32 {%0,%1}, [%2];" : "=r"(uk.x), "=r"(uk.y) : "r"(k_s + brow));
+      asm volatile("ld.shared.v2.u32 {%0,%1}, [%2];" : "=r"(uv.x), "=r"(uv.y) : "r"(v_s + brow));
+      int n_new = HAS_DEG ? degs[2 * j + 1] : 1;
+      if (members) {
+        float fk[4], fv[4];
+        unpack4(uk, fk);
+        unpack4(uv, fv);
+        if (HAS_DEG) {
+          const float wb = (float)n_new;
+#pragma unroll
+          for (int e = 0; e < 4; ++e) { fk[e] *= wb; fv[e] *= wb; }
+        }
+        while (members) {
+          const int ai = __ffs(members) - 1;
+          members &= members - 1;
+          const uint32_t arow = (2u * ai) * kRowBytes + lane * 8u;
+          uint2 mk, mv;
+          asm volatile("ld.shared.v2.u32 {%0,%1}, [%2];" : "=r"(mk.x), "=r"(mk.y) : "r"(k_s + arow));
+          asm volatile("ld.shared.v2.u32 {%0,%1}, [%2];" : "=r"(mv.x), "=r"(mv.y) : "r"(v_s + arow));
+          float gk[4], gv[4];
+          unpack4(mk, gk);
+          unpack4(mv, gv);
+          if (HAS_DEG) {
+            const int wa = degs[2 * ai];
+            const float w = (float)wa;
+            n_new += wa;
+#pragma unroll
+            for (int e = 0; e < 4; ++e) { fk[e] = fmaf(w, gk[e], fk[e]); fv[e] = fmaf(w, gv[e], fv[e]); }
+          } else {
+            n_new += 1;
+#pragma unroll
+            for (int e = 0; e < 4; ++e) { fk[e] += gk[e]; fv[e] += gv[e]; }
+          }
+        }
+        const float inv = 1.0f / (float)n_new;
+        uk.x = pack_bf16x2(fk[0] * inv, fk[1] * inv);
+        uk.y = pack_bf16x2(fk[2] * inv, fk[3] * inv);
+        uv.x = pack_bf16x2(fv[0] * inv, fv[1] * inv);
+        uv.y = pack_bf16x2(fv[2] * inv, fv[3] * inv);
+      }
+      *reinterpret_cast<uint2*>(kdst + (int64_t)j * kD) = uk;  // a B token nobody chose is copied bit for bit
+      *reinterpret_cast<uint2*>(vdst + (int64_t)j * kD) = uv;
+      if (lane == j) my_deg = n_new;
+    }
+    a.deg_dst[out_row0 + lane] = my_deg;
+    if (a.logdeg_dst) a.logdeg_dst[out_row0 + lane] = logf((float)my_deg);
+    if (a.assign) {
+      int32_t* as = a.assign + lh * a.assign_stride + a.lo + ch * kC;
+      const int32_t slot0 = (int32_t)(a.out_lo + ch * (kC / 2));
+      as[2 * lane] = slot0 + my_best;   // A token 2*lane joins its B token's slot
+      as[2 * lane + 1] = slot0 + lane;  // B token 2*lane+1 keeps slot `lane` of the chunk
+    }
+
+    // ---- this stage is free again: fetch the warp's next chunk
+    __syncwarp();
+    if (item + stride < a.n_items && lane == 0) {
+      asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+      issue(item + stride);
+    }
+  }
+}
+
+int sm_count() {
+  static int cached = 0;
+  if (cached == 0) {
+    int dev = 0, n = 0;
+    if (cudaGetDevice(&dev) == cudaSuccess && cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev) == cudaSuccess && n > 0)
+      cached = n;
+    else
+      return 148;
+  }
+  return cached;
+}
+
+template <int NW>
+cudaError_t launch_fast_nw(const FastArgs& a, cudaStream_t st) {
+  const size_t smem = (size_t)NW * (kStageBytes + kExtraBytes);
+  const int64_t ctas = std::min<int64_t>(sm_count(), (a.n_items + NW - 1) / NW);
+  cudaError_t e;
+  if (a.deg_src) {
+    if ((e = cudaFuncSetAttribute(round_fast_kernel<NW, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem)) != cudaSuccess) return e;
+    round_fast_kernel<NW, true><<<(unsigned)ctas, NW * 32, smem, st>>>(a);
+  } else {
+    if ((e = cudaFuncSetAttribute(round_fast_kernel<NW, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem)) != cudaSuccess) return e;
+    round_fast_kernel<NW, false><<<(unsigned)ctas, NW * 32, smem, st>>>(a);
+  }
+  return cudaGetLastError();
+}
+
+}  // namespace
+
+bool round_fast_supported(const RoundArgs& a, int dtype, int D) {
+  return dtype == 1 && D == 128 && a.chunk == kC && a.mode == kModeAll && a.status != nullptr;
+}
+
+// Full chunks of a ratio-1 round.  The shorter last chunk, if any, is left to the general kernel.
+cudaError_t launch_round_fast(const RoundArgs& r, int64_t n_full, cudaStream_t st) {
+  if (n_full <= 0) return cudaSuccess;
+  FastArgs a{};
+  a.k_src = static_cast<const __nv_bfloat16*>(r.k_src);
+  a.v_src = static_cast<const __nv_bfloat16*>(r.v_src);
+  a.deg_src = r.deg_src;
+  a.k_dst = static_cast<__nv_bfloat16*>(r.k_dst);
+  a.v_dst = static_cast<__nv_bfloat16*>(r.v_dst);
+  a.deg_dst = r.deg_dst;
+  a.logdeg_dst = r.logdeg_dst;
+  a.assign = r.assign;
+  a.assign_stride = r.assign_stride;
+  a.src_cap = r.src_cap;
+  a.dst_cap = r.dst_cap;
+  a.lo = r.lo;
+  a.out_lo = r.out_lo;
+  a.n_full = n_full;
+  a.n_items = n_full * r.LH;
+  a.status = r.status;
+  return launch_fast_nw<7>(a, st);
+}
+
+}  // namespace ckv

@@ -27,6 +27,7 @@ struct RoundArgs {
   int64_t assign_stride;
   int64_t src_cap, dst_cap;
   int64_t lo, hi;
+  int64_t out_lo;          // dst position of the first chunk's first survivor (kModeAll, kModeChunkTopM)
   int32_t chunk, n_chunks;
   int32_t mode;
   int32_t m_full, m_tail;  // kModeChunkTopM: merges in a full chunk / in the shorter last chunk
@@ -37,6 +38,7 @@ struct RoundArgs {
   int32_t* chunk_out_off;  // [LH, n_chunks]      kModeExternal: dst position of the chunk's first survivor
   int64_t edge_stride;     // n_chunks * chunk / 2
   int32_t LH;
+  int32_t* status;         // device word in the workspace: nonzero after a bounded wait gave up
 };
 
 // Copy `count` token rows (K, V, degree) of every slab from src_off to dst_off.
@@ -83,5 +85,7 @@ cudaError_t launch_compose_assign(int32_t* total, const int32_t* step, int64_t n
                                   cudaStream_t st);
 cudaError_t launch_decode(const DecodeArgs& a, int dtype, int D, cudaStream_t st);
 size_t round_smem_bytes(int chunk, int D);
+bool round_fast_supported(const RoundArgs& a, int dtype, int D);
+cudaError_t launch_round_fast(const RoundArgs& a, int64_t n_full, cudaStream_t st);
 
 }  // namespace ckv

@@ -37,7 +37,7 @@ def run_gpu_prefill(K, V, deg, p, want_assign=True, cap_extra=3):
     ws = torch.empty(b.workspace_bytes(src, p), dtype=torch.uint8, device=DEV)
     assign = torch.full((L, H, s), -7, dtype=torch.int32, device=DEV) if want_assign else None
     r = b.compress_prefill(src, dst, p, ws, assign)
-    torch.cuda.synchronize()
+    assert b.workspace_status(ws) == 0      # synchronises; nonzero would mean a bounded wait gave up
     assert r == rounds and dst.len == out_len
     return dst, assign, rounds
 
@@ -73,6 +73,15 @@ def test_round_all_edges(dtype, chunk, s, sink, recent):
     """Ratio 1: every edge merges; ragged last chunks, odd chunks, single-token chunks, degrees > 1 on input."""
     b = B()
     single_round_case(2, 3, s, dtype, one_round(b, chunk, 1.0, b.SELECT_GLOBAL, sink, recent), seed=chunk + s, deg_max=5)
+
+
+@pytest.mark.parametrize("deg_max", [1, 7])
+@pytest.mark.parametrize("s,sink,recent", [(64, 0, 0), (8192, 0, 0), (8229, 0, 0), (4000, 16, 64), (12345, 3, 1)])
+def test_round_bf16_chunk64_ratio1(deg_max, s, sink, recent):
+    """The configuration the benchmark times (bf16, chunk 64, ratio 1): many full chunks per head plus a shorter
+    last one, with and without degrees on input."""
+    b = B()
+    single_round_case(3, 5, s, "bf16", one_round(b, 64, 1.0, b.SELECT_GLOBAL, sink, recent), seed=s + deg_max, deg_max=deg_max)
 
 
 @pytest.mark.parametrize("dtype", ["f32", "bf16"])
