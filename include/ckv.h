@@ -133,6 +133,23 @@ int ckv_decode_attn(const ckv_layer_view* views_dev, int32_t Bz, int32_t H, int3
                     const void* q, void* out, float scale, int64_t max_len, void* workspace,
                     size_t workspace_bytes, void* cuda_stream);
 
+/* ckv_decode_attn for callers that cannot hand over a workspace because they cannot allocate device
+ * memory at the point of the call: code running inside a serving engine's steady-state loop whose memory
+ * pool is frozen after start-up, a plug-in that is given only its input and output tensors, or a host
+ * that must not call cudaMalloc (it synchronises the device).  The split partials go to a fixed 4 MiB
+ * array that is part of the library image, so every GPU that loads the library holds those 4 MiB until
+ * the process exits.  Same arguments, results and status codes as ckv_decode_attn, minus the workspace.
+ * Limits: Bz * H * G * 132 floats per split must fit in the array (1 Mi floats), else CKV_ERR_CAPACITY;
+ * when the usual number of sequence splits does not fit, fewer splits are used (slower, same result).
+ * The call allocates and frees nothing.  The first call on each device looks up the array's device
+ * address (a host-side runtime query, that device being current) and should therefore come before any
+ * stream capture.  All calls on a device share the one array, which keeps whatever the last call
+ * wrote (nothing in it needs clearing: each launch overwrites every partial it later reads); two
+ * calls whose kernels overlap on the GPU (different streams) race on it -- serialise them.
+ * The paper has no counterpart for this entry point. */
+int ckv_decode_attn_static(const ckv_layer_view* views_dev, int32_t Bz, int32_t H, int32_t G, int32_t D, int32_t dtype,
+                           const void* q, void* out, float scale, int64_t max_len, void* cuda_stream);
+
 /* Host-only: a static string for a ckv_status. */
 const char* ckv_status_string(int status);
 

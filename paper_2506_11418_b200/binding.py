@@ -19,7 +19,8 @@ SELECT_GLOBAL, SELECT_CHUNK = 0, 1
 OK = 0
 
 EXPORTS = ["ckv_compress_plan", "ckv_workspace_bytes", "ckv_compress_prefill", "ckv_compress_append",
-           "ckv_decode_workspace_bytes", "ckv_decode_attn", "ckv_status_string", "ckv_workspace_status"]
+           "ckv_decode_workspace_bytes", "ckv_decode_attn", "ckv_status_string", "ckv_workspace_status",
+           "ckv_decode_attn_static"]
 
 
 class CkvCache(C.Structure):
@@ -63,6 +64,9 @@ def _load():
     lib.ckv_decode_attn.restype = C.c_int
     lib.ckv_decode_attn.argtypes = [C.c_void_p, C.c_int32, C.c_int32, C.c_int32, C.c_int32, C.c_int32, C.c_void_p,
                                     C.c_void_p, C.c_float, C.c_int64, C.c_void_p, C.c_size_t, C.c_void_p]
+    lib.ckv_decode_attn_static.restype = C.c_int
+    lib.ckv_decode_attn_static.argtypes = [C.c_void_p, C.c_int32, C.c_int32, C.c_int32, C.c_int32, C.c_int32, C.c_void_p,
+                                           C.c_void_p, C.c_float, C.c_int64, C.c_void_p]
     return lib
 
 
@@ -201,3 +205,12 @@ def decode_attn(views: torch.Tensor, H: int, G: int, q: torch.Tensor, out: torch
     assert HG == H * G and q.is_contiguous() and out.is_contiguous()
     _check(lib.ckv_decode_attn(views.data_ptr(), Bz, H, G, D, dtype_code(q.dtype), q.data_ptr(), out.data_ptr(), scale,
                                max_len, workspace.data_ptr(), workspace.numel() * workspace.element_size(), _stream_ptr()))
+
+
+def decode_attn_static(views: torch.Tensor, H: int, G: int, q: torch.Tensor, out: torch.Tensor, scale: float, max_len: int):
+    """ckv_decode_attn_static on the current stream: decode attention without a caller workspace, for callers
+    that cannot allocate device memory; the split partials use a fixed 4 MiB array inside the library."""
+    Bz, HG, D = q.shape
+    assert HG == H * G and q.is_contiguous() and out.is_contiguous()
+    _check(lib.ckv_decode_attn_static(views.data_ptr(), Bz, H, G, D, dtype_code(q.dtype), q.data_ptr(), out.data_ptr(),
+                                      scale, max_len, _stream_ptr()))

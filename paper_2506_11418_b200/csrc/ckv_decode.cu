@@ -253,3 +253,56 @@ cudaError_t launch_decode(const DecodeArgs& a, int dtype, int D, cudaStream_t st
 }
 
 }  // namespace ckv
+
+// ---- entry point that allocates nothing ---------------------------------------------------------
+// Split partials live in a fixed array inside the library image instead of a caller workspace.
+namespace {
+
+constexpr size_t kStaticScratchFloats = (size_t)1 << 20;  // 4 MiB
+static __device__ __align__(256) float g_decode_scratch[kStaticScratchFloats];
+
+constexpr int kMaxDevices = 64;
+float* g_scratch_ptr[kMaxDevices];  // device address of g_decode_scratch per device, resolved on first use
+
+}  // namespace
+
+extern "C" int ckv_decode_attn_static(const ckv_layer_view* views_dev, int32_t Bz, int32_t H, int32_t G, int32_t D,
+                                      int32_t dtype, const void* q, void* out, float scale, int64_t max_len,
+                                      void* cuda_stream) {
+  if (!views_dev || !q || !out || Bz <= 0 || H <= 0 || G <= 0 || max_len < 0) return CKV_ERR_INVALID_ARG;
+  if (dtype != CKV_F32 && dtype != CKV_BF16) return CKV_ERR_INVALID_ARG;
+  if (D != 128 || G > 8 || H > 65535 || Bz > 65535) return CKV_ERR_UNSUPPORTED;
+  if ((reinterpret_cast<uintptr_t>(q) & 15u) || (reinterpret_cast<uintptr_t>(out) & 15u)) return CKV_ERR_ALIGNMENT;
+  const int64_t pairs = (int64_t)Bz * H;
+  const int64_t max_splits = max_len + 127 > 128 ? (max_len + 127) / 128 : 1;
+  int64_t n_splits = (4 * 148 + pairs - 1) / pairs;
+  if (n_splits > max_splits) n_splits = max_splits;
+  if (n_splits < 1) n_splits = 1;
+  // the fixed array bounds the problem size: shrink the split count to fit, reject if even one split does not
+  const int64_t per_split = pairs * G * (D + 4);
+  if (per_split > (int64_t)kStaticScratchFloats) return CKV_ERR_CAPACITY;
+  if (n_splits * per_split > (int64_t)kStaticScratchFloats) n_splits = (int64_t)kStaticScratchFloats / per_split;
+
+  int dev = -1;
+  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices) return CKV_ERR_CUDA;
+  if (!g_scratch_ptr[dev]) {
+    // In host code `g_decode_scratch` names a host-side shadow of the symbol, not device memory: ask the
+    // runtime for the address the array has on the current device and hand that to the kernels.
+    void* p = nullptr;
+    if (cudaGetSymbolAddress(&p, g_decode_scratch) != cudaSuccess || !p) return CKV_ERR_CUDA;
+    g_scratch_ptr[dev] = static_cast<float*>(p);
+  }
+  ckv::DecodeArgs a{};
+  a.views = views_dev;
+  a.q = q;
+  a.out = out;
+  a.partial = g_scratch_ptr[dev];
+  a.Bz = Bz;
+  a.H = H;
+  a.G = G;
+  a.n_splits = (int32_t)n_splits;
+  const int64_t span = ((max_len + n_splits - 1) / n_splits + 127) / 128 * 128;
+  a.span = span < 128 ? 128 : span;
+  a.scale = scale;
+  return ckv::launch_decode(a, dtype, D, static_cast<cudaStream_t>(cuda_stream)) == cudaSuccess ? CKV_OK : CKV_ERR_CUDA;
+}
