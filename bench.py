@@ -19,7 +19,6 @@ import json
 import math
 import os
 import statistics
-import subprocess
 import sys
 import time
 
@@ -57,43 +56,50 @@ def decode_bytes(rows, D, es):
 # --------------------------------------------------------------------------- clocks
 
 class ClockSampler:
-    FIELDS = "clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown," \
-             "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap"
+    """Samples SM clock and throttle reasons through NVML from a thread while the timed region runs (read-only)."""
 
-    def __init__(self, index: int):
-        self.proc = None
+    def __init__(self, index: int, period_s: float = 0.005):
+        import threading
+        self.samples, self.reasons, self.smax, self.err = [], set(), None, None
+        self._stop = threading.Event()
         try:
-            self.proc = subprocess.Popen(["nvidia-smi", "-i", str(index), f"--query-gpu={self.FIELDS}",
-                                          "--format=csv,noheader,nounits", "-lms", "100"],
-                                         stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
-        except OSError:
-            self.proc = None
+            import pynvml
+            pynvml.nvmlInit()
+            self.nv = pynvml
+            self.h = pynvml.nvmlDeviceGetHandleByIndex(index)
+            self.smax = float(pynvml.nvmlDeviceGetMaxClockInfo(self.h, pynvml.NVML_CLOCK_SM))
+        except Exception as e:  # noqa: BLE001
+            self.nv, self.err = None, f"nvml unavailable: {e}"
+            return
+        self.period = period_s
+        self.thread = threading.Thread(target=self._run, daemon=True)
+        self.thread.start()
+
+    def _run(self):
+        nv = self.nv
+        names = {"hw_slowdown": nv.nvmlClocksThrottleReasonHwSlowdown,
+                 "hw_thermal_slowdown": nv.nvmlClocksThrottleReasonHwThermalSlowdown,
+                 "sw_thermal_slowdown": nv.nvmlClocksThrottleReasonSwThermalSlowdown,
+                 "sw_power_cap": nv.nvmlClocksThrottleReasonSwPowerCap}
+        while not self._stop.is_set():
+            try:
+                self.samples.append(float(nv.nvmlDeviceGetClockInfo(self.h, nv.NVML_CLOCK_SM)))
+                mask = nv.nvmlDeviceGetCurrentClocksThrottleReasons(self.h)
+                for n, bit in names.items():
+                    if mask & bit:
+                        self.reasons.add(n)
+            except Exception as e:  # noqa: BLE001
+                self.err = str(e)
+                return
+            self._stop.wait(self.period)
 
     def stop(self):
-        if self.proc is None:
-            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
-        self.proc.terminate()
-        try:
-            out, _ = self.proc.communicate(timeout=5)
-        except subprocess.TimeoutExpired:
-            self.proc.kill()
-            out, _ = self.proc.communicate()
-        sm, smax, reasons = [], None, set()
-        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
-        for line in out.strip().splitlines():
-            f = [x.strip() for x in line.split(",")]
-            if len(f) < 7:
-                continue
-            try:
-                sm.append(float(f[0]))
-                smax = float(f[1])
-            except ValueError:
-                continue
-            for n, v in zip(names, f[3:7]):
-                if v.lower().startswith("active"):
-                    reasons.add(n)
-        return {"sm_mhz": statistics.median(sm) if sm else None, "sm_max_mhz": smax, "reasons": sorted(reasons),
-                "samples": len(sm)}
+        if self.nv is None:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": [self.err]}
+        self._stop.set()
+        self.thread.join(timeout=2)
+        return {"sm_mhz": statistics.median(self.samples) if self.samples else None, "sm_max_mhz": self.smax,
+                "reasons": sorted(self.reasons), "samples": len(self.samples)}
 
 
 # --------------------------------------------------------------------------- CPU oracle leg
@@ -169,6 +175,8 @@ def run_gpu(args):
 
     cfg = synth.CONFIGS[WORKLOAD]
     L, H, G, s, D, c = cfg["L"], cfg["H"], cfg["G"], cfg["s"], cfg["d"], cfg["chunk"]
+    if args.layers > 0:
+        L = args.layers
     es = 2
     seed = cfg["seed"] + 7919 * rank
     K = synth.ar1_keys(L, H, s, D, cfg["rho"], cfg["mean_std"], seed=seed, dtype="bf16", device=dev)
@@ -249,7 +257,7 @@ def run_gpu(args):
     extra = {"compress_ms": comp_ms, "compress_tokens_per_s": s / (comp_ms * 1e-3), "decode_ms_all_layers": dec_ms,
              "decode_gbs_batch1": dec_achieved}
 
-    if rank == 0 and not args.skip_decode_cfg4:
+    if rank == 0 and not args.skip_decode_cfg4 and args.layers == 0:
         extra["decode_cfg4"] = bench_decode_cfg4(b, synth, dev, peaks["hbm_gbs"])
 
     # end to end: inputs start in pinned host memory, the compressed cache and the decode output end there
@@ -272,7 +280,7 @@ def run_gpu(args):
         line = {"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": max(args.warmup, 3),
                 "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "bf16",
                 "data": "synthetic",
-                "config": {"workload": WORKLOAD, "layers": L, "kv_heads": H, "q_heads": H * G, "head_dim": D, "seq": s,
+                "config": {"workload": WORKLOAD if args.layers == 0 else f"{WORKLOAD} cut to {L} layers (not the benchmark workload)", "layers": L, "kv_heads": H, "q_heads": H * G, "head_dim": D, "seq": s,
                            "chunk": c, "retain": out_len / s, "step": "compress_prefill + append 64 + decode all layers",
                            "l2": "inputs (4 GiB) exceed L2"},
                 "clocks": clocks, "e2e": e2e, "gpu_launches": launches_per_step * args.steps, "roofline": roofline,
@@ -370,6 +378,7 @@ def main():
     ap.add_argument("--steps", type=int, default=20)
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="ckv", choices=["ckv", "reference"])
+    ap.add_argument("--layers", type=int, default=0, help="use only this many layers of the workload (profiling a small case)")
     ap.add_argument("--skip-e2e", action="store_true")
     ap.add_argument("--skip-cpu", action="store_true")
     ap.add_argument("--skip-decode-cfg4", action="store_true")

@@ -423,10 +423,7 @@ int ckv_workspace_status(const void* workspace, void* cuda_stream, int32_t* stat
 
 size_t ckv_decode_workspace_bytes(int32_t Bz, int32_t H, int32_t G, int32_t D, int64_t max_len) {
   if (Bz <= 0 || H <= 0 || G <= 0 || D <= 0 || max_len < 0) return 0;
-  const int64_t max_splits = std::max<int64_t>(1, (max_len + 127) / 128);
-  const int64_t want = (4 * 148 + (int64_t)Bz * H - 1) / ((int64_t)Bz * H);
-  const int64_t n_splits = std::max<int64_t>(1, std::min(want, max_splits));
-  return align_up((size_t)Bz * H * G * n_splits * (D + 4) * 4) + 256;
+  return align_up(decode_partial_floats(Bz, H, G, D, max_len) * sizeof(float)) + 256;
 }
 
 int ckv_decode_attn(const ckv_layer_view* views_dev, int32_t Bz, int32_t H, int32_t G, int32_t D, int32_t dtype,
@@ -438,14 +435,11 @@ int ckv_decode_attn(const ckv_layer_view* views_dev, int32_t Bz, int32_t H, int3
   if (!aligned16(q) || !aligned16(out)) return CKV_ERR_ALIGNMENT;
   const size_t need = ckv_decode_workspace_bytes(Bz, H, G, D, max_len);
   if (!workspace || workspace_bytes < need || !aligned16(workspace)) return CKV_ERR_WORKSPACE;
-  const int64_t max_splits = std::max<int64_t>(1, (max_len + 127) / 128);
-  const int64_t want = (4 * 148 + (int64_t)Bz * H - 1) / ((int64_t)Bz * H);
   DecodeArgs a{};
   a.views = views_dev; a.q = q; a.out = out;
   a.partial = static_cast<float*>(workspace);
   a.Bz = Bz; a.H = H; a.G = G;
-  a.n_splits = (int32_t)std::max<int64_t>(1, std::min(want, max_splits));
-  a.span = std::max<int64_t>(128, ((max_len + a.n_splits - 1) / a.n_splits + 127) / 128 * 128);
+  decode_plan(Bz, H, dtype, max_len, 0, G, D, &a.n_splits, &a.span);
   a.scale = scale;
   return launch_decode(a, dtype, D, static_cast<cudaStream_t>(cuda_stream)) == cudaSuccess ? CKV_OK : CKV_ERR_CUDA;
 }

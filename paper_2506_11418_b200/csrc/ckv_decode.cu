@@ -3,6 +3,7 @@
 // Split-K flash decoding: grid (split, KV head, sequence); each warp walks tiles of 32 tokens of
 // its CTA's span with an online softmax, partial (max, sum, out[D]) per split go to the
 // workspace and a second kernel combines them.  Scores and sums are fp32 in the exp2 domain.
+#include <algorithm>
 #include <cfloat>
 
 #include "../../include/ckv.h"
@@ -72,7 +73,7 @@ template <typename T, int D, int G>
 __global__ void __launch_bounds__(kDecThreads) decode_split_kernel(const DecodeArgs a) {
   static_assert(D == 128 && G <= kMaxG, "one lane owns four output columns");
   using S = DecodeSmem<T, D>;
-  extern __shared__ __align__(16) unsigned char smem_raw[];
+  extern __shared__ __align__(128) unsigned char smem_raw[];
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const int split = blockIdx.x, h = blockIdx.y, b = blockIdx.z;
   unsigned char* ktile = smem_raw + warp * S::kTileBytes;
@@ -247,9 +248,261 @@ cudaError_t launch_decode_t(const DecodeArgs& a, cudaStream_t st) {
 
 }  // namespace
 
+namespace {
+
+// ---- fast path: bf16, tensor cores, warp-private cp.async pipeline ------------------------------------
+// Each warp walks its own span of the sequence in tiles of 32 tokens through a 3-stage ring in shared
+// memory (K tile, V tile, log-degrees), filled with 16-byte cp.async copies into an XOR-swizzled layout
+// so that ldmatrix is conflict-free.  Per tile:
+//   S[head, token]   = Q K^T      mma.sync m16n8k16 (heads padded to 16 rows, K through ldmatrix)
+//   online softmax in the exp2 domain with the log-degree bias of Eq. 3
+//   O^T[d, head]    += V^T P      mma.sync, V through ldmatrix.trans; P is the score accumulator re-packed
+//                                 to bf16, already in the layout the B operand needs
+// No CTA-wide barrier is used; a warp whose split is empty leaves at once.
+
+constexpr int kFT = 32;                         // tokens per tile
+constexpr int kFStages = 3;
+constexpr int kFWarps = 4;
+constexpr int kFTileBytes = kFT * 256;          // one bf16 tile of K or V
+constexpr int kFStageBytes = 2 * kFTileBytes + kFT * 4;
+constexpr size_t kFSmemBytes = (size_t)kFWarps * kFStages * kFStageBytes;
+
+__device__ __forceinline__ void cp_async16(uint32_t dst, const void* src, uint32_t src_bytes) {
+  asm volatile("cp.async.cg.shared.global [%0], [%1], 16, %2;" ::"r"(dst), "l"(src), "r"(src_bytes) : "memory");
+}
+__device__ __forceinline__ void cp_async4(uint32_t dst, const void* src, uint32_t src_bytes) {
+  asm volatile("cp.async.ca.shared.global [%0], [%1], 4, %2;" ::"r"(dst), "l"(src), "r"(src_bytes) : "memory");
+}
+__device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;" ::: "memory"); }
+template <int N>
+__device__ __forceinline__ void cp_async_wait() { asm volatile("cp.async.wait_group %0;" ::"n"(N) : "memory"); }
+
+__device__ __forceinline__ void ldsm_x4(uint32_t addr, uint32_t (&r)[4]) {
+  asm volatile("ldmatrix.sync.aligned.m8n8.x4.shared.b16 {%0,%1,%2,%3}, [%4];"
+               : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]) : "r"(addr));
+}
+__device__ __forceinline__ void ldsm_x4_trans(uint32_t addr, uint32_t (&r)[4]) {
+  asm volatile("ldmatrix.sync.aligned.m8n8.x4.trans.shared.b16 {%0,%1,%2,%3}, [%4];"
+               : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]) : "r"(addr));
+}
+__device__ __forceinline__ void mma_bf16_16816(float (&d)[4], uint32_t a0, uint32_t a1, uint32_t a2, uint32_t a3,
+                                               uint32_t b0, uint32_t b1) {
+  asm volatile(
+      "mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
+      : "+f"(d[0]), "+f"(d[1]), "+f"(d[2]), "+f"(d[3])
+      : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1));
+}
+
+__global__ void __launch_bounds__(kFWarps * 32, 1) decode_fast_kernel(const DecodeArgs a) {
+  constexpr int D = 128;
+  extern __shared__ __align__(128) unsigned char smem_raw[];
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+  const int g = lane >> 2, t = lane & 3;
+  const int split = blockIdx.x * kFWarps + warp;
+  if (split >= a.n_splits) return;
+  const int h = blockIdx.y, b = blockIdx.z, G = a.G;
+  const ckv_layer_view view = reinterpret_cast<const ckv_layer_view*>(a.views)[b];
+  const int64_t len = view.len;
+  const int64_t t_begin = min(len, (int64_t)split * a.span);
+  const int64_t t_end = min(len, t_begin + a.span);
+  const int ntiles = (int)((t_end - t_begin + kFT - 1) / kFT);
+  const __nv_bfloat16* kbase = reinterpret_cast<const __nv_bfloat16*>(view.k) + (int64_t)h * view.cap * D;
+  const __nv_bfloat16* vbase = reinterpret_cast<const __nv_bfloat16*>(view.v) + (int64_t)h * view.cap * D;
+  const float* ldbase = view.logdeg ? view.logdeg + (int64_t)h * view.cap : nullptr;
+  const uint32_t ring = (uint32_t)__cvta_generic_to_shared(smem_raw) + (uint32_t)warp * kFStages * kFStageBytes;
+  const float* ring_ld = reinterpret_cast<const float*>(smem_raw + (size_t)warp * kFStages * kFStageBytes);
+
+  // query fragments (A operand, rows = heads; rows >= G are zero)
+  uint32_t qa[8][2];
+  {
+    const uint32_t* qrow = reinterpret_cast<const uint32_t*>(reinterpret_cast<const __nv_bfloat16*>(a.q) +
+                                                             (((int64_t)b * a.H + h) * G + g) * D);
+#pragma unroll
+    for (int ks = 0; ks < 8; ++ks) {
+      qa[ks][0] = g < G ? qrow[8 * ks + t] : 0u;      // elements 16 ks + 2t, +1
+      qa[ks][1] = g < G ? qrow[8 * ks + 4 + t] : 0u;  // elements 16 ks + 8 + 2t, +1
+    }
+  }
+  const float sc = a.scale * kLog2e;
+
+  auto issue = [&](int tile) {
+    const int64_t t0 = t_begin + (int64_t)tile * kFT;
+    const uint32_t st = ring + (uint32_t)(tile % kFStages) * kFStageBytes;
+    const int c = lane & 15;
+#pragma unroll
+    for (int i = 0; i < 16; ++i) {
+      const int r = (lane >> 4) + 2 * i;
+      const bool ok = t0 + r < t_end;
+      const int64_t row = ok ? t0 + r : t_begin;  // clamped address, zero-filled when out of range
+      const uint32_t off = (uint32_t)r * 256u + (uint32_t)((c ^ (r & 7)) << 4);
+      cp_async16(st + off, kbase + row * D + c * 8, ok ? 16u : 0u);
+      cp_async16(st + kFTileBytes + off, vbase + row * D + c * 8, ok ? 16u : 0u);
+    }
+    if (ldbase) {  // one log-degree per lane; 4-byte copies have no alignment demands on the slab
+      const bool ok = t0 + lane < t_end;
+      cp_async4(st + 2 * kFTileBytes + lane * 4, ldbase + (ok ? t0 + lane : t_begin), ok ? 4u : 0u);
+    }
+  };
+
+  float oacc[8][4];
+#pragma unroll
+  for (int i = 0; i < 8; ++i) oacc[i][0] = oacc[i][1] = oacc[i][2] = oacc[i][3] = 0.f;
+  float m_run = -INFINITY, l_run = 0.f;  // for head g (this thread's share of the tokens)
+
+#pragma unroll
+  for (int i = 0; i < kFStages - 1; ++i) {
+    if (i < ntiles) issue(i);
+    cp_async_commit();
+  }
+  for (int tile = 0; tile < ntiles; ++tile) {
+    cp_async_wait<kFStages - 2>();
+    __syncwarp();
+    if (tile + kFStages - 1 < ntiles) issue(tile + kFStages - 1);
+    cp_async_commit();
+    const int stage = tile % kFStages;
+    const uint32_t ks_ = ring + (uint32_t)stage * kFStageBytes, vs_ = ks_ + kFTileBytes;
+    const float* lds = ring_ld + (size_t)stage * (kFStageBytes / 4) + 2 * kFTileBytes / 4;
+    const int nt = (int)min((int64_t)kFT, t_end - (t_begin + (int64_t)tile * kFT));
+
+    // ---- S = Q K^T for 32 tokens: n tile j covers tokens 8j .. 8j+7
+    float sacc[4][4];
+#pragma unroll
+    for (int j = 0; j < 4; ++j) sacc[j][0] = sacc[j][1] = sacc[j][2] = sacc[j][3] = 0.f;
+#pragma unroll
+    for (int kq = 0; kq < 4; ++kq) {
+#pragma unroll
+      for (int j = 0; j < 4; ++j) {
+        const int tok = 8 * j + (lane & 7);
+        const int chunk = 4 * kq + (lane >> 3);
+        uint32_t r[4];
+        ldsm_x4(ks_ + (uint32_t)tok * 256u + (uint32_t)((chunk ^ (tok & 7)) << 4), r);
+        mma_bf16_16816(sacc[j], qa[2 * kq][0], 0u, qa[2 * kq][1], 0u, r[0], r[1]);
+        mma_bf16_16816(sacc[j], qa[2 * kq + 1][0], 0u, qa[2 * kq + 1][1], 0u, r[2], r[3]);
+      }
+    }
+    // ---- bias, mask, online softmax (thread holds head g, tokens 8j + 2t, 8j + 2t + 1)
+    float p[4][2];
+    float tmax = -INFINITY;
+#pragma unroll
+    for (int j = 0; j < 4; ++j) {
+#pragma unroll
+      for (int e = 0; e < 2; ++e) {
+        const int tok = 8 * j + 2 * t + e;
+        float s = sacc[j][e] * sc + (ldbase ? lds[tok] * kLog2e : 0.f);
+        s = tok < nt ? s : -INFINITY;
+        p[j][e] = s;
+        tmax = fmaxf(tmax, s);
+      }
+    }
+    tmax = fmaxf(tmax, __shfl_xor_sync(0xffffffffu, tmax, 1));
+    tmax = fmaxf(tmax, __shfl_xor_sync(0xffffffffu, tmax, 2));
+    const float m_new = fmaxf(m_run, tmax);
+    const float corr = exp2f(m_run - m_new);
+    m_run = m_new;
+    float psum = 0.f;
+    uint32_t pb[4];
+#pragma unroll
+    for (int j = 0; j < 4; ++j) {
+      const float p0 = exp2f(p[j][0] - m_new), p1 = exp2f(p[j][1] - m_new);
+      psum += p0 + p1;
+      pb[j] = pack_bf16x2(p0, p1);
+    }
+    l_run = l_run * corr + psum;
+    // the output accumulator holds heads 2t and 2t+1: fetch their correction factors from quads 2t and 2t+1
+    const float c0 = __shfl_sync(0xffffffffu, corr, 8 * t), c1 = __shfl_sync(0xffffffffu, corr, 8 * t + 4);
+#pragma unroll
+    for (int i = 0; i < 8; ++i) {
+      oacc[i][0] *= c0; oacc[i][1] *= c1; oacc[i][2] *= c0; oacc[i][3] *= c1;
+    }
+    // ---- O^T += V^T P: m tile i covers d = 16 i .. 16 i + 15, k step s covers tokens 16 s .. 16 s + 15
+#pragma unroll
+    for (int s = 0; s < 2; ++s) {
+#pragma unroll
+      for (int i = 0; i < 8; ++i) {
+        const int mi = lane >> 3;
+        const int tok = 16 * s + 8 * (mi >> 1) + (lane & 7);
+        const int chunk = 2 * i + (mi & 1);
+        uint32_t r[4];
+        ldsm_x4_trans(vs_ + (uint32_t)tok * 256u + (uint32_t)((chunk ^ (tok & 7)) << 4), r);
+        mma_bf16_16816(oacc[i], r[0], r[1], r[2], r[3], pb[2 * s], pb[2 * s + 1]);
+      }
+    }
+  }
+  cp_async_wait<0>();
+
+  // ---- this split's partial: out[D], max, sum per query head
+  l_run += __shfl_xor_sync(0xffffffffu, l_run, 1);
+  l_run += __shfl_xor_sync(0xffffffffu, l_run, 2);
+  float* pbase = a.partial + ((((int64_t)b * a.H + h) * G) * a.n_splits + split) * (D + 4);
+  const int64_t hstride = (int64_t)a.n_splits * (D + 4);
+  if (t == 0 && g < G) {
+    pbase[g * hstride + D] = m_run;
+    pbase[g * hstride + D + 1] = l_run;
+  }
+#pragma unroll
+  for (int e = 0; e < 2; ++e) {
+    const int head = 2 * t + e;
+    if (head < G) {
+      float* dst = pbase + head * hstride;
+#pragma unroll
+      for (int i = 0; i < 8; ++i) {
+        dst[16 * i + g] = oacc[i][e];
+        dst[16 * i + 8 + g] = oacc[i][2 + e];
+      }
+    }
+  }
+}
+
+cudaError_t launch_decode_fast(const DecodeArgs& a, cudaStream_t st) {
+  cudaError_t e = cudaFuncSetAttribute(decode_fast_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kFSmemBytes);
+  if (e != cudaSuccess) return e;
+  const dim3 grid((unsigned)((a.n_splits + kFWarps - 1) / kFWarps), (unsigned)a.H, (unsigned)a.Bz);
+  decode_fast_kernel<<<grid, kFWarps * 32, kFSmemBytes, st>>>(a);
+  if ((e = cudaGetLastError()) != cudaSuccess) return e;
+  decode_combine_kernel<__nv_bfloat16, 128><<<(unsigned)(a.Bz * a.H * a.G), 32, 0, st>>>(a);
+  return cudaGetLastError();
+}
+
+}  // namespace
+
+// How a decode call is split over the sequence: the general kernel takes one span per CTA, the bf16
+// kernel one span per warp (four per CTA).
+void decode_plan(int32_t Bz, int32_t H, int dtype, int64_t max_len, int64_t max_partial_floats, int32_t G, int32_t D,
+                 int32_t* n_splits, int64_t* span) {
+  const int64_t pairs = (int64_t)Bz * H;
+  int64_t ns, gran;
+  if (dtype == 1) {
+    gran = 32;
+    const int64_t cap = std::max<int64_t>(1, (max_len + 127) / 128);  // at least 128 tokens per warp
+    ns = std::min(cap, (6 * 148 * 4 + pairs - 1) / pairs);
+    if (ns > 4) ns = (ns + 3) / 4 * 4;
+  } else {
+    gran = 128;
+    const int64_t cap = std::max<int64_t>(1, (max_len + 127) / 128);
+    ns = std::min(cap, (4 * 148 + pairs - 1) / pairs);
+  }
+  ns = std::max<int64_t>(ns, 1);
+  const int64_t per_split = pairs * G * (D + 4);
+  if (max_partial_floats > 0 && ns * per_split > max_partial_floats) ns = std::max<int64_t>(1, max_partial_floats / per_split);
+  *n_splits = (int32_t)ns;
+  *span = std::max<int64_t>(gran, ((max_len + ns - 1) / ns + gran - 1) / gran * gran);
+}
+
+size_t decode_partial_floats(int32_t Bz, int32_t H, int32_t G, int32_t D, int64_t max_len) {
+  size_t need = 0;
+  for (int dtype = 0; dtype < 2; ++dtype) {
+    int32_t ns;
+    int64_t span;
+    decode_plan(Bz, H, dtype, max_len, 0, G, D, &ns, &span);
+    need = std::max(need, (size_t)Bz * H * G * ns * (D + 4));
+  }
+  return need;
+}
+
 cudaError_t launch_decode(const DecodeArgs& a, int dtype, int D, cudaStream_t st) {
   if (D != 128) return cudaErrorInvalidValue;
-  return dtype == 0 ? launch_decode_t<float>(a, st) : launch_decode_t<__nv_bfloat16>(a, st);
+  if (dtype == 1) return launch_decode_fast(a, st);
+  return launch_decode_t<float>(a, st);
 }
 
 }  // namespace ckv
@@ -273,15 +526,12 @@ extern "C" int ckv_decode_attn_static(const ckv_layer_view* views_dev, int32_t B
   if (dtype != CKV_F32 && dtype != CKV_BF16) return CKV_ERR_INVALID_ARG;
   if (D != 128 || G > 8 || H > 65535 || Bz > 65535) return CKV_ERR_UNSUPPORTED;
   if ((reinterpret_cast<uintptr_t>(q) & 15u) || (reinterpret_cast<uintptr_t>(out) & 15u)) return CKV_ERR_ALIGNMENT;
-  const int64_t pairs = (int64_t)Bz * H;
-  const int64_t max_splits = max_len + 127 > 128 ? (max_len + 127) / 128 : 1;
-  int64_t n_splits = (4 * 148 + pairs - 1) / pairs;
-  if (n_splits > max_splits) n_splits = max_splits;
-  if (n_splits < 1) n_splits = 1;
-  // the fixed array bounds the problem size: shrink the split count to fit, reject if even one split does not
-  const int64_t per_split = pairs * G * (D + 4);
-  if (per_split > (int64_t)kStaticScratchFloats) return CKV_ERR_CAPACITY;
-  if (n_splits * per_split > (int64_t)kStaticScratchFloats) n_splits = (int64_t)kStaticScratchFloats / per_split;
+  // the fixed array bounds the problem size: fewer sequence splits when the usual count does not fit, rejected if
+  // even one split does not
+  if ((int64_t)Bz * H * G * (D + 4) > (int64_t)kStaticScratchFloats) return CKV_ERR_CAPACITY;
+  int32_t n_splits;
+  int64_t span;
+  ckv::decode_plan(Bz, H, dtype, max_len, (int64_t)kStaticScratchFloats, G, D, &n_splits, &span);
 
   int dev = -1;
   if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices) return CKV_ERR_CUDA;
@@ -300,9 +550,8 @@ extern "C" int ckv_decode_attn_static(const ckv_layer_view* views_dev, int32_t B
   a.Bz = Bz;
   a.H = H;
   a.G = G;
-  a.n_splits = (int32_t)n_splits;
-  const int64_t span = ((max_len + n_splits - 1) / n_splits + 127) / 128 * 128;
-  a.span = span < 128 ? 128 : span;
+  a.n_splits = n_splits;
+  a.span = span;
   a.scale = scale;
   return ckv::launch_decode(a, dtype, D, static_cast<cudaStream_t>(cuda_stream)) == cudaSuccess ? CKV_OK : CKV_ERR_CUDA;
 }

@@ -84,6 +84,9 @@ cudaError_t launch_select(const SelectArgs& a, cudaStream_t st);
 cudaError_t launch_compose_assign(int32_t* total, const int32_t* step, int64_t n_src, int64_t step_stride, int32_t LH,
                                   cudaStream_t st);
 cudaError_t launch_decode(const DecodeArgs& a, int dtype, int D, cudaStream_t st);
+void decode_plan(int32_t Bz, int32_t H, int dtype, int64_t max_len, int64_t max_partial_floats, int32_t G, int32_t D,
+                 int32_t* n_splits, int64_t* span);
+size_t decode_partial_floats(int32_t Bz, int32_t H, int32_t G, int32_t D, int64_t max_len);
 size_t round_smem_bytes(int chunk, int D);
 bool round_fast_supported(const RoundArgs& a, int dtype, int D);
 cudaError_t launch_round_fast(const RoundArgs& a, int64_t n_full, cudaStream_t st);
