@@ -257,7 +257,7 @@ def run_gpu(args):
     extra = {"compress_ms": comp_ms, "compress_tokens_per_s": s / (comp_ms * 1e-3), "decode_ms_all_layers": dec_ms,
              "decode_gbs_batch1": dec_achieved}
 
-    if rank == 0 and not args.skip_decode_cfg4 and args.layers == 0:
+    if rank == 0 and not args.skip_decode_cfg4:
         extra["decode_cfg4"] = bench_decode_cfg4(b, synth, dev, peaks["hbm_gbs"])
 
     # end to end: inputs start in pinned host memory, the compressed cache and the decode output end there
