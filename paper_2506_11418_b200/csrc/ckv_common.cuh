@@ -37,6 +37,16 @@ __device__ __forceinline__ void store4(__nv_bfloat16* p, float4 v) {
   *reinterpret_cast<uint2*>(p) = u;
 }
 
+// ---- programmatic dependent launch ------------------------------------------------------------
+// A kernel launched with the programmatic-stream-serialization attribute may become resident before
+// the kernel ahead of it in the stream has finished.  griddep_wait() blocks until that kernel has
+// completed and its writes are visible (a no-op for an ordinary launch), so it comes before the
+// first read of anything an earlier kernel may have written; griddep_launch() lets the next such
+// kernel in the stream start becoming resident.
+
+__device__ __forceinline__ void griddep_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+__device__ __forceinline__ void griddep_launch() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
+
 // ---- warp reductions ------------------------------------------------------------------------
 
 __device__ __forceinline__ float warp_sum(float x) {

@@ -198,24 +198,56 @@ __global__ void __launch_bounds__(kDecThreads) decode_split_kernel(const DecodeA
   }
 }
 
+// Merges the split partials of one query head: out = sum_s 2^(m_s - m) o_s / sum_s 2^(m_s - m) l_s.
+// One CTA per (sequence, query head); the four warps take every fourth split, a lane owns four columns.
+constexpr int kCombThreads = 128;
+
 template <typename T, int D>
-__global__ void __launch_bounds__(D / 4) decode_combine_kernel(const DecodeArgs a) {
+__global__ void __launch_bounds__(kCombThreads) decode_combine_kernel(const DecodeArgs a) {
+  static_assert(D == 128, "a lane owns four of the 128 columns");
+  constexpr int P = D + 4, W = kCombThreads / 32;
+  __shared__ float s_max[W];
+  __shared__ float s_sum[W];
+  __shared__ float4 s_out[W][32];
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const int64_t row = blockIdx.x;  // (b, query head)
-  const int lane4 = threadIdx.x;   // four output columns each
-  const float* p = a.partial + row * a.n_splits * (D + 4);
+  const int n = a.n_splits;
+  griddep_wait();
+  griddep_launch();
+  const float* p = a.partial + row * n * P;
   float mm = -INFINITY;
-  for (int s = 0; s < a.n_splits; ++s) mm = fmaxf(mm, p[(size_t)s * (D + 4) + D]);
+  for (int s = tid; s < n; s += kCombThreads) mm = fmaxf(mm, p[(size_t)s * P + D]);
+  mm = warp_max(mm);
+  if (lane == 0) s_max[warp] = mm;
+  __syncthreads();
+  mm = fmaxf(fmaxf(s_max[0], s_max[1]), fmaxf(s_max[2], s_max[3]));
+
   float4 o = make_float4(0.f, 0.f, 0.f, 0.f);
   float ll = 0.f;
-  for (int s = 0; s < a.n_splits; ++s) {
-    const float* r = p + (size_t)s * (D + 4);
-    const float f = (r[D] == -INFINITY) ? 0.f : exp2f(r[D] - mm);
-    const float4 x = *reinterpret_cast<const float4*>(r + lane4 * 4);
+#pragma unroll 4
+  for (int s = warp; s < n; s += W) {
+    const float* r = p + (size_t)s * P;
+    const float ms = r[D];
+    const float f = (ms == -INFINITY) ? 0.f : exp2f(ms - mm);
+    const float4 x = *reinterpret_cast<const float4*>(r + lane * 4);
     o.x = fmaf(f, x.x, o.x); o.y = fmaf(f, x.y, o.y); o.z = fmaf(f, x.z, o.z); o.w = fmaf(f, x.w, o.w);
     ll = fmaf(f, r[D + 1], ll);
   }
-  const float inv = ll > 0.f ? 1.f / ll : 0.f;
-  store4(reinterpret_cast<T*>(a.out) + row * D + lane4 * 4, make_float4(o.x * inv, o.y * inv, o.z * inv, o.w * inv));
+  s_out[warp][lane] = o;
+  if (lane == 0) s_sum[warp] = ll;
+  __syncthreads();
+  if (warp == 0) {
+    o = s_out[0][lane];
+    ll = s_sum[0];
+#pragma unroll
+    for (int w = 1; w < W; ++w) {
+      const float4 x = s_out[w][lane];
+      o.x += x.x; o.y += x.y; o.z += x.z; o.w += x.w;
+      ll += s_sum[w];
+    }
+    const float inv = ll > 0.f ? 1.f / ll : 0.f;
+    store4(reinterpret_cast<T*>(a.out) + row * D + lane * 4, make_float4(o.x * inv, o.y * inv, o.z * inv, o.w * inv));
+  }
 }
 
 template <typename T, int G>
@@ -227,8 +259,7 @@ cudaError_t launch_decode_g(const DecodeArgs& a, cudaStream_t st) {
   const dim3 grid((unsigned)a.n_splits, (unsigned)a.H, (unsigned)a.Bz);
   decode_split_kernel<T, D, G><<<grid, kDecThreads, smem, st>>>(a);
   if ((e = cudaGetLastError()) != cudaSuccess) return e;
-  decode_combine_kernel<T, D><<<(unsigned)(a.Bz * a.H * G), D / 4, 0, st>>>(a);
-  return cudaGetLastError();
+  return launch_dependent(decode_combine_kernel<T, D>, dim3((unsigned)(a.Bz * a.H * G)), dim3(kCombThreads), 0, st, a);
 }
 
 template <typename T>
@@ -299,12 +330,16 @@ __global__ void __launch_bounds__(kFWarps * 32, 1) decode_fast_kernel(const Deco
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
   const int g = lane >> 2, t = lane & 3;
   const int split = blockIdx.x * kFWarps + warp;
+  griddep_wait();    // the views, the queries and the partial buffer may belong to the kernel ahead in the stream
+  griddep_launch();  // the combine kernel may become resident; it waits for this grid before it reads
   if (split >= a.n_splits) return;
   const int h = blockIdx.y, b = blockIdx.z, G = a.G;
   const ckv_layer_view view = reinterpret_cast<const ckv_layer_view*>(a.views)[b];
   const int64_t len = view.len;
-  const int64_t t_begin = min(len, (int64_t)split * a.span);
-  const int64_t t_end = min(len, t_begin + a.span);
+  // the sequence's own tiles are dealt evenly to the splits (a ragged batch stays balanced)
+  const int64_t seq_tiles = (len + kFT - 1) / kFT;
+  const int64_t t_begin = kFT * (seq_tiles * split / a.n_splits);
+  const int64_t t_end = min(len, kFT * (seq_tiles * (split + 1) / a.n_splits));
   const int ntiles = (int)((t_end - t_begin + kFT - 1) / kFT);
   const __nv_bfloat16* kbase = reinterpret_cast<const __nv_bfloat16*>(view.k) + (int64_t)h * view.cap * D;
   const __nv_bfloat16* vbase = reinterpret_cast<const __nv_bfloat16*>(view.v) + (int64_t)h * view.cap * D;
@@ -457,10 +492,9 @@ cudaError_t launch_decode_fast(const DecodeArgs& a, cudaStream_t st) {
   cudaError_t e = cudaFuncSetAttribute(decode_fast_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kFSmemBytes);
   if (e != cudaSuccess) return e;
   const dim3 grid((unsigned)((a.n_splits + kFWarps - 1) / kFWarps), (unsigned)a.H, (unsigned)a.Bz);
-  decode_fast_kernel<<<grid, kFWarps * 32, kFSmemBytes, st>>>(a);
-  if ((e = cudaGetLastError()) != cudaSuccess) return e;
-  decode_combine_kernel<__nv_bfloat16, 128><<<(unsigned)(a.Bz * a.H * a.G), 32, 0, st>>>(a);
-  return cudaGetLastError();
+  if ((e = launch_dependent(decode_fast_kernel, grid, dim3(kFWarps * 32), kFSmemBytes, st, a)) != cudaSuccess) return e;
+  return launch_dependent(decode_combine_kernel<__nv_bfloat16, 128>, dim3((unsigned)(a.Bz * a.H * a.G)), dim3(kCombThreads), 0,
+                          st, a);
 }
 
 }  // namespace
@@ -472,10 +506,23 @@ void decode_plan(int32_t Bz, int32_t H, int dtype, int64_t max_len, int64_t max_
   const int64_t pairs = (int64_t)Bz * H;
   int64_t ns, gran;
   if (dtype == 1) {
+    // One CTA per SM (the rings fill its shared memory), four splits per CTA.  Choose the CTAs per (sequence, head)
+    // that minimise waves x (tiles per warp + a fixed cost of about two tile times per CTA), with at least four
+    // tiles per warp so that the ring has something to overlap.
     gran = 32;
-    const int64_t cap = std::max<int64_t>(1, (max_len + 127) / 128);  // at least 128 tokens per warp
-    ns = std::min(cap, (6 * 148 * 4 + pairs - 1) / pairs);
-    if (ns > 4) ns = (ns + 3) / 4 * 4;
+    const int64_t tiles = std::max<int64_t>(1, (max_len + kFT - 1) / kFT);
+    const int64_t max_cpp = std::min<int64_t>(64, std::max<int64_t>(1, tiles / (4 * kFWarps)));
+    int64_t best = 1, best_cost = INT64_MAX;
+    for (int64_t cpp = 1; cpp <= max_cpp; ++cpp) {
+      const int64_t waves = (pairs * cpp + 147) / 148;
+      const int64_t per_warp = (tiles + cpp * kFWarps - 1) / (cpp * kFWarps);
+      const int64_t cost = waves * (per_warp + 2);
+      if (cost < best_cost) {
+        best_cost = cost;
+        best = cpp;
+      }
+    }
+    ns = best * kFWarps;
   } else {
     gran = 128;
     const int64_t cap = std::max<int64_t>(1, (max_len + 127) / 128);

@@ -78,6 +78,24 @@ struct DecodeArgs {
   float scale;
 };
 
+// Launch with programmatic stream serialization: the kernel may become resident while the kernel ahead of it
+// in the stream drains; it must call griddep_wait() before it touches anything that kernel produced.
+template <typename... KArgs, typename... Args>
+inline cudaError_t launch_dependent(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t st,
+                                    Args&&... args) {
+  cudaLaunchConfig_t cfg{};
+  cfg.gridDim = grid;
+  cfg.blockDim = block;
+  cfg.dynamicSmemBytes = smem;
+  cfg.stream = st;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[0].val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = 1;
+  return cudaLaunchKernelEx(&cfg, kernel, static_cast<KArgs>(args)...);
+}
+
 cudaError_t launch_round(const RoundArgs& a, int dtype, int D, cudaStream_t st);
 cudaError_t launch_copy(const CopyArgs& a, int dtype, int D, cudaStream_t st);
 cudaError_t launch_select(const SelectArgs& a, cudaStream_t st);
