@@ -173,13 +173,17 @@ cudaError_t run_round(const RoundPlan& rp, const Buf& src, const Buf& dst, int L
   a.LH = LH;
   a.status = reinterpret_cast<int32_t*>(ws);
   a.edge_stride = (int64_t)rp.n_chunks * (chunk / 2);
+  // bf16 with chunk 64 / 128 / 256 runs on the tile kernel, everything else on the general one
+  auto launch_any = [&](const RoundArgs& x) {
+    return round_tile_supported(x, dtype, D) ? launch_round_tile(x, st) : launch_round(x, dtype, D, st);
+  };
   if (rp.mode == kModeExternal) {
     a.edge_sim = reinterpret_cast<float*>(ws + w.edge_sim);
     a.edge_b = reinterpret_cast<int32_t*>(ws + w.edge_b);
     a.sel = ws + w.sel;
     a.chunk_out_off = reinterpret_cast<int32_t*>(ws + w.chunk_off);
     a.mode = kModeMatchOnly;
-    if ((e = launch_round(a, dtype, D, st)) != cudaSuccess) return e;
+    if ((e = launch_any(a)) != cudaSuccess) return e;
     SelectArgs s{};
     s.edge_sim = a.edge_sim; s.sel = a.sel; s.chunk_out_off = a.chunk_out_off;
     s.edge_stride = a.edge_stride; s.M = rp.M; s.lo = rp.lo; s.chunk = chunk; s.n_chunks = rp.n_chunks; s.LH = LH;
@@ -187,7 +191,7 @@ cudaError_t run_round(const RoundPlan& rp, const Buf& src, const Buf& dst, int L
   }
   a.mode = rp.mode;
   if (round_fast_supported(a, dtype, D)) {
-    // full chunks on the fast kernel, the shorter last chunk (if any) on the general one
+    // ratio 1 at chunk 64: full chunks on the warp-per-chunk kernel, the shorter last chunk (if any) on its own
     const int64_t mid = rp.hi - rp.lo;
     const int64_t n_full = mid / chunk;
     if ((e = launch_round_fast(a, n_full, st)) != cudaSuccess) return e;
@@ -196,7 +200,7 @@ cudaError_t run_round(const RoundPlan& rp, const Buf& src, const Buf& dst, int L
     a.out_lo = rp.lo + n_full * a.out_stride;
     a.n_chunks = 1;
   }
-  return launch_round(a, dtype, D, st);
+  return launch_any(a);
 }
 
 // Runs the planned rounds from `src` into `dst` (ping-pong through the workspace's tmp cache).
