@@ -53,6 +53,29 @@ def decode_bytes(rows, D, es):
     return rows * (2 * D * es + 4)
 
 
+# --------------------------------------------------------------------------- DRAM traffic from the ncu capture
+
+# dram__bytes_read.sum + dram__bytes_write.sum of round_fast_kernel per token-vector, from the capture summarised in
+# profiles/round_fast_kernel_llama8b_4layers.md (1 048 576 token-vectors per launch; traffic grows in proportion to
+# the token-vectors processed, so it is scaled to the launch timed here).  Valid only for the kernel source it
+# was taken from: the digest below is of ckv_compress_fast.cu at that time.
+NCU_TRAFFIC = {"bytes_per_token_vector": (536906240 + 238654976) / 1048576,
+               "source": "paper_2506_11418_b200/csrc/ckv_compress_fast.cu",
+               "sha256": "35b926748f5ee0c98632724ff5ddf6213e90e13ba1e3ebcac1929a9613547c85"}
+
+
+def ncu_traffic(token_vectors: int):
+    import hashlib
+    try:
+        with open(os.path.join(ROOT, NCU_TRAFFIC["source"]), "rb") as f:
+            digest = hashlib.sha256(f.read()).hexdigest()
+    except OSError:
+        return None
+    if digest != NCU_TRAFFIC["sha256"]:
+        return None  # the kernel has changed since the counters were taken
+    return NCU_TRAFFIC["bytes_per_token_vector"] * token_vectors
+
+
 # --------------------------------------------------------------------------- clocks
 
 class ClockSampler:
@@ -137,9 +160,8 @@ def oracle_pass(x) -> float:
 
 
 def run_reference(args):
-    rank = int(os.environ.get("RANK", "0"))
-    if rank != 0:
-        return
+    if int(os.environ.get("RANK", "0")) != 0:
+        return  # under a multi-rank launch rank 0 alone times the oracle
     x = oracle_inputs(2)
     for _ in range(min(args.warmup, 1)):
         oracle_pass(x)
@@ -159,26 +181,22 @@ def run_reference(args):
 
 def run_gpu(args):
     import torch
-    import torch.distributed as dist
 
-    from paper_2506_11418_b200 import binding as b, synth
+    from paper_2506_11418_b200 import binding as b, parallel, synth
 
-    world = int(os.environ.get("WORLD_SIZE", "1"))
-    rank = int(os.environ.get("RANK", "0"))
-    local = int(os.environ.get("LOCAL_RANK", "0"))
+    rank, local, world = parallel.env_world()
     if not torch.cuda.is_available():
         raise SystemExit("bench.py needs a CUDA device; there is no CPU fallback")
     torch.cuda.set_device(local)
     dev = torch.device("cuda", local)
-    if world > 1:
-        dist.init_process_group("nccl", device_id=dev)
+    parallel.init("nccl", dev)
 
     cfg = synth.CONFIGS[WORKLOAD]
     L, H, G, s, D, c = cfg["L"], cfg["H"], cfg["G"], cfg["s"], cfg["d"], cfg["chunk"]
     if args.layers > 0:
         L = args.layers
     es = 2
-    seed = cfg["seed"] + 7919 * rank
+    seed = parallel.rank_seed(cfg["seed"], rank)
     K = synth.ar1_keys(L, H, s, D, cfg["rho"], cfg["mean_std"], seed=seed, dtype="bf16", device=dev)
     V = synth.normal_values(L, H, s, D, seed=seed, dtype="bf16", device=dev)
     kn = synth.ar1_keys(L, H, c, D, cfg["rho"], cfg["mean_std"], seed=seed + 1, dtype="bf16", device=dev)
@@ -221,9 +239,7 @@ def run_gpu(args):
         assert dst.len == final_len
 
     def barrier():
-        if world > 1:
-            dist.barrier()
-        torch.cuda.synchronize()
+        parallel.barrier(dev)
 
     for _ in range(max(args.warmup, 3)):
         step(False)
@@ -236,11 +252,7 @@ def run_gpu(args):
     t_end.record()
     barrier()
     clocks = sampler.stop() if sampler else None
-    elapsed_ms = t_start.elapsed_time(t_end)
-    if world > 1:
-        t = torch.tensor([elapsed_ms], device=dev)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        elapsed_ms = float(t.item())
+    elapsed_ms = parallel.max_over_ranks(t_start.elapsed_time(t_end), dev)
     ms_per_step = elapsed_ms / args.steps
     value = world * s * args.steps / (elapsed_ms * 1e-3)
 
@@ -251,7 +263,8 @@ def run_gpu(args):
     achieved = cbytes / (comp_ms * 1e-3) / 1e9
     roofline = {"bound": "hbm", "kernel": "compress round kernel (one launch per ckv_compress_prefill)", "achieved": achieved,
                 "peak": peaks["hbm_gbs"], "peak_kind": peak_kind, "unit": "GB/s", "frac": achieved / peaks["hbm_gbs"],
-                "traffic": None, "bytes_per_launch": cbytes, "ms_per_launch": comp_ms}
+                "traffic": ncu_traffic(L * H * s), "bytes_per_launch": cbytes, "ms_per_launch": comp_ms,
+                "frac_of_nominal_8tbs": achieved / 8000.0}
     dbytes = decode_bytes(H * final_len, D, es)
     dec_achieved = dbytes * L / (dec_ms * 1e-3) / 1e9
     extra = {"compress_ms": comp_ms, "compress_tokens_per_s": s / (comp_ms * 1e-3), "decode_ms_all_layers": dec_ms,
@@ -265,9 +278,7 @@ def run_gpu(args):
     if not args.skip_e2e:
         e2e = bench_e2e(b, torch, dev, K, V, kn, vn, q, step, dst, final_len, out, s, world, max(2, min(args.steps, 5)))
         if world > 1:
-            t = torch.tensor([e2e["ms_per_step"]], device=dev)
-            dist.all_reduce(t, op=dist.ReduceOp.MAX)
-            e2e["ms_per_step"] = float(t.item())
+            e2e["ms_per_step"] = parallel.max_over_ranks(e2e["ms_per_step"], dev)
             e2e["value"] = world * s / (e2e["ms_per_step"] * 1e-3)
 
     cpu = None
@@ -286,8 +297,7 @@ def run_gpu(args):
                 "clocks": clocks, "e2e": e2e, "gpu_launches": launches_per_step * args.steps, "roofline": roofline,
                 "cpu_baseline": cpu, "detail": extra}
         print(json.dumps(line))
-    if world > 1:
-        dist.destroy_process_group()
+    parallel.finish()
 
 
 def bench_e2e(b, torch, dev, K, V, kn, vn, q, step, dst, final_len, out, s, world, iters):

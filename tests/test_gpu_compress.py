@@ -149,10 +149,16 @@ def test_short_sequences_are_copied():
 
 
 def multi_round_case(L, H, s, dtype, p, seed):
-    """End to end against the oracle's multi-round driver; if a near tie made the GPU choose differently,
-    fall back to checking every round against an oracle round fed with the GPU's own previous output."""
-    b = B()
     K, V, _ = make_inputs(L, H, s, dtype, seed)
+    return multi_round_check(K, V, dtype, p)
+
+
+def multi_round_check(K, V, dtype, p):
+    """End to end against the oracle's multi-round driver; if a near tie made the GPU choose differently,
+    fall back to checking every round against an oracle round fed with the GPU's own previous output.
+    Returns the statistics, with the GPU result under "dst" and "assign"."""
+    b = B()
+    L, H, s, _ = K.shape
     dst, assign, rounds = run_gpu_prefill(K, V, None, p)
     po = PU.oracle_params(p)
     Ko, Vo, do, asg, logs = O.compress_prefill(PU.to_np64(K), PU.to_np64(V), None, po, storage=dtype)
@@ -160,7 +166,7 @@ def multi_round_case(L, H, s, dtype, p, seed):
     g = PU.gpu_cache_to_np(dst, assign)
     # invariants that hold whatever the clusters are: degrees sum to the original length (Sec. 3)
     np.testing.assert_array_equal(g["deg"].sum(axis=2), np.full((L, H), s))
-    stats = dict(rounds=rounds)
+    stats = dict(rounds=rounds, dst=dst, assign=assign)
     if np.array_equal(g["assign"], asg):
         np.testing.assert_array_equal(g["deg"], do)
         for l in range(L):
