@@ -167,14 +167,23 @@ cudaError_t run_round(const RoundPlan& rp, const Buf& src, const Buf& dst, int L
   a.src_cap = src.cap; a.dst_cap = dst.cap;
   a.lo = rp.lo; a.hi = rp.hi;
   a.chunk = chunk; a.n_chunks = rp.n_chunks;
+  a.chunk_first = 0; a.n_launch = rp.n_chunks;
   a.m_full = rp.m_full; a.m_tail = rp.m_tail;
   a.out_stride = chunk - rp.m_full;
   a.out_lo = rp.lo;
   a.LH = LH;
   a.status = reinterpret_cast<int32_t*>(ws);
   a.edge_stride = (int64_t)rp.n_chunks * (chunk / 2);
-  // bf16 with chunk 64 / 128 / 256 runs on the tile kernel, everything else on the general one
-  auto launch_any = [&](const RoundArgs& x) {
+  // bf16 with chunk 64 / 128 / 256 runs on the tile kernel, everything else on the general one; at chunk 64 the full
+  // chunks go to the warp-per-chunk kernel and only the shorter last chunk (if any) to the tile kernel
+  auto launch_pass = [&](RoundArgs x) -> cudaError_t {
+    if (round_fast_supported(x, dtype, D)) {
+      const int64_t n_full = (rp.hi - rp.lo) / chunk;
+      cudaError_t err = launch_round_fast(x, n_full, st);
+      if (err != cudaSuccess || rp.n_chunks == n_full) return err;
+      x.chunk_first = (int32_t)n_full;
+      x.n_launch = 1;
+    }
     return round_tile_supported(x, dtype, D) ? launch_round_tile(x, st) : launch_round(x, dtype, D, st);
   };
   if (rp.mode == kModeExternal) {
@@ -183,24 +192,14 @@ cudaError_t run_round(const RoundPlan& rp, const Buf& src, const Buf& dst, int L
     a.sel = ws + w.sel;
     a.chunk_out_off = reinterpret_cast<int32_t*>(ws + w.chunk_off);
     a.mode = kModeMatchOnly;
-    if ((e = launch_any(a)) != cudaSuccess) return e;
+    if ((e = launch_pass(a)) != cudaSuccess) return e;
     SelectArgs s{};
     s.edge_sim = a.edge_sim; s.sel = a.sel; s.chunk_out_off = a.chunk_out_off;
     s.edge_stride = a.edge_stride; s.M = rp.M; s.lo = rp.lo; s.chunk = chunk; s.n_chunks = rp.n_chunks; s.LH = LH;
     if ((e = launch_select(s, st)) != cudaSuccess) return e;
   }
   a.mode = rp.mode;
-  if (round_fast_supported(a, dtype, D)) {
-    // ratio 1 at chunk 64: full chunks on the warp-per-chunk kernel, the shorter last chunk (if any) on its own
-    const int64_t mid = rp.hi - rp.lo;
-    const int64_t n_full = mid / chunk;
-    if ((e = launch_round_fast(a, n_full, st)) != cudaSuccess) return e;
-    if (rp.n_chunks == n_full) return cudaSuccess;
-    a.lo = rp.lo + n_full * chunk;
-    a.out_lo = rp.lo + n_full * a.out_stride;
-    a.n_chunks = 1;
-  }
-  return launch_any(a);
+  return launch_pass(a);
 }
 
 // Runs the planned rounds from `src` into `dst` (ping-pong through the workspace's tmp cache).

@@ -53,7 +53,7 @@ __global__ void __launch_bounds__(kRoundThreads) round_kernel(const RoundArgs a)
   int* outpos = selflag + hc;
 
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-  const int chunk_id = blockIdx.x;
+  const int chunk_id = a.chunk_first + blockIdx.x;
   const int lh = blockIdx.y;
   const int64_t beg = a.lo + (int64_t)chunk_id * c;
   const int clen = (int)min((int64_t)c, a.hi - beg);
@@ -387,9 +387,9 @@ size_t round_smem_bytes(int chunk, int D) { return D == 128 ? RoundSmem<128>::by
 
 cudaError_t launch_round(const RoundArgs& a, int dtype, int D, cudaStream_t st) {
   if (D != 128) return cudaErrorInvalidValue;
-  if (a.n_chunks <= 0) return cudaSuccess;
+  if (a.n_launch <= 0) return cudaSuccess;
   const size_t smem = RoundSmem<128>::bytes(a.chunk);
-  const dim3 grid((unsigned)a.n_chunks, (unsigned)a.LH);
+  const dim3 grid((unsigned)a.n_launch, (unsigned)a.LH);
   cudaError_t e;
   if (dtype == 0) {
     if ((e = set_smem(round_kernel<float, 128>, smem)) != cudaSuccess) return e;

@@ -139,12 +139,13 @@ __global__ void __launch_bounds__(TileCfg<C>::T, TileCfg<C>::kCtasPerSm) round_t
   __nv_bfloat16* k_dst = reinterpret_cast<__nv_bfloat16*>(a.k_dst);
   __nv_bfloat16* v_dst = reinterpret_cast<__nv_bfloat16*>(a.v_dst);
   const int n_chunks = a.n_chunks, LH = a.LH;
-  const int step_lh = (int)gridDim.x / n_chunks, step_ch = (int)gridDim.x % n_chunks;
+  const int n_launch = a.n_launch, ch_end = a.chunk_first + n_launch;  // this launch's chunks of every slab
+  const int step_lh = (int)gridDim.x / n_launch, step_ch = (int)gridDim.x % n_launch;
   auto advance = [&](Cursor& c) {
     c.lh += step_lh;
     c.ch += step_ch;
-    if (c.ch >= n_chunks) {
-      c.ch -= n_chunks;
+    if (c.ch >= ch_end) {
+      c.ch -= n_launch;
       ++c.lh;
     }
   };
@@ -170,7 +171,7 @@ __global__ void __launch_bounds__(TileCfg<C>::T, TileCfg<C>::kCtasPerSm) round_t
     cp_async_commit();
   };
   // Groups are committed in the order V(n + PV), K(n + PK) at the start of item n, after a prologue of the same shape.
-  Cursor cur{(int)blockIdx.x / n_chunks, (int)blockIdx.x % n_chunks};
+  Cursor cur{(int)blockIdx.x / n_launch, a.chunk_first + (int)blockIdx.x % n_launch};
   Cursor ahead = cur;  // item n + PK
   for (int j = 0; j < PK; ++j) {
     if (PV == PK) issue(ahead, j, true); else cp_async_commit();
@@ -495,7 +496,7 @@ template <int C>
 cudaError_t launch_tile_c(const RoundArgs& a, cudaStream_t st) {
   using Cfg = TileCfg<C>;
   static_assert(Cfg::kBytes <= 227 * 1024, "shared memory");
-  const int64_t n_items = (int64_t)a.n_chunks * a.LH;
+  const int64_t n_items = (int64_t)a.n_launch * a.LH;
   if (n_items <= 0) return cudaSuccess;
   cudaError_t e = cudaFuncSetAttribute(round_tile_kernel<C>, cudaFuncAttributeMaxDynamicSharedMemorySize, Cfg::kBytes);
   if (e != cudaSuccess) return e;

@@ -28,7 +28,9 @@ struct RoundArgs {
   int64_t src_cap, dst_cap;
   int64_t lo, hi;
   int64_t out_lo;          // dst position of the first chunk's first survivor (kModeAll, kModeChunkTopM)
-  int32_t chunk, n_chunks;
+  int32_t chunk, n_chunks;  // chunk size; chunks per slab (the stride of the per-chunk arrays)
+  int32_t chunk_first;      // this launch covers chunks [chunk_first, chunk_first + n_launch) of every slab
+  int32_t n_launch;
   int32_t mode;
   int32_t m_full, m_tail;  // kModeChunkTopM: merges in a full chunk / in the shorter last chunk
   int64_t out_stride;      // kModeAll, kModeChunkTopM: survivors of a full chunk
