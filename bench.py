@@ -59,9 +59,9 @@ def decode_bytes(rows, D, es):
 # profiles/round_fast_kernel_llama8b_4layers.md (1 048 576 token-vectors per launch; traffic grows in proportion to
 # the token-vectors processed, so it is scaled to the launch timed here).  Valid only for the kernel source it
 # was taken from: the digest below is of ckv_compress_fast.cu at that time.
-NCU_TRAFFIC = {"bytes_per_token_vector": (536906240 + 238654976) / 1048576,
+NCU_TRAFFIC = {"bytes_per_token_vector": (536905728 + 239911168) / 1048576,
                "source": "paper_2506_11418_b200/csrc/ckv_compress_fast.cu",
-               "sha256": "35b926748f5ee0c98632724ff5ddf6213e90e13ba1e3ebcac1929a9613547c85"}
+               "sha256": "b96ba7869f546928105c380bd1f9a43bde79e7911966ff761b457233a26960bf"}
 
 
 def ncu_traffic(token_vectors: int):
@@ -272,6 +272,8 @@ def run_gpu(args):
 
     if rank == 0 and not args.skip_decode_cfg4:
         extra["decode_cfg4"] = bench_decode_cfg4(b, synth, dev, peaks["hbm_gbs"])
+    if rank == 0 and not args.skip_variants:
+        extra["compress_variants"] = bench_compress_variants(b, synth, dev, K, V, peaks["hbm_gbs"], args.layers == 0)
 
     # end to end: inputs start in pinned host memory, the compressed cache and the decode output end there
     e2e = None
@@ -339,6 +341,68 @@ def bench_e2e(b, torch, dev, K, V, kn, vn, q, step, dst, final_len, out, s, worl
             "ms_per_step": ms, "steps": iters}
 
 
+def bench_compress_variants(b, synth, dev, K, V, peak_gbs, with_128k):
+    """ckv_compress_prefill alone on the same keys and values with other chunk sizes, ratios and ranking scopes (outside
+    the timed region).  `gbs` counts what the method has to move if every round read its input once and wrote its
+    output once; a round that ranks across chunks reads K twice, which is not credited."""
+    import torch
+    L, H, s, D = K.shape
+    P = b.Params
+    paper = dict(n_sink=16, n_recent=64, n_rounds_max=16, r_init=0.8, r_decay=0.2, r_min=0.2)
+    variants = [
+        ("chunk64 ratio1 sinks16 recent64", P(chunk=64, n_sink=16, n_recent=64, n_rounds_max=1, r_init=1.0, r_decay=0.0, r_min=1.0)),
+        ("chunk64 ratio0.5 ranked per chunk", P(chunk=64, n_sink=0, n_recent=0, n_rounds_max=1, r_init=0.5, r_decay=0.0, r_min=0.5, select=b.SELECT_CHUNK)),
+        ("chunk64 ratio0.8 ranked per head", P(chunk=64, n_sink=16, n_recent=64, n_rounds_max=1, r_init=0.8, r_decay=0.0, r_min=0.8)),
+        ("chunk128 ratio1", P(chunk=128, n_sink=0, n_recent=0, n_rounds_max=1, r_init=1.0, r_decay=0.0, r_min=1.0)),
+        ("chunk256 ratio1", P(chunk=256, n_sink=0, n_recent=0, n_rounds_max=1, r_init=1.0, r_decay=0.0, r_min=1.0)),
+        ("chunk64 paper schedule to 25%", P(chunk=64, budget=s // 4, **paper)),
+        ("chunk256 paper schedule to 25%", P(chunk=256, budget=s // 4, **paper)),
+    ]
+    res = {}
+
+    def time_one(name, Kx, Vx, p, iters):
+        n = Kx.shape[2]
+        src = b.Cache(Kx, Vx, None, None, n)
+        out_len, rounds, cap = b.compress_plan(n, p)
+        dst = b.Cache.empty(L, H, cap, D, Kx.dtype, dev)
+        ws = torch.empty(b.workspace_bytes(src, p), dtype=torch.uint8, device=dev)
+        for _ in range(2):
+            b.compress_prefill(src, dst, p, ws)
+        torch.cuda.synchronize()
+        t0, t1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        t0.record()
+        for _ in range(iters):
+            b.compress_prefill(src, dst, p, ws)
+        t1.record()
+        torch.cuda.synchronize()
+        ms = t0.elapsed_time(t1) / iters
+        # every round reads its input once and writes its output once
+        lens, cur = [n], n
+        for j in range(rounds):
+            pj = P(chunk=p.chunk, n_sink=p.n_sink, n_recent=p.n_recent, n_rounds_max=j + 1, r_init=p.r_init, r_decay=p.r_decay,
+                   r_min=p.r_min, select=p.select, budget=p.budget)
+            cur = b.compress_plan(n, pj)[0]
+            lens.append(cur)
+        nbytes = sum(L * H * (lens[j] * (2 * D * 2 + 4) + lens[j + 1] * (2 * D * 2 + 8)) for j in range(rounds))
+        res[name] = {"seq": n, "out_len": out_len, "rounds": rounds, "ms": ms, "tokens_per_s": n / (ms * 1e-3),
+                     "gbs": nbytes / (ms * 1e-3) / 1e9, "frac_of_peak": nbytes / (ms * 1e-3) / 1e9 / peak_gbs,
+                     "status": b.workspace_status(ws)}
+        del dst, ws
+
+    for name, p in variants:
+        time_one(name, K, V, p, 5)
+    if with_128k:
+        cfg = synth.CONFIGS["llama8b_128k"]
+        K3 = synth.ar1_keys(L, H, cfg["s"], D, cfg["rho"], cfg["mean_std"], seed=cfg["seed"], dtype="bf16", device=dev)
+        V3 = synth.normal_values(L, H, cfg["s"], D, seed=cfg["seed"], dtype="bf16", device=dev)
+        time_one("llama8b_128k chunk64 two rounds ratio1 (to 25%)", K3, V3,
+                 P(chunk=64, n_sink=0, n_recent=0, n_rounds_max=2, r_init=1.0, r_decay=0.0, r_min=1.0), 3)
+        time_one("llama8b_128k chunk64 paper schedule to 25%", K3, V3, P(chunk=64, budget=cfg["s"] // 4, **paper), 3)
+        del K3, V3
+    torch.cuda.empty_cache()
+    return res
+
+
 def bench_decode_cfg4(b, synth, dev, peak_gbs):
     """Decode attention on the batch-32 shape: 8192 centroids (+256 appended) vs the uncompressed 32768-token cache."""
     import torch
@@ -392,6 +456,7 @@ def main():
     ap.add_argument("--skip-e2e", action="store_true")
     ap.add_argument("--skip-cpu", action="store_true")
     ap.add_argument("--skip-decode-cfg4", action="store_true")
+    ap.add_argument("--skip-variants", action="store_true")
     args = ap.parse_args()
     if args.impl == "reference":
         run_reference(args)
