@@ -274,6 +274,7 @@ def run_gpu(args):
         extra["decode_cfg4"] = bench_decode_cfg4(b, synth, dev, peaks["hbm_gbs"])
     if rank == 0 and not args.skip_variants:
         extra["compress_variants"] = bench_compress_variants(b, synth, dev, K, V, peaks["hbm_gbs"], args.layers == 0)
+        extra["recluster"] = bench_recluster(b, synth, dev, K, V)
 
     # end to end: inputs start in pinned host memory, the compressed cache and the decode output end there
     e2e = None
@@ -401,6 +402,42 @@ def bench_compress_variants(b, synth, dev, K, V, peak_gbs, with_128k):
         del K3, V3
     torch.cuda.empty_cache()
     return res
+
+
+def bench_recluster(b, synth, dev, K, V):
+    """Fixed-budget decoding branch (ckv_compress_append_recluster): a cache of B = 8192 slots per head with degrees
+    above one, g = 256 appended tokens, then the re-clustering round over the whole cache back to B (paper defaults:
+    16 sinks, 64 recent tokens, ratio 0.8, ranked per head)."""
+    import torch
+    L, H, _, D = K.shape
+    B, g = 8192, 256
+    p = b.Params(chunk=64, n_sink=16, n_recent=64, n_rounds_max=1, r_init=0.8, r_decay=0.2, r_min=0.2, budget=B)
+    live, spare = (b.Cache.empty(L, H, B + g, D, K.dtype, dev) for _ in range(2))
+    for c in (live, spare):
+        c.k.copy_(K[:, :, :B + g])
+        c.v.copy_(V[:, :, :B + g])
+        c.deg.fill_(4)
+        c.logdeg.fill_(math.log(4.0))
+    live.len = B
+    shape = b.Cache.empty(1, 1, 1, D, K.dtype, dev)
+    shape.k = live.k
+    shape.v = live.v
+    shape.len = B + g
+    ws = torch.empty(b.workspace_bytes(shape, p), dtype=torch.uint8, device=dev)
+    kn, vn = K[:, :, B:B + g].contiguous(), V[:, :, B:B + g].contiguous()
+    times = []
+    for it in range(7):
+        t0, t1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        t0.record()
+        calls = b.compress_append_recluster(live, spare, kn, vn, p, g, ws)
+        t1.record()
+        torch.cuda.synchronize()
+        assert calls == 1 and live.len == B
+        if it >= 2:
+            times.append(t0.elapsed_time(t1))
+    ms = statistics.mean(times)
+    return {"budget": B, "interval": g, "ms_per_trigger_all_layers": ms, "us_per_decode_step_amortised": 1e3 * ms / g,
+            "status": b.workspace_status(ws)}
 
 
 def bench_decode_cfg4(b, synth, dev, peak_gbs):

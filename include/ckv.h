@@ -106,6 +106,20 @@ int ckv_compress_prefill(const ckv_cache* src, ckv_cache* dst, const ckv_params*
 int ckv_compress_append(ckv_cache* cache, const void* k_new, const void* v_new, int32_t t_new,
                         const ckv_params* params, void* workspace, size_t workspace_bytes, void* cuda_stream);
 
+/* Algorithm 1, decoding branch, as printed: `K = [K, k], V = [V, v], N = [N, 1]`, and `if s >= B + g` one call of
+ * CentroidKV over the whole cache, with B = params->budget (> 0) and g = interval (> 0).  The round keeps the sinks
+ * and recent tokens, carries the degrees along, uses the ratio of round 0 (params->r_init; n_rounds_max is not
+ * used) and, with CKV_SELECT_GLOBAL, merges min(floor(r * n_edges), s - B) edges, so the cache returns to B whenever
+ * the ratio allows.  A round cannot run in place: it compresses `cache` into `spare` and the two structs then swap
+ * their buffers (k, v, deg, logdeg, cap), so that on return `cache` again describes the live cache and `spare` the
+ * other buffer; both need deg, the same L, H, D, dtype and a capacity of at least budget + interval.  t_new tokens
+ * are processed as t_new decoding steps.  cache->len (host field) is updated, cache->pending set to 0;
+ * *reclusterings (host, optional) receives the number of rounds run.  Workspace: ckv_workspace_bytes for a cache of
+ * this shape with len = budget + interval and n_rounds_max = 1.  CKV_ERR_NO_PROGRESS if a round merges nothing. */
+int ckv_compress_append_recluster(ckv_cache* cache, ckv_cache* spare, const void* k_new, const void* v_new, int32_t t_new,
+                                  const ckv_params* params, int32_t interval, void* workspace, size_t workspace_bytes,
+                                  void* cuda_stream, int64_t* reclusterings);
+
 /* The kernels wait on asynchronous copies with a bounded number of polls; a wait that gives up sets a
  * status word at the start of the workspace instead of hanging.  This call copies that word to
  * *status_host (host pointer) and synchronises the stream: 0 = every wait completed, nonzero = some

@@ -14,7 +14,8 @@ bf16, see `round_to_dtype`); everything here is fp64, except that a similarity i
 rounded to fp32 before it decides an argmax or a ranking, because the kernel takes
 those decisions in fp32 and both sides must decide in the same precision.
 
-Pins (tests/test_oracle_pins.py): brute-force matching on chunks of 4-8 tokens,
+Pins (tests/test_oracle_pins.py): brute-force matching on chunks of 4-8 tokens (also at
+every trigger of the fixed-budget decoding branch),
 ratio 0 is the identity, identical keys merge to their exact mean, degree and
 first-moment conservation, N = 1 reduces approximate attention to softmax
 attention, the q = 0 closed form, the replication identity, the duplicated-key
@@ -313,6 +314,30 @@ def compress_append(K, V, deg, pending, k_new, v_new, p: Params, storage: str | 
             deg = np.concatenate([deg[:, :, :w0], dw], axis=2)
             pending = 0
     return K, V, deg, pending
+
+
+def append_recluster(K, V, deg, k_new, v_new, p: Params, interval: int, storage: str | None = None):
+    """Algorithm 1, decoding branch, as printed: for every generated token K = [K, k], V = [V, v],
+    N = [N, 1], s = s + 1, and `if s >= B + g` one call of CentroidKV over the whole cache (sinks
+    and recent tokens kept, the degrees carried along) with the compression ratio of round 0.
+    With edges ranked per head the call merges min(floor(r * n_edges), s - B) edges, so the cache
+    returns to the budget B whenever the ratio allows it (the paper is silent on how a single call
+    lands on B; this is the reading taken for the pre-filling loop as well).
+    Returns (K, V, deg, number of re-clusterings)."""
+    L, H, _, d = K.shape
+    if p.budget <= 0:
+        raise ValueError("the fixed-budget trigger needs a budget B")
+    calls = 0
+    for t in range(k_new.shape[2]):
+        K = np.concatenate([K, k_new[:, :, t:t + 1]], axis=2)
+        V = np.concatenate([V, v_new[:, :, t:t + 1]], axis=2)
+        deg = np.concatenate([deg, np.ones((L, H, 1), dtype=deg.dtype)], axis=2)
+        if K.shape[2] >= p.budget + interval:
+            K, V, deg, _, log = csm_round(K, V, deg, p, ratio_for_round(p, 0), storage)
+            if log.s_out == log.s_in:
+                raise RuntimeError("no progress: the round merges nothing although the cache exceeds its budget")
+            calls += 1
+    return K, V, deg, calls
 
 
 # --------------------------------------------------------------------------- Eq. 1 and Eq. 3: attention

@@ -20,7 +20,7 @@ OK = 0
 
 EXPORTS = ["ckv_compress_plan", "ckv_workspace_bytes", "ckv_compress_prefill", "ckv_compress_append",
            "ckv_decode_workspace_bytes", "ckv_decode_attn", "ckv_status_string", "ckv_workspace_status",
-           "ckv_decode_attn_static"]
+           "ckv_decode_attn_static", "ckv_compress_append_recluster"]
 
 
 class CkvCache(C.Structure):
@@ -57,6 +57,10 @@ def _load():
     lib.ckv_compress_append.restype = C.c_int
     lib.ckv_compress_append.argtypes = [C.POINTER(CkvCache), C.c_void_p, C.c_void_p, C.c_int32, C.POINTER(CkvParams),
                                         C.c_void_p, C.c_size_t, C.c_void_p]
+    lib.ckv_compress_append_recluster.restype = C.c_int
+    lib.ckv_compress_append_recluster.argtypes = [C.POINTER(CkvCache), C.POINTER(CkvCache), C.c_void_p, C.c_void_p, C.c_int32,
+                                                  C.POINTER(CkvParams), C.c_int32, C.c_void_p, C.c_size_t, C.c_void_p,
+                                                  C.POINTER(C.c_int64)]
     lib.ckv_workspace_status.restype = C.c_int
     lib.ckv_workspace_status.argtypes = [C.c_void_p, C.c_void_p, C.POINTER(C.c_int32)]
     lib.ckv_decode_workspace_bytes.restype = C.c_size_t
@@ -173,6 +177,26 @@ def compress_append(cache: Cache, k_new: torch.Tensor, v_new: torch.Tensor, para
     _check(lib.ckv_compress_append(C.byref(cc), k_new.data_ptr(), v_new.data_ptr(), k_new.shape[2], C.byref(params.c()),
                                    workspace.data_ptr(), workspace.numel() * workspace.element_size(), _stream_ptr()))
     cache.len, cache.pending = cc.len, cc.pending
+
+
+def compress_append_recluster(cache: Cache, spare: Cache, k_new: torch.Tensor, v_new: torch.Tensor, params: Params,
+                              interval: int, workspace: torch.Tensor) -> int:
+    """ckv_compress_append_recluster on the current stream: append, and one clustering round over the whole cache
+    whenever it reaches budget + interval tokens.  The two Cache objects trade tensors like the C structs trade
+    buffers, so `cache` always holds the live cache.  Returns the number of re-clusterings."""
+    assert k_new.is_contiguous() and v_new.is_contiguous() and k_new.shape == v_new.shape
+    cc, cs, calls = cache.c(), spare.c(), C.c_int64()
+    live_before = cc.k
+    _check(lib.ckv_compress_append_recluster(C.byref(cc), C.byref(cs), k_new.data_ptr(), v_new.data_ptr(), k_new.shape[2],
+                                             C.byref(params.c()), interval, workspace.data_ptr(),
+                                             workspace.numel() * workspace.element_size(), _stream_ptr(), C.byref(calls)))
+    if cc.k != live_before:   # an odd number of rounds ran: the tensors trade places
+        cache.k, spare.k = spare.k, cache.k
+        cache.v, spare.v = spare.v, cache.v
+        cache.deg, spare.deg = spare.deg, cache.deg
+        cache.logdeg, spare.logdeg = spare.logdeg, cache.logdeg
+    cache.len, cache.pending = cc.len, cc.pending
+    return calls.value
 
 
 def workspace_status(workspace: torch.Tensor) -> int:

@@ -1,6 +1,7 @@
 // Host side of the C ABI: argument checks, the round schedule of Algorithm 1 / Eq. 4, workspace
 // layout, and the launch sequences.  No device memory is allocated here.
 #include <cmath>
+#include <utility>
 #include <cstring>
 #include <vector>
 
@@ -413,6 +414,88 @@ int ckv_compress_append(ckv_cache* cache, const void* k_new, const void* v_new, 
       cache->len = w0 + win_out;
     }
     if (cache->pending == c) cache->pending = 0;
+  }
+  return CKV_OK;
+}
+
+int ckv_compress_append_recluster(ckv_cache* cache, ckv_cache* spare, const void* k_new, const void* v_new, int32_t t_new,
+                                  const ckv_params* params, int32_t interval, void* workspace, size_t workspace_bytes,
+                                  void* cuda_stream, int64_t* reclusterings) {
+  int st;
+  if ((st = check_params(params)) != CKV_OK) return st;
+  if ((st = check_cache_shape(cache)) != CKV_OK) return st;
+  if ((st = check_cache_shape(spare, false)) != CKV_OK) return st;
+  if (params->budget <= 0 || interval <= 0) return CKV_ERR_INVALID_ARG;
+  if (t_new < 0 || (t_new > 0 && (!k_new || !v_new))) return CKV_ERR_INVALID_ARG;
+  if (cache->L != spare->L || cache->H != spare->H || cache->D != spare->D || cache->dtype != spare->dtype) return CKV_ERR_INVALID_ARG;
+  if (!cache->k || !cache->v || !cache->deg || !spare->k || !spare->v || !spare->deg) return CKV_ERR_INVALID_ARG;
+  if (!aligned16(cache->k) || !aligned16(cache->v) || !aligned16(spare->k) || !aligned16(spare->v) || !aligned16(k_new) ||
+      !aligned16(v_new))
+    return CKV_ERR_ALIGNMENT;
+  const int64_t LH = (int64_t)cache->L * cache->H;
+  const int D = cache->D, es = esize_of(cache->dtype);
+  const int64_t trigger = params->budget + (int64_t)interval;
+  if (cache->cap < trigger || spare->cap < trigger) return CKV_ERR_CAPACITY;
+  const size_t a_bytes = (size_t)LH * cache->cap * D * es, b_bytes = (size_t)LH * spare->cap * D * es;
+  if (overlaps(cache->k, a_bytes, spare->k, b_bytes) || overlaps(cache->v, a_bytes, spare->v, b_bytes) ||
+      overlaps(cache->k, a_bytes, spare->v, b_bytes) || overlaps(cache->v, a_bytes, spare->k, b_bytes))
+    return CKV_ERR_INVALID_ARG;
+  ckv_params one = *params;  // Algorithm 1 calls CentroidKV once per trigger
+  one.n_rounds_max = 1;
+  cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
+  unsigned char* ws = static_cast<unsigned char*>(workspace);
+
+  // The lengths are a function of shapes only: walk the steps on the host first, so that an unreachable budget or
+  // a short workspace is reported before anything is enqueued; then walk them again and launch.
+  for (int pass = 0; pass < 2; ++pass) {
+    const bool dry = pass == 0;
+    ckv_cache live = *cache, other = *spare;
+    int64_t calls = 0;
+    // the status word is defined after every call, also one that only appends
+    if (!dry && workspace && workspace_bytes >= 256 && cudaMemsetAsync(workspace, 0, 256, stream) != cudaSuccess) return CKV_ERR_CUDA;
+    for (int32_t done = 0; done < t_new || live.len >= trigger;) {
+      if (live.len >= trigger) {
+        // `if s >= B + g`: one round over the whole cache into the other buffer, then the buffers trade places
+        std::vector<RoundPlan> plan;
+        if ((st = plan_rounds(live.len, one, plan)) != CKV_OK) return st;
+        if (plan.empty() || plan.back().s_out >= live.len) return CKV_ERR_NO_PROGRESS;
+        Workspace w = layout_workspace(LH, D, es, one.chunk, plan, false);
+        if (dry) {
+          if (!workspace || workspace_bytes < w.total || !aligned16(workspace)) return CKV_ERR_WORKSPACE;
+        } else {
+          const Buf src{live.k, live.v, live.deg, live.logdeg, live.cap};
+          const Buf dst{other.k, other.v, other.deg, other.logdeg, other.cap};
+          if ((st = run_plan(plan, src, dst, live.len, (int)LH, D, live.dtype, one.chunk, nullptr, w, ws, stream)) != CKV_OK) return st;
+        }
+        std::swap(live.k, other.k);
+        std::swap(live.v, other.v);
+        std::swap(live.deg, other.deg);
+        std::swap(live.logdeg, other.logdeg);
+        std::swap(live.cap, other.cap);
+        live.len = plan.back().s_out;
+        ++calls;
+        continue;
+      }
+      const int32_t take = (int32_t)std::min<int64_t>(t_new - done, trigger - live.len);
+      if (!dry) {
+        CopyArgs cp{};  // K = [K, k], V = [V, v], N = [N, 1]
+        cp.k_src = k_new; cp.v_src = v_new; cp.deg_src = nullptr;
+        cp.k_dst = live.k; cp.v_dst = live.v; cp.deg_dst = live.deg; cp.logdeg_dst = live.logdeg;
+        cp.src_cap = t_new; cp.dst_cap = live.cap; cp.src_off = done; cp.dst_off = live.len; cp.count = take;
+        cp.LH = (int)LH;
+        if (launch_copy(cp, live.dtype, D, stream) != cudaSuccess) return CKV_ERR_CUDA;
+      }
+      live.len += take;
+      done += take;
+    }
+    if (!dry) {
+      live.pending = 0;
+      other.len = 0;
+      other.pending = 0;
+      *cache = live;
+      *spare = other;
+      if (reclusterings) *reclusterings = calls;
+    }
   }
   return CKV_OK;
 }

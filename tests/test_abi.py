@@ -105,3 +105,26 @@ def test_argument_checks_happen_before_any_launch(b):
     assert b.lib.ckv_decode_attn(0x1000, 1, 1, 4, 128, b.BF16, 0x1000, 0x2000, 0.1, 10, None, 0, None) == 4
     assert b.lib.ckv_workspace_bytes(C.byref(src), C.byref(p)) == 0
     assert b.lib.ckv_decode_workspace_bytes(32, 8, 4, 128, 8448) >= 32 * 32 * 3 * 132 * 4
+
+
+def test_append_recluster_argument_checks_need_no_gpu(b):
+    """Everything ckv_compress_append_recluster can refuse is refused on the host before a launch (dummy pointers)."""
+    L, H, D, cap = 1, 2, 128, 400
+
+    def cache(base, length, cap=cap):
+        return b.CkvCache(base, base + 0x1000000, base + 0x2000000, None, L, H, D, b.BF16, cap, length, 0)
+
+    def call(p, live, spare, interval, t_new=4, ws_bytes=1 << 30):
+        calls = C.c_int64(-1)
+        return b.lib.ckv_compress_append_recluster(C.byref(live), C.byref(spare), 0x9000000, 0xA000000, t_new, C.byref(p.c()), interval,
+                                                   0xB000000, ws_bytes, None, C.byref(calls))
+
+    ok = b.Params(chunk=64, n_sink=4, n_recent=8, n_rounds_max=1, r_init=1.0, r_decay=0.0, r_min=1.0, budget=300)
+    assert call(b.Params(chunk=64, budget=0), cache(0x10000000, 300), cache(0x20000000, 0), 16) == 1      # no budget
+    assert call(ok, cache(0x10000000, 300), cache(0x20000000, 0), 0) == 1                                    # no interval
+    assert call(ok, cache(0x10000000, 300), cache(0x20000000, 0, cap=310), 16) == 3                          # spare too small
+    assert call(ok, cache(0x10000000, 300), cache(0x10000000, 0), 16) == 1                                   # same buffer
+    nothing = b.Params(chunk=64, n_sink=4, n_recent=8, n_rounds_max=1, r_init=0.0, r_decay=0.0, r_min=0.0, budget=300)
+    live = cache(0x10000000, 315)
+    assert call(nothing, live, cache(0x20000000, 0), 16) == 5 and live.len == 315                            # merges nothing
+    assert call(ok, cache(0x10000000, 315), cache(0x20000000, 0), 16, ws_bytes=64) == 4                       # workspace too small

@@ -206,6 +206,39 @@ def test_p4_append_keeps_degree_sum_and_triggers_per_chunk():
     np.testing.assert_allclose((da[..., None] * Va).sum(axis=2), V.sum(axis=2) + vn.sum(axis=2), rtol=1e-10)
 
 
+@pytest.mark.parametrize("r,g", [(1.0, 3), (0.5, 4), (0.3, 2)])
+def test_fixed_budget_trigger_replayed_with_brute_force_rounds(r, g):
+    """Algorithm 1's decoding branch: the cache is re-clustered whenever it reaches B + g tokens.  Replay: plain
+    concatenation token by token and, at each trigger, the brute-force round on the whole cache with
+    M = min(floor(r * n_edges), s - B) merges."""
+    rng = np.random.default_rng(11)
+    s0, d, c, B, sink, recent = 14, 4, 6, 14, 2, 3
+    K, V = rand_cache(rng, 1, 1, s0, d, ar=0.7)
+    deg = np.ones((1, 1, s0), dtype=np.int64)
+    kn, vn = rand_cache(rng, 1, 1, 11, d, ar=0.7)
+    p = O.Params(chunk=c, n_sink=sink, n_recent=recent, r_init=r, r_decay=0.1, r_min=0.1, budget=B, select=O.SELECT_GLOBAL)
+    Ko, Vo, do, calls = O.append_recluster(K, V, deg, kn, vn, p, g)
+    Kb, Vb, db, n_calls = K[0, 0], V[0, 0], deg[0, 0], 0
+    for t in range(kn.shape[2]):
+        Kb = np.concatenate([Kb, kn[0, 0, t:t + 1]])
+        Vb = np.concatenate([Vb, vn[0, 0, t:t + 1]])
+        db = np.concatenate([db, [1]])
+        if len(Kb) >= B + g:
+            s = len(Kb)
+            mid = s - sink - recent
+            n_edges = (mid // c) * (c // 2) + ((mid % c + 1) // 2 if mid % c >= 2 else 0)
+            M = min(int(math.floor(r * n_edges + 1e-9)), s - B)
+            Kb, Vb, db, ne = brute_round(Kb.tolist(), Vb.tolist(), db.tolist(), sink, recent, c, M)
+            assert ne == n_edges and len(Kb) == s - M
+            n_calls += 1
+    assert calls == n_calls >= 2
+    np.testing.assert_allclose(Ko[0, 0], Kb, rtol=1e-12, atol=1e-12)
+    np.testing.assert_allclose(Vo[0, 0], Vb, rtol=1e-12, atol=1e-12)
+    np.testing.assert_array_equal(do[0, 0], db)
+    assert do.sum() == s0 + kn.shape[2]                            # every token ever written is accounted for (Sec. 3)
+    np.testing.assert_array_equal(Ko[0, 0, :sink], K[0, 0, :sink])  # sinks are never merged
+
+
 def test_p12_at_most_half_and_borders_untouched():
     rng = np.random.default_rng(5)
     s, n1, n2 = 101, 6, 9
