@@ -272,6 +272,7 @@ def run_gpu(args):
 
     if rank == 0 and not args.skip_decode_cfg4:
         extra["decode_cfg4"] = bench_decode_cfg4(b, synth, dev, peaks["hbm_gbs"])
+        extra["decode_cfg4_paged"] = bench_decode_paged(b, synth, dev, peaks["hbm_gbs"])
     if rank == 0 and not args.skip_variants:
         extra["compress_variants"] = bench_compress_variants(b, synth, dev, K, V, peaks["hbm_gbs"], args.layers == 0)
         extra["recluster"] = bench_recluster(b, synth, dev, K, V)
@@ -438,6 +439,40 @@ def bench_recluster(b, synth, dev, K, V):
     ms = statistics.mean(times)
     return {"budget": B, "interval": g, "ms_per_trigger_all_layers": ms, "us_per_decode_step_amortised": 1e3 * ms / g,
             "status": b.workspace_status(ws)}
+
+
+def bench_decode_paged(b, synth, dev, peak_gbs):
+    """The decode_b32 shape (batch 32, 8192 centroids) in a paged cache: 64-token pages scattered over one pool."""
+    import torch
+    cfg = synth.CONFIGS["decode_b32"]
+    Bz, H, G, D, slots, P = cfg["batch"], cfg["H"], cfg["G"], cfg["d"], cfg["slots"], 64
+    per_seq = slots // P
+    pool = Bz * per_seq
+    g = torch.Generator(dev).manual_seed(17)
+    kp = torch.randn((pool, H, P, D), device=dev, generator=g).to(torch.bfloat16)
+    vp = torch.randn((pool, H, P, D), device=dev, generator=g).to(torch.bfloat16)
+    lp = torch.rand((pool, H, P), device=dev, generator=g) * 2.0
+    perm = torch.randperm(pool, generator=torch.Generator().manual_seed(5)).to(torch.int32).to(dev)
+    tables = [perm[i * per_seq:(i + 1) * per_seq].contiguous() for i in range(Bz)]
+    views = b.paged_views(tables, [slots] * Bz, dev)
+    q = synth.queries(Bz, H * G, D, seed=3, dtype="bf16", device=dev)
+    out = torch.empty_like(q)
+    ws = torch.empty(b.decode_workspace_bytes(Bz, H, G, D, slots), dtype=torch.uint8, device=dev)
+    scale = 1.0 / math.sqrt(D)
+    for _ in range(5):
+        b.decode_attn_paged(views, kp, vp, lp, H, G, q, out, scale, slots, ws)
+    torch.cuda.synchronize()
+    iters = 50
+    t0, t1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    t0.record()
+    for _ in range(iters):
+        b.decode_attn_paged(views, kp, vp, lp, H, G, q, out, scale, slots, ws)
+    t1.record()
+    torch.cuda.synchronize()
+    us = 1e3 * t0.elapsed_time(t1) / iters
+    nbytes = decode_bytes(Bz * H * slots, D, 2)
+    return {"slots": slots, "page_tokens": P, "us_per_layer_step": us, "gbs": nbytes / (us * 1e-6) / 1e9,
+            "frac_of_peak": nbytes / (us * 1e-6) / 1e9 / peak_gbs}
 
 
 def bench_decode_cfg4(b, synth, dev, peak_gbs):

@@ -147,6 +147,34 @@ int ckv_decode_attn(const ckv_layer_view* views_dev, int32_t Bz, int32_t H, int3
                     const void* q, void* out, float scale, int64_t max_len, void* workspace,
                     size_t workspace_bytes, void* cuda_stream);
 
+/* ---- Paged cache (the block layout of serving engines; the paper's Appendix on its vLLM integration names the flow
+ * read pages -> compress -> write back).  One layer's pool: k_pages, v_pages [n_pages, H, page_tokens, D],
+ * deg_pages int32 and logdeg_pages fp32 [n_pages, H, page_tokens]; page_tokens a power of two >= 32.  A sequence owns
+ * the pages its block table lists: logical token t sits in page block_table[t / page_tokens] at offset t % page_tokens.
+ * Which pages are free is the caller's bookkeeping: after a compression to out_len tokens a sequence needs
+ * ceil(out_len / page_tokens) pages and can return the rest. */
+typedef struct ckv_paged_view {
+  const int32_t* block_table; /* device, at least ceil(len / page_tokens) entries */
+  int64_t len;
+} ckv_paged_view;
+
+/* Eq. 3 over a paged cache: as ckv_decode_attn, with views_dev a device array [Bz] of ckv_paged_view.  bf16 only in
+ * this version (CKV_ERR_UNSUPPORTED otherwise); logdeg_pages NULL = all degrees one.  Workspace as ckv_decode_attn. */
+int ckv_decode_attn_paged(const ckv_paged_view* views_dev, const void* k_pages, const void* v_pages, const float* logdeg_pages,
+                          int32_t page_tokens, int32_t Bz, int32_t H, int32_t G, int32_t D, int32_t dtype, const void* q,
+                          void* out, float scale, int64_t max_len, void* workspace, size_t workspace_bytes, void* cuda_stream);
+
+/* Copies one sequence's first `len` tokens of one layer between its pages and a contiguous slab k, v [H, cap, D],
+ * deg [H, cap] (logdeg [H, cap] optional): gather = pages -> slab (to run ckv_compress_* on it), scatter = slab -> pages
+ * (degrees and their logarithms are written to the pages as well; deg NULL on scatter = all ones).  deg_pages may be
+ * NULL on gather (the slab then gets ones).  block_table: device, ceil(len / page_tokens) entries. */
+int ckv_pages_gather(const int32_t* block_table, int64_t len, const void* k_pages, const void* v_pages, const int32_t* deg_pages,
+                     int32_t page_tokens, int32_t H, int32_t D, int32_t dtype, void* k, void* v, int32_t* deg, float* logdeg,
+                     int64_t cap, void* cuda_stream);
+int ckv_pages_scatter(const int32_t* block_table, int64_t len, const void* k, const void* v, const int32_t* deg, int64_t cap,
+                      int32_t page_tokens, int32_t H, int32_t D, int32_t dtype, void* k_pages, void* v_pages, int32_t* deg_pages,
+                      float* logdeg_pages, void* cuda_stream);
+
 /* ckv_decode_attn for callers that cannot hand over a workspace because they cannot allocate device
  * memory at the point of the call: code running inside a serving engine's steady-state loop whose memory
  * pool is frozen after start-up, a plug-in that is given only its input and output tensors, or a host

@@ -363,3 +363,21 @@ def app_attn(q, K, V, deg, scale):
 def attn(q, K, V, scale):
     """Eq. 1: exact softmax attention (Eq. 3 with every degree equal to one)."""
     return app_attn(q, K, V, None, scale)
+
+
+# --------------------------------------------------------------------------- paged cache (block layout of serving engines)
+
+def gather_pages(pages, block_table, length: int):
+    """A paged cache stores logical token t of a sequence in page block_table[t // P] at offset t % P.
+    pages: [n_pages, H, P, ...]; returns the sequence's first `length` tokens as [H, length, ...]."""
+    P = pages.shape[2]
+    t = np.arange(length)
+    page = np.asarray(block_table)[t // P]
+    return np.moveaxis(pages[page, :, t % P], 0, 1)
+
+
+def app_attn_paged(q, k_pages, v_pages, deg_pages, block_table, length: int, scale):
+    """Eq. 3 over a paged cache: by definition the attention over the gathered sequence."""
+    deg = gather_pages(deg_pages, block_table, length) if deg_pages is not None else None
+    return app_attn(q, gather_pages(k_pages, block_table, length), gather_pages(v_pages, block_table, length), deg, scale)
+

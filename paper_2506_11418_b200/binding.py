@@ -20,7 +20,8 @@ OK = 0
 
 EXPORTS = ["ckv_compress_plan", "ckv_workspace_bytes", "ckv_compress_prefill", "ckv_compress_append",
            "ckv_decode_workspace_bytes", "ckv_decode_attn", "ckv_status_string", "ckv_workspace_status",
-           "ckv_decode_attn_static", "ckv_compress_append_recluster"]
+           "ckv_decode_attn_static", "ckv_compress_append_recluster", "ckv_decode_attn_paged", "ckv_pages_gather",
+           "ckv_pages_scatter"]
 
 
 class CkvCache(C.Structure):
@@ -61,6 +62,16 @@ def _load():
     lib.ckv_compress_append_recluster.argtypes = [C.POINTER(CkvCache), C.POINTER(CkvCache), C.c_void_p, C.c_void_p, C.c_int32,
                                                   C.POINTER(CkvParams), C.c_int32, C.c_void_p, C.c_size_t, C.c_void_p,
                                                   C.POINTER(C.c_int64)]
+    lib.ckv_decode_attn_paged.restype = C.c_int
+    lib.ckv_decode_attn_paged.argtypes = [C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_int32, C.c_int32, C.c_int32, C.c_int32,
+                                          C.c_int32, C.c_int32, C.c_void_p, C.c_void_p, C.c_float, C.c_int64, C.c_void_p, C.c_size_t,
+                                          C.c_void_p]
+    lib.ckv_pages_gather.restype = C.c_int
+    lib.ckv_pages_gather.argtypes = [C.c_void_p, C.c_int64, C.c_void_p, C.c_void_p, C.c_void_p, C.c_int32, C.c_int32, C.c_int32,
+                                     C.c_int32, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_int64, C.c_void_p]
+    lib.ckv_pages_scatter.restype = C.c_int
+    lib.ckv_pages_scatter.argtypes = [C.c_void_p, C.c_int64, C.c_void_p, C.c_void_p, C.c_void_p, C.c_int64, C.c_int32, C.c_int32,
+                                      C.c_int32, C.c_int32, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p]
     lib.ckv_workspace_status.restype = C.c_int
     lib.ckv_workspace_status.argtypes = [C.c_void_p, C.c_void_p, C.POINTER(C.c_int32)]
     lib.ckv_decode_workspace_bytes.restype = C.c_size_t
@@ -238,3 +249,40 @@ def decode_attn_static(views: torch.Tensor, H: int, G: int, q: torch.Tensor, out
     assert HG == H * G and q.is_contiguous() and out.is_contiguous()
     _check(lib.ckv_decode_attn_static(views.data_ptr(), Bz, H, G, D, dtype_code(q.dtype), q.data_ptr(), out.data_ptr(),
                                       scale, max_len, _stream_ptr()))
+
+
+# ---- paged cache: one layer's pool k_pages, v_pages [n_pages, H, P, D], deg_pages int32 / logdeg_pages fp32 [n_pages, H, P]
+
+def _ptr(t):
+    return t.data_ptr() if t is not None else None
+
+
+def paged_views(block_tables, lens, device="cuda") -> torch.Tensor:
+    """Device array of ckv_paged_view (two int64 words each) from per-sequence block-table tensors on the GPU."""
+    return torch.tensor([[t.data_ptr(), n] for t, n in zip(block_tables, lens)], dtype=torch.int64).to(device)
+
+
+def decode_attn_paged(views: torch.Tensor, k_pages, v_pages, logdeg_pages, H: int, G: int, q, out, scale: float, max_len: int,
+                      workspace: torch.Tensor):
+    """ckv_decode_attn_paged on the current stream."""
+    Bz, HG, D = q.shape
+    assert HG == H * G and q.is_contiguous() and out.is_contiguous() and k_pages.is_contiguous() and v_pages.is_contiguous()
+    _check(lib.ckv_decode_attn_paged(views.data_ptr(), k_pages.data_ptr(), v_pages.data_ptr(), _ptr(logdeg_pages), k_pages.shape[2],
+                                     Bz, H, G, D, dtype_code(q.dtype), q.data_ptr(), out.data_ptr(), scale, max_len,
+                                     workspace.data_ptr(), workspace.numel() * workspace.element_size(), _stream_ptr()))
+
+
+def pages_gather(block_table, length, k_pages, v_pages, deg_pages, k, v, deg, logdeg=None):
+    """ckv_pages_gather: pages -> contiguous slab k, v [H, cap, D], deg [H, cap] of one layer."""
+    _, H, P, D = k_pages.shape
+    _check(lib.ckv_pages_gather(block_table.data_ptr(), length, k_pages.data_ptr(), v_pages.data_ptr(), _ptr(deg_pages), P, H, D,
+                                dtype_code(k_pages.dtype), k.data_ptr(), v.data_ptr(), _ptr(deg), _ptr(logdeg), k.shape[1], _stream_ptr()))
+
+
+def pages_scatter(block_table, length, k, v, deg, k_pages, v_pages, deg_pages, logdeg_pages):
+    """ckv_pages_scatter: contiguous slab -> pages (degrees and log-degrees included)."""
+    _, H, P, D = k_pages.shape
+    _check(lib.ckv_pages_scatter(block_table.data_ptr(), length, k.data_ptr(), v.data_ptr(), _ptr(deg), k.shape[1], P, H, D,
+                                 dtype_code(k_pages.dtype), k_pages.data_ptr(), v_pages.data_ptr(), _ptr(deg_pages),
+                                 _ptr(logdeg_pages), _stream_ptr()))
+

@@ -324,6 +324,10 @@ __device__ __forceinline__ void mma_bf16_16816(float (&d)[4], uint32_t a0, uint3
       : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1));
 }
 
+// PAGED: the cache lives in fixed-size pages, [n_pages, H, page_tokens, D], and a per-sequence block table maps
+// logical block i (tokens i * page_tokens ...) to its page; page_tokens is a multiple of the tile, so a tile never
+// straddles pages.  Each lane keeps one entry of the table (32 blocks per refill), handed out by shuffle.
+template <bool PAGED>
 __global__ void __launch_bounds__(kFWarps * 32, 1) decode_fast_kernel(const DecodeArgs a) {
   constexpr int D = 128;
   extern __shared__ __align__(128) unsigned char smem_raw[];
@@ -334,16 +338,30 @@ __global__ void __launch_bounds__(kFWarps * 32, 1) decode_fast_kernel(const Deco
   griddep_launch();  // the combine kernel may become resident; it waits for this grid before it reads
   if (split >= a.n_splits) return;
   const int h = blockIdx.y, b = blockIdx.z, G = a.G;
-  const ckv_layer_view view = reinterpret_cast<const ckv_layer_view*>(a.views)[b];
+  ckv_layer_view view{};
+  const int32_t* table = nullptr;
+  if (PAGED) {
+    const ckv_paged_view pv = reinterpret_cast<const ckv_paged_view*>(a.views)[b];
+    table = pv.block_table;
+    view.len = pv.len;
+  } else {
+    view = reinterpret_cast<const ckv_layer_view*>(a.views)[b];
+  }
   const int64_t len = view.len;
   // the sequence's own tiles are dealt evenly to the splits (a ragged batch stays balanced)
   const int64_t seq_tiles = (len + kFT - 1) / kFT;
   const int64_t t_begin = kFT * (seq_tiles * split / a.n_splits);
   const int64_t t_end = min(len, kFT * (seq_tiles * (split + 1) / a.n_splits));
   const int ntiles = (int)((t_end - t_begin + kFT - 1) / kFT);
-  const __nv_bfloat16* kbase = reinterpret_cast<const __nv_bfloat16*>(view.k) + (int64_t)h * view.cap * D;
-  const __nv_bfloat16* vbase = reinterpret_cast<const __nv_bfloat16*>(view.v) + (int64_t)h * view.cap * D;
-  const float* ldbase = view.logdeg ? view.logdeg + (int64_t)h * view.cap : nullptr;
+  const __nv_bfloat16* kbase = PAGED ? reinterpret_cast<const __nv_bfloat16*>(a.k_pages)
+                                     : reinterpret_cast<const __nv_bfloat16*>(view.k) + (int64_t)h * view.cap * D;
+  const __nv_bfloat16* vbase = PAGED ? reinterpret_cast<const __nv_bfloat16*>(a.v_pages)
+                                     : reinterpret_cast<const __nv_bfloat16*>(view.v) + (int64_t)h * view.cap * D;
+  const float* ldbase = PAGED ? a.logdeg_pages : (view.logdeg ? view.logdeg + (int64_t)h * view.cap : nullptr);
+  // paged: block table entries [blk0, blk0 + 32) of this sequence, one per lane
+  const int64_t n_blocks = PAGED ? (len + ((int64_t)1 << a.page_shift) - 1) >> a.page_shift : 0;
+  int64_t blk0 = PAGED ? t_begin >> a.page_shift : 0;
+  int my_page = (PAGED && ntiles > 0 && blk0 + lane < n_blocks) ? table[blk0 + lane] : 0;
   const uint32_t ring = (uint32_t)__cvta_generic_to_shared(smem_raw) + (uint32_t)warp * kFStages * kFStageBytes;
   const float* ring_ld = reinterpret_cast<const float*>(smem_raw + (size_t)warp * kFStages * kFStageBytes);
 
@@ -364,18 +382,29 @@ __global__ void __launch_bounds__(kFWarps * 32, 1) decode_fast_kernel(const Deco
     const int64_t t0 = t_begin + (int64_t)tile * kFT;
     const uint32_t st = ring + (uint32_t)(tile % kFStages) * kFStageBytes;
     const int c = lane & 15;
+    // row0: where the tile's first token sits in the K / V / log-degree arrays; rows of a tile are contiguous
+    int64_t row0 = t0;
+    if (PAGED) {
+      const int64_t blk = t0 >> a.page_shift;
+      if (blk >= blk0 + 32) {  // next 32 entries of the table (tiles are issued in order)
+        blk0 = blk;
+        my_page = blk0 + lane < n_blocks ? table[blk0 + lane] : 0;
+      }
+      const int page = __shfl_sync(0xffffffffu, my_page, (int)(blk - blk0));
+      row0 = (((int64_t)page * a.H + h) << a.page_shift) + (t0 & (((int64_t)1 << a.page_shift) - 1));
+    }
 #pragma unroll
     for (int i = 0; i < 16; ++i) {
       const int r = (lane >> 4) + 2 * i;
       const bool ok = t0 + r < t_end;
-      const int64_t row = ok ? t0 + r : t_begin;  // clamped address, zero-filled when out of range
+      const int64_t row = ok ? row0 + r : row0;  // clamped address, zero-filled when out of range
       const uint32_t off = (uint32_t)r * 256u + (uint32_t)((c ^ (r & 7)) << 4);
       cp_async16(st + off, kbase + row * D + c * 8, ok ? 16u : 0u);
       cp_async16(st + kFTileBytes + off, vbase + row * D + c * 8, ok ? 16u : 0u);
     }
     if (ldbase) {  // one log-degree per lane; 4-byte copies have no alignment demands on the slab
       const bool ok = t0 + lane < t_end;
-      cp_async4(st + 2 * kFTileBytes + lane * 4, ldbase + (ok ? t0 + lane : t_begin), ok ? 4u : 0u);
+      cp_async4(st + 2 * kFTileBytes + lane * 4, ldbase + (ok ? row0 + lane : row0), ok ? 4u : 0u);
     }
   };
 
@@ -488,11 +517,12 @@ __global__ void __launch_bounds__(kFWarps * 32, 1) decode_fast_kernel(const Deco
   }
 }
 
+template <bool PAGED>
 cudaError_t launch_decode_fast(const DecodeArgs& a, cudaStream_t st) {
-  cudaError_t e = cudaFuncSetAttribute(decode_fast_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kFSmemBytes);
+  cudaError_t e = cudaFuncSetAttribute(decode_fast_kernel<PAGED>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kFSmemBytes);
   if (e != cudaSuccess) return e;
   const dim3 grid((unsigned)((a.n_splits + kFWarps - 1) / kFWarps), (unsigned)a.H, (unsigned)a.Bz);
-  if ((e = launch_dependent(decode_fast_kernel, grid, dim3(kFWarps * 32), kFSmemBytes, st, a)) != cudaSuccess) return e;
+  if ((e = launch_dependent(decode_fast_kernel<PAGED>, grid, dim3(kFWarps * 32), kFSmemBytes, st, a)) != cudaSuccess) return e;
   return launch_dependent(decode_combine_kernel<__nv_bfloat16, 128>, dim3((unsigned)(a.Bz * a.H * a.G)), dim3(kCombThreads), 0,
                           st, a);
 }
@@ -548,9 +578,11 @@ size_t decode_partial_floats(int32_t Bz, int32_t H, int32_t G, int32_t D, int64_
 
 cudaError_t launch_decode(const DecodeArgs& a, int dtype, int D, cudaStream_t st) {
   if (D != 128) return cudaErrorInvalidValue;
-  if (dtype == 1) return launch_decode_fast(a, st);
+  if (dtype == 1) return launch_decode_fast<false>(a, st);
   return launch_decode_t<float>(a, st);
 }
+
+cudaError_t launch_decode_paged(const DecodeArgs& a, cudaStream_t st) { return launch_decode_fast<true>(a, st); }
 
 }  // namespace ckv
 

@@ -70,7 +70,7 @@ struct SelectArgs {
 };
 
 struct DecodeArgs {
-  const void* views;  // const ckv_layer_view*
+  const void* views;  // const ckv_layer_view*, or const ckv_paged_view* when the cache is paged
   const void* q;
   void* out;
   float* partial;     // [Bz, H*G, n_splits, D + 4]: out[D], max, sum, pad
@@ -78,6 +78,11 @@ struct DecodeArgs {
   int32_t n_splits;
   int64_t span;       // tokens per split
   float scale;
+  // paged cache (bf16 kernel only): pages of `page_tokens` tokens, [n_pages, H, page_tokens, D]
+  const void* k_pages;
+  const void* v_pages;
+  const float* logdeg_pages;  // [n_pages, H, page_tokens] or null
+  int32_t page_shift;         // log2(page_tokens), page_tokens >= 32
 };
 
 // Launch with programmatic stream serialization: the kernel may become resident while the kernel ahead of it
@@ -104,6 +109,7 @@ cudaError_t launch_select(const SelectArgs& a, cudaStream_t st);
 cudaError_t launch_compose_assign(int32_t* total, const int32_t* step, int64_t n_src, int64_t step_stride, int32_t LH,
                                   cudaStream_t st);
 cudaError_t launch_decode(const DecodeArgs& a, int dtype, int D, cudaStream_t st);
+cudaError_t launch_decode_paged(const DecodeArgs& a, cudaStream_t st);
 void decode_plan(int32_t Bz, int32_t H, int dtype, int64_t max_len, int64_t max_partial_floats, int32_t G, int32_t D,
                  int32_t* n_splits, int64_t* span);
 size_t decode_partial_floats(int32_t Bz, int32_t H, int32_t G, int32_t D, int64_t max_len);

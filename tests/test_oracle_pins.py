@@ -397,3 +397,27 @@ def test_p13_ar1_edges_join_neighbours():
     e = O.match_head(K[0, 0], 0, 0, 64)
     assert np.mean(np.abs(e.a_pos - e.b_pos) == 1) > 0.9
     assert 0.8 < float(np.mean(e.sim)) < 0.97   # E[cos] at distance 1 is about rho = 0.9
+
+
+def test_paged_attention_does_not_depend_on_where_the_pages_are():
+    """A paged cache is the same sequence whatever pages hold it: with the blocks scattered over a larger pool in a
+    random order the result equals Eq. 3 on the contiguous cache, which the pins above fix."""
+    rng = np.random.default_rng(21)
+    H, G, d, P, n = 2, 2, 8, 4, 19
+    K, V = rng.standard_normal((H, n, d)), rng.standard_normal((H, n, d))
+    deg = rng.integers(1, 5, (H, n))
+    q = rng.standard_normal((H * G, d))
+    n_blocks, pool = (n + P - 1) // P, 11
+    table = rng.permutation(pool)[:n_blocks]
+    kp, vp = rng.standard_normal((pool, H, P, d)), rng.standard_normal((pool, H, P, d))   # junk everywhere else
+    dp = rng.integers(1, 9, (pool, H, P))
+    for t in range(n):
+        kp[table[t // P], :, t % P], vp[table[t // P], :, t % P], dp[table[t // P], :, t % P] = K[:, t], V[:, t], deg[:, t]
+    np.testing.assert_array_equal(O.gather_pages(kp, table, n), K)
+    np.testing.assert_allclose(O.app_attn_paged(q, kp, vp, dp, table, n, 0.3), O.app_attn(q, K, V, deg, 0.3), rtol=1e-13)
+    np.testing.assert_allclose(O.app_attn_paged(q, kp, vp, None, table, n, 0.3), textbook_attention_heads(q, K, V, 0.3, G), rtol=1e-12)
+
+
+def textbook_attention_heads(q, K, V, scale, G):
+    return np.stack([softmax(K[j // G] @ q[j] * scale) @ V[j // G] for j in range(q.shape[0])])
+
