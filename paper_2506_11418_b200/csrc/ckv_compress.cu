@@ -276,7 +276,9 @@ __device__ __forceinline__ uint32_t sim_key(float s) {
 }
 
 constexpr int kSelThreads = 1024;
+constexpr int kSelRun = 64;  // edges per thread and sweep of the position-order pass (one bit each in a 64-bit mask)
 
+// exclusive prefix of x over the block, and the block total
 __device__ __forceinline__ int block_exscan(int x, int* total, int* warp_tot) {
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
   int inc = x;
@@ -287,52 +289,73 @@ __device__ __forceinline__ int block_exscan(int x, int* total, int* warp_tot) {
   }
   if (lane == 31) warp_tot[warp] = inc;
   __syncthreads();
-  int before = 0, tot = 0;
-  for (int w = 0; w < kSelThreads / 32; ++w) {
-    const int t = warp_tot[w];
-    before += (w < warp) ? t : 0;
-    tot += t;
+  const int wt = warp_tot[lane];  // kSelThreads / 32 == 32 warps: one total per lane
+  int winc = wt;
+#pragma unroll
+  for (int o = 1; o < 32; o <<= 1) {
+    const int y = __shfl_up_sync(0xffffffffu, winc, o);
+    if (lane >= o) winc += y;
   }
+  const int before = __shfl_sync(0xffffffffu, winc - wt, warp);
+  *total = __shfl_sync(0xffffffffu, winc, 31);
   __syncthreads();
-  *total = tot;
   return before + inc - x;
 }
 
 __global__ void __launch_bounds__(kSelThreads) select_kernel(const SelectArgs a) {
+  static_assert(kSelThreads == 1024, "one warp total per lane in block_exscan");
   __shared__ uint32_t hist[256];
   __shared__ uint32_t s_prefix, s_rem;
   __shared__ int warp_tot[kSelThreads / 32];
-  const int tid = threadIdx.x;
+  const int tid = threadIdx.x, lane = tid & 31;
   const int lh = blockIdx.x;
   const int64_t n = a.edge_stride;
   const float* sim = a.edge_sim + (int64_t)lh * n;
   const int hc = a.chunk >> 1;
   const bool none = a.M <= 0;
 
+  // ---- the key of the M-th best edge: 4 x 8-bit radix select from the top byte down
   uint32_t prefix = 0, mask = 0, rem = (uint32_t)a.M;
   if (!none) {
+    const int64_t n_up = (n + kSelThreads - 1) / kSelThreads * kSelThreads;  // whole warps stay in the loop
     for (int pass = 3; pass >= 0; --pass) {
       const int shift = pass * 8;
       for (int i = tid; i < 256; i += kSelThreads) hist[i] = 0;
       __syncthreads();
-      for (int64_t i = tid; i < n; i += kSelThreads) {
-        const uint32_t key = sim_key(sim[i]);
-        if ((key & mask) == prefix) atomicAdd(&hist[(key >> shift) & 255u], 1u);
+      for (int64_t i = tid; i < n_up; i += kSelThreads) {
+        const uint32_t key = i < n ? sim_key(sim[i]) : 0u;
+        const bool in = i < n && (key & mask) == prefix;
+        // similarities cluster, so most lanes hit the same bin: one atomic per distinct bin of the warp
+        const uint32_t bin = in ? ((key >> shift) & 255u) : 256u;
+        const unsigned peers = __match_any_sync(0xffffffffu, bin);
+        if (in && lane == __ffs(peers) - 1) atomicAdd(&hist[bin], (uint32_t)__popc(peers));
       }
       __syncthreads();
-      if (tid == 0) {
-        uint32_t cum = 0, r = rem, p = prefix;
-        for (int bin = 255; bin >= 0; --bin) {
-          const uint32_t h = hist[bin];
-          if (cum + h >= r) {
-            p |= (uint32_t)bin << shift;
-            r -= cum;
-            break;
-          }
-          cum += h;
+      if (tid < 32) {
+        // lane L owns bins 255 - 8 L ... 248 - 8 L (descending); find the bin where the count from the top reaches rem
+        uint32_t own = 0;
+#pragma unroll
+        for (int j = 0; j < 8; ++j) own += hist[255 - 8 * lane - j];
+        uint32_t inc = own;
+#pragma unroll
+        for (int o = 1; o < 32; o <<= 1) {
+          const uint32_t y = __shfl_up_sync(0xffffffffu, inc, o);
+          if (lane >= o) inc += y;
         }
-        s_prefix = p;
-        s_rem = r;
+        const uint32_t above = inc - own;  // edges in bins above this lane's
+        if (above < rem && rem <= inc) {   // exactly one lane
+          uint32_t cum = above;
+          for (int j = 0; j < 8; ++j) {
+            const int bin = 255 - 8 * lane - j;
+            const uint32_t h = hist[bin];
+            if (cum + h >= rem) {
+              s_prefix = prefix | ((uint32_t)bin << shift);
+              s_rem = rem - cum;
+              break;
+            }
+            cum += h;
+          }
+        }
       }
       __syncthreads();
       prefix = s_prefix;
@@ -343,23 +366,34 @@ __global__ void __launch_bounds__(kSelThreads) select_kernel(const SelectArgs a)
   const uint32_t T = prefix;   // key of the M-th best edge
   const int quota = (int)rem;  // how many edges equal to T are merged: the earliest ones
 
-  int sel_run = 0, eq_run = 0;
-  for (int64_t base = 0; base < n; base += kSelThreads) {
-    const int64_t i = base + tid;
-    const bool valid = i < n;
-    const uint32_t key = valid ? sim_key(sim[i]) : 0u;
-    const int eq = (valid && !none && key == T) ? 1 : 0;
-    const int gt = (valid && !none && key > T) ? 1 : 0;
+  // ---- one pass in position order: every thread owns a run of consecutive edges
+  int sel_run = 0, eq_run = 0;  // totals of the sweeps before this one
+  for (int64_t base = 0; base < n; base += (int64_t)kSelThreads * kSelRun) {
+    const int64_t first = base + (int64_t)tid * kSelRun;
+    const int len = (int)max((int64_t)0, min((int64_t)kSelRun, n - first));
+    unsigned long long gt_bits = 0ull, eq_bits = 0ull;
+    for (int j = 0; j < len; ++j) {
+      const uint32_t key = sim_key(sim[first + j]);
+      if (!none && key > T) gt_bits |= 1ull << j;
+      if (!none && key == T) eq_bits |= 1ull << j;
+    }
     int eq_tot, s_tot;
-    const int eq_ex = block_exscan(eq, &eq_tot, warp_tot);
-    const int s = (gt || (eq && eq_run + eq_ex < quota)) ? 1 : 0;
-    const int s_ex = block_exscan(s, &s_tot, warp_tot);
-    if (valid) {
-      a.sel[(int64_t)lh * n + i] = (uint8_t)s;
+    const int eq_ex = eq_run + block_exscan(__popcll(eq_bits), &eq_tot, warp_tot);
+    // the earliest `quota` edges equal to the threshold are merged
+    const int take = max(0, min(__popcll(eq_bits), quota - eq_ex));
+    unsigned long long sel_bits = gt_bits;
+    for (unsigned long long e = eq_bits, k = 0; e && (int)k < take; e &= e - 1, ++k) sel_bits |= e & (~e + 1ull);
+    const int s_ex = sel_run + block_exscan(__popcll(sel_bits), &s_tot, warp_tot);
+    int before = s_ex;
+    for (int j = 0; j < len; ++j) {
+      const int64_t i = first + j;
+      const int sbit = (int)((sel_bits >> j) & 1ull);
+      a.sel[(int64_t)lh * n + i] = (uint8_t)sbit;
       if (i % hc == 0) {
         const int64_t ch = i / hc;
-        a.chunk_out_off[(int64_t)lh * a.n_chunks + ch] = (int32_t)(a.lo + ch * a.chunk - (sel_run + s_ex));
+        a.chunk_out_off[(int64_t)lh * a.n_chunks + ch] = (int32_t)(a.lo + ch * a.chunk - before);
       }
+      before += sbit;
     }
     eq_run += eq_tot;
     sel_run += s_tot;
