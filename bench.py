@@ -273,6 +273,8 @@ def run_gpu(args):
     if rank == 0 and not args.skip_decode_cfg4:
         extra["decode_cfg4"] = bench_decode_cfg4(b, synth, dev, peaks["hbm_gbs"])
         extra["decode_cfg4_paged"] = bench_decode_paged(b, synth, dev, peaks["hbm_gbs"])
+    if rank == 0 and not args.skip_serving and args.layers == 0:
+        extra["serving_mix"] = bench_serving_mix(b, synth, dev, peaks["hbm_gbs"])
     if rank == 0 and not args.skip_variants:
         extra["compress_variants"] = bench_compress_variants(b, synth, dev, K, V, peaks["hbm_gbs"], args.layers == 0)
         extra["recluster"] = bench_recluster(b, synth, dev, K, V)
@@ -405,6 +407,84 @@ def bench_compress_variants(b, synth, dev, K, V, peak_gbs, with_128k):
     return res
 
 
+def bench_serving_mix(b, synth, dev, peak_gbs, steps=128):
+    """Workload serving_mix: batch 64, context lengths uniform on [4096, 65536], 32 layers x 8 KV heads, caches already
+    compressed to 25 % (their content does not matter for timing: random values, degrees 4).  Lock-step decoding: every
+    step appends one token to every sequence (ckv_compress_append, which clusters each completed chunk of 64 appended
+    tokens 64 -> 32 -> 16) and runs ckv_decode_attn for all 32 layers over the ragged batch.  The uncompressed comparison
+    keeps the full contexts of the same batch on 8 layers (32 would not fit) and is scaled to 32."""
+    import torch
+    cfg = synth.CONFIGS["serving_mix"]
+    Bz, L, H, G, D, c = cfg["batch"], cfg["L"], cfg["H"], cfg["G"], cfg["d"], cfg["chunk"]
+    ctx = synth.context_lengths(Bz, cfg["ctx"][0], cfg["ctx"][1], seed=cfg["seed"])
+    p = b.Params(chunk=c, n_sink=0, n_recent=0, n_rounds_max=2, r_init=1.0, r_decay=0.0, r_min=1.0)
+    scale = 1.0 / math.sqrt(D)
+
+    def run(layers, lens, compressed, n_steps):
+        g = torch.Generator(dev).manual_seed(23)
+        caches = []
+        for n in lens:
+            cap = n + n_steps + c
+            k = torch.empty((layers, H, cap, D), dtype=torch.bfloat16, device=dev).normal_(generator=g)
+            v = torch.empty((layers, H, cap, D), dtype=torch.bfloat16, device=dev).normal_(generator=g)
+            deg = torch.full((layers, H, cap), 4 if compressed else 1, dtype=torch.int32, device=dev)
+            caches.append(b.Cache(k, v, deg, torch.log(deg.float()) if compressed else None, n))
+        ws = torch.empty(b.workspace_bytes(caches[0], p), dtype=torch.uint8, device=dev)
+        wsd = torch.empty(b.decode_workspace_bytes(Bz, H, G, D, max(lens) + n_steps), dtype=torch.uint8, device=dev)
+        kn = torch.empty((layers, H, Bz, D), dtype=torch.bfloat16, device=dev).normal_(generator=g)
+        vn = torch.empty((layers, H, Bz, D), dtype=torch.bfloat16, device=dev).normal_(generator=g)
+        new = [(kn[:, :, i:i + 1].contiguous(), vn[:, :, i:i + 1].contiguous()) for i in range(Bz)]
+        q = synth.queries(Bz, H * G, D, seed=3, dtype="bf16", device=dev)
+        out = torch.empty_like(q)
+        att_ev = []
+
+        def one_step(record):
+            for i, cache in enumerate(caches):
+                if compressed:
+                    b.compress_append(cache, new[i][0], new[i][1], p, ws)
+                else:   # the uncompressed cache only grows: same copy, no trigger
+                    cache.k[:, :, cache.len] = new[i][0][:, :, 0]
+                    cache.v[:, :, cache.len] = new[i][1][:, :, 0]
+                    cache.len += 1
+            max_len = max(x.len for x in caches)
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            e0.record()
+            for l in range(layers):
+                b.decode_attn(b.layer_views(caches, l, dev), H, G, q, out, scale, max_len, wsd)
+            e1.record()
+            if record:
+                att_ev.append((e0, e1))
+
+        for _ in range(3):
+            one_step(False)
+        torch.cuda.synchronize()
+        t0, t1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        t0.record()
+        for _ in range(n_steps - 3):
+            one_step(True)
+        t1.record()
+        torch.cuda.synchronize()
+        ms_step = t0.elapsed_time(t1) / (n_steps - 3)
+        ms_att = statistics.mean(x.elapsed_time(y) for x, y in att_ev)
+        rows = sum(x.len for x in caches) * H
+        del caches
+        torch.cuda.empty_cache()
+        return ms_step, ms_att, rows
+
+    comp_lens = [n // 4 for n in ctx]
+    ms_step, ms_att, rows = run(L, comp_lens, True, steps)
+    nbytes = decode_bytes(rows, D, 2) * L
+    res = {"batch": Bz, "layers": L, "steps": steps - 3, "context_tokens_total": sum(ctx), "cached_slots_total": rows // H,
+           "ms_per_step": ms_step, "ms_attention_per_step": ms_att, "decode_tok_s": Bz / (ms_step * 1e-3),
+           "attention_gbs": nbytes / (ms_att * 1e-3) / 1e9, "attention_frac_of_peak": nbytes / (ms_att * 1e-3) / 1e9 / peak_gbs}
+    Lu = 8
+    ms_step_u, ms_att_u, _ = run(Lu, ctx, False, 16)
+    res["uncompressed"] = {"layers_run": Lu, "ms_attention_per_step_32_layers": ms_att_u * L / Lu,
+                           "decode_tok_s_attention_only": Bz / (ms_att_u * L / Lu * 1e-3)}
+    res["attention_speedup"] = res["uncompressed"]["ms_attention_per_step_32_layers"] / ms_att
+    return res
+
+
 def bench_recluster(b, synth, dev, K, V):
     """Fixed-budget decoding branch (ckv_compress_append_recluster): a cache of B = 8192 slots per head with degrees
     above one, g = 256 appended tokens, then the re-clustering round over the whole cache back to B (paper defaults:
@@ -529,6 +609,7 @@ def main():
     ap.add_argument("--skip-cpu", action="store_true")
     ap.add_argument("--skip-decode-cfg4", action="store_true")
     ap.add_argument("--skip-variants", action="store_true")
+    ap.add_argument("--skip-serving", action="store_true")
     args = ap.parse_args()
     if args.impl == "reference":
         run_reference(args)
