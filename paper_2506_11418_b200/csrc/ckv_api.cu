@@ -175,12 +175,13 @@ cudaError_t run_round(const RoundPlan& rp, const Buf& src, const Buf& dst, int L
   a.LH = LH;
   a.status = reinterpret_cast<int32_t*>(ws);
   a.edge_stride = (int64_t)rp.n_chunks * (chunk / 2);
-  // bf16 with chunk 64 / 128 / 256 runs on the tile kernel, everything else on the general one; at chunk 64 the full
-  // chunks go to the warp-per-chunk kernel and only the shorter last chunk (if any) to the tile kernel
+  // bf16: the full chunks of chunk 64 go to the warp-per-chunk kernel, those of chunk 256 to the tcgen05 kernel, chunk 128
+  // and every shorter last chunk to the tile kernel; everything else runs on the general kernel
   auto launch_pass = [&](RoundArgs x) -> cudaError_t {
-    if (round_fast_supported(x, dtype, D)) {
+    const bool fast = round_fast_supported(x, dtype, D), umma = !fast && round_umma_supported(x, dtype, D);
+    if (fast || umma) {
       const int64_t n_full = (rp.hi - rp.lo) / chunk;
-      cudaError_t err = launch_round_fast(x, n_full, st);
+      cudaError_t err = fast ? launch_round_fast(x, n_full, st) : launch_round_umma(x, n_full, st);
       if (err != cudaSuccess || rp.n_chunks == n_full) return err;
       x.chunk_first = (int32_t)n_full;
       x.n_launch = 1;

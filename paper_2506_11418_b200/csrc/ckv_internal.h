@@ -116,6 +116,8 @@ size_t decode_partial_floats(int32_t Bz, int32_t H, int32_t G, int32_t D, int64_
 size_t round_smem_bytes(int chunk, int D);
 bool round_fast_supported(const RoundArgs& a, int dtype, int D);
 cudaError_t launch_round_fast(const RoundArgs& a, int64_t n_full, cudaStream_t st);
+bool round_umma_supported(const RoundArgs& a, int dtype, int D);
+cudaError_t launch_round_umma(const RoundArgs& a, int64_t n_full, cudaStream_t st);
 bool round_tile_supported(const RoundArgs& a, int dtype, int D);
 cudaError_t launch_round_tile(const RoundArgs& a, cudaStream_t st);
 
