@@ -1,7 +1,7 @@
 // Chunked Soft Matching round at chunk 256 (the paper's default), bf16, head_dim 128, full chunks, every selection
 // mode: the two contractions of a chunk run on the 5th-generation tensor cores with accumulators in tensor memory.
 //
-// One persistent CTA (8 warps) per SM walks the chunks.  Per chunk:
+// One persistent CTA (16 warps) per SM walks the chunks.  Per chunk:
 //   fetch     the K tile and the V tile arrive by TMA (cp.async.bulk.tensor, 128-byte swizzle); the tensor map views
 //             the cache as (column, parity, token pair, slab), so the A tokens (1st, 3rd, ...) and the B tokens land
 //             de-interleaved, each as two 128 x 64 operand tiles in the canonical swizzled layout.  K is fetched one
@@ -36,7 +36,7 @@ using namespace ptx;
 constexpr int kUC = 256;               // chunk
 constexpr int kUM = 128;               // A tokens = B tokens per chunk
 constexpr int kUD = 128;               // head_dim
-constexpr int kUThreads = 256;
+constexpr int kUThreads = 512;
 constexpr int kHalf = kUM * 128;       // one operand tile: 128 rows x 64 columns (128 bytes), swizzled: 16 KiB
 constexpr int kTileU = 4 * kHalf;      // A cols 0-63 | A cols 64-127 | B cols 0-63 | B cols 64-127
 constexpr uint32_t kTmemCols = 512;    // S: columns [0, 128); merged K: [128, 256); merged V: [256, 384)
@@ -50,9 +50,9 @@ constexpr int oUDeg = oUInv + 1024;             // int   [256] degrees by local 
 constexpr int oUDsum = oUDeg + 1024;            // int   [128] summed degree of each B token's cluster
 constexpr int oUBestB = oUDsum + 512;           // int   [128]
 constexpr int oUBestS = oUBestB + 512;          // float [128]
-constexpr int oUPartS = oUBestS + 512;          // float [128][2]
-constexpr int oUPartB = oUPartS + 1024;         // int   [128][2]
-constexpr int oUTw = oUPartB + 1024;            // uint  [3][128]: target B index << 16 | bf16 weight piece
+constexpr int oUPartS = oUBestS + 512;          // float [128][4]
+constexpr int oUPartB = oUPartS + 2048;         // int   [128][4]
+constexpr int oUTw = oUPartB + 2048;            // uint  [3][128]: target B index << 16 | bf16 weight piece
 constexpr int oUMask = oUTw + 1536;             // uint  [4]
 constexpr int oUNewDeg = oUMask + 16;           // int   [256]
 constexpr int oURowOf = oUNewDeg + 1024;        // ushort[256]: (part << 7 | row) of each output row
@@ -166,7 +166,7 @@ round_umma_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constan
     const int64_t beg = a.lo + (int64_t)ch * kUC;
     const int64_t eslot = lh * a.edge_stride + (int64_t)ch * kUM;
     int my_deg = 1, ext_b = -1, ext_sel = 0;
-    if (a.deg_src) my_deg = a.deg_src[lh * a.src_cap + beg + tid];
+    if (a.deg_src && tid < kUC) my_deg = a.deg_src[lh * a.src_cap + beg + tid];
     if (mode == kModeExternal && tid < kUM) {
       ext_b = a.edge_b[eslot + tid];
       ext_sel = a.sel[eslot + tid];
@@ -182,8 +182,10 @@ round_umma_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constan
         return;
       }
     }
-    degs[tid] = my_deg;
-    if (tid & 1) dsum[tid >> 1] = my_deg;  // a cluster starts with its B token's own degree
+    if (tid < kUC) {
+      degs[tid] = my_deg;
+      if (tid & 1) dsum[tid >> 1] = my_deg;  // a cluster starts with its B token's own degree
+    }
 
     if (need_sim) {
       // ---- S = A B^T on the tensor cores: K = 128 in eight steps of 16 (32 bytes inside the 128-byte swizzled row)
@@ -197,40 +199,35 @@ round_umma_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constan
         }
         umma_commit(bar_sim);
       }
-      // ---- squared norms from diagonals while the MMA runs: warp w takes B tokens 16 w .. 16 w + 15 (and, for the
-      //      ranking modes, A tokens 16 w .. 16 w + 15)
+      // ---- squared norms from diagonals while the MMA runs: warps 0-7 take 16 B tokens each, warps 8-15 (for the
+      //      ranking modes) 16 A tokens each
       {
-        float nb0[4] = {0.f, 0.f, 0.f, 0.f}, nb1[4] = {0.f, 0.f, 0.f, 0.f};
-        float na0[4] = {0.f, 0.f, 0.f, 0.f}, na1[4] = {0.f, 0.f, 0.f, 0.f};
-        const int rb = 16 * warp + (lane & 7);
+        const int w8 = warp & 7;
+        const bool for_a = warp >= 8;
+        if (!for_a || need_cos) {
+          float n0[4] = {0.f, 0.f, 0.f, 0.f}, n1[4] = {0.f, 0.f, 0.f, 0.f};
+          const uint32_t part = k_s + (for_a ? 0u : 2u * kHalf);
+          const int r0 = 16 * w8 + (lane & 7);
 #pragma unroll
-        for (int kq = 0; kq < 4; ++kq) {
-          uint32_t p[4], q[4];
-          ldsm_x4(k_s + 2 * kHalf + sw_off(rb, 4 * kq + (lane >> 3)), p);
-          ldsm_x4(k_s + 2 * kHalf + sw_off(rb + 8, 4 * kq + (lane >> 3)), q);
-          mma_bf16(nb0, p[0], q[0], p[1], q[1], p[0], p[1]);
-          mma_bf16(nb0, p[2], q[2], p[3], q[3], p[2], p[3]);
-          mma_bf16(nb1, p[0], q[0], p[1], q[1], q[0], q[1]);
-          mma_bf16(nb1, p[2], q[2], p[3], q[3], q[2], q[3]);
-          if (need_cos) {
-            uint32_t f0[4], f1[4];
-            const int ra = 16 * warp + (lane & 7) + ((lane >> 3) & 1) * 8;
-            ldsm_x4(k_s + sw_off(ra, 4 * kq + (lane >> 4)), f0);
-            ldsm_x4(k_s + sw_off(ra, 4 * kq + 2 + (lane >> 4)), f1);
-            mma_bf16(na0, f0[0], f0[1], f0[2], f0[3], f0[0], f0[2]);
-            mma_bf16(na0, f1[0], f1[1], f1[2], f1[3], f1[0], f1[2]);
-            mma_bf16(na1, f0[0], f0[1], f0[2], f0[3], f0[1], f0[3]);
-            mma_bf16(na1, f1[0], f1[1], f1[2], f1[3], f1[1], f1[3]);
+          for (int kq = 0; kq < 4; ++kq) {
+            uint32_t p[4], q[4];
+            ldsm_x4(part + sw_off(r0, 4 * kq + (lane >> 3)), p);
+            ldsm_x4(part + sw_off(r0 + 8, 4 * kq + (lane >> 3)), q);
+            // rows 0-7 <- the first eight tokens, rows 8-15 <- the next eight; columns: the first eight, then the next
+            mma_bf16(n0, p[0], q[0], p[1], q[1], p[0], p[1]);
+            mma_bf16(n0, p[2], q[2], p[3], q[3], p[2], p[3]);
+            mma_bf16(n1, p[0], q[0], p[1], q[1], q[0], q[1]);
+            mma_bf16(n1, p[2], q[2], p[3], q[3], q[2], q[3]);
           }
-        }
-        // the diagonal entry of row r sits in lane 4 r' + r'/2 (r' = r mod 8), register r' & 1 (+2 for rows 8-15)
-        if (t == (g >> 1)) {
-          const float s0 = (g & 1) ? nb0[1] : nb0[0], s1 = (g & 1) ? nb1[3] : nb1[2];
-          inv_nrm[kUM + 16 * warp + g] = s0 > 0.f ? rsqrtf(s0) : 0.f;  // a zero key has similarity 0 with everything
-          inv_nrm[kUM + 16 * warp + 8 + g] = s1 > 0.f ? rsqrtf(s1) : 0.f;
-          const float a0 = (g & 1) ? na0[1] : na0[0], a1 = (g & 1) ? na1[3] : na1[2];
-          inv_nrm[16 * warp + g] = need_cos ? (a0 > 0.f ? rsqrtf(a0) : 0.f) : 1.f;
-          inv_nrm[16 * warp + 8 + g] = need_cos ? (a1 > 0.f ? rsqrtf(a1) : 0.f) : 1.f;
+          // the diagonal entry of row r sits in lane 4 r' + r'/2 (r' = r mod 8), register r' & 1 (+2 for rows 8-15)
+          if (t == (g >> 1)) {
+            const float s0 = (g & 1) ? n0[1] : n0[0], s1 = (g & 1) ? n1[3] : n1[2];
+            const int base = (for_a ? 0 : kUM) + 16 * w8;
+            inv_nrm[base + g] = s0 > 0.f ? rsqrtf(s0) : 0.f;  // a zero key has similarity 0 with everything
+            inv_nrm[base + 8 + g] = s1 > 0.f ? rsqrtf(s1) : 0.f;
+          }
+        } else if (lane < 16) {
+          inv_nrm[16 * w8 + lane] = 1.f;  // the argmax alone does not need |a|
         }
       }
       {
@@ -241,34 +238,31 @@ round_umma_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constan
         }
         ph_sim ^= 1;
       }
-      // ---- Eq. 2 and the row argmax: this thread owns A token 32 (warp % 4) + lane and 64 of the 128 columns
+      // ---- Eq. 2 and the row argmax: this thread owns A token 32 (warp % 4) + lane and 32 of the 128 columns
       {
         tc_fence_after();
-        const int ai = 32 * (warp & 3) + lane, c0 = 64 * (warp >> 2);
+        const int ai = 32 * (warp & 3) + lane, cq = warp >> 2, c0 = 32 * cq;
         const float inva = inv_nrm[ai];
         float bv = -INFINITY;
         int bi = INT_MAX;
+        float v[32];
+        tmem_ld32(tmem + ((uint32_t)(32 * (warp & 3)) << 16) + (uint32_t)c0, v);
 #pragma unroll
-        for (int h = 0; h < 2; ++h) {
-          float v[32];
-          tmem_ld32(tmem + ((uint32_t)(32 * (warp & 3)) << 16) + (uint32_t)(c0 + 32 * h), v);
+        for (int j = 0; j < 32; j += 4) {
+          const float4 ib = *reinterpret_cast<const float4*>(inv_nrm + kUM + c0 + j);
+          const float ibs[4] = {ib.x, ib.y, ib.z, ib.w};
 #pragma unroll
-          for (int j = 0; j < 32; j += 4) {
-            const float4 ib = *reinterpret_cast<const float4*>(inv_nrm + kUM + c0 + 32 * h + j);
-            const float ibs[4] = {ib.x, ib.y, ib.z, ib.w};
-#pragma unroll
-            for (int e = 0; e < 4; ++e) {
-              float sim = v[j + e] * ibs[e] * inva;
-              sim += 0.f;  // -0 -> +0, so that the ranking orders zeros as equal
-              if (sim > bv) {  // columns in increasing order: the lowest index wins ties
-                bv = sim;
-                bi = c0 + 32 * h + j + e;
-              }
+          for (int e = 0; e < 4; ++e) {
+            float sim = v[j + e] * ibs[e] * inva;
+            sim += 0.f;  // -0 -> +0, so that the ranking orders zeros as equal
+            if (sim > bv) {  // columns in increasing order: the lowest index wins ties
+              bv = sim;
+              bi = c0 + j + e;
             }
           }
         }
-        part_s[ai * 2 + (warp >> 2)] = bv;
-        part_b[ai * 2 + (warp >> 2)] = bi;
+        part_s[ai * 4 + cq] = bv;
+        part_b[ai * 4 + cq] = bi;
         tc_fence_before();
       }
     }
@@ -279,13 +273,15 @@ round_umma_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constan
       float bv = -INFINITY;
       int bi = -1;
       if (need_sim) {
-        const float s0 = part_s[2 * tid], s1 = part_s[2 * tid + 1];
-        const int b0 = part_b[2 * tid], b1 = part_b[2 * tid + 1];
-        bv = s0;
-        bi = b0;
-        if (b0 == INT_MAX || (b1 != INT_MAX && s1 > s0)) {  // the second half holds the higher columns: strict >
-          bv = s1;
-          bi = b1;
+        bi = INT_MAX;
+#pragma unroll
+        for (int q = 0; q < 4; ++q) {  // column quarters in increasing order: strict > keeps the lowest index
+          const float ps = part_s[4 * tid + q];
+          const int pb = part_b[4 * tid + q];
+          if (pb != INT_MAX && (bi == INT_MAX || ps > bv)) {
+            bv = ps;
+            bi = pb;
+          }
         }
         if (bi == INT_MAX) bi = -1;
         best_s[tid] = bv;
@@ -349,7 +345,7 @@ round_umma_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constan
       }
       return cnt;
     };
-    {
+    if (tid < kUC) {
       const int ai = tid >> 1;
       const bool gone = !(tid & 1) && sel_bit(ai);
       const int keeper = gone ? 2 * best_b[ai] + 1 : tid;
@@ -375,7 +371,7 @@ round_umma_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constan
     for (int piece = 0; piece < n_pieces; ++piece) {
       for (int ah = 0; ah < 2; ++ah) {
 #pragma unroll
-        for (int i = 0; i < 4; ++i)
+        for (int i = 0; i < kHalf / 16 / kUThreads; ++i)
           asm volatile("st.shared.v4.u32 [%0], {%1,%1,%1,%1};" ::"r"(w_s + (uint32_t)(tid + kUThreads * i) * 16u), "r"(0u) : "memory");
         __syncthreads();
         if (tid < 64) {
@@ -410,17 +406,17 @@ round_umma_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constan
       }
     }
 
-    // ---- epilogue: thread = centroid row b of one tile (warps 0-3: K, warps 4-7: V): own term, division, rounding;
+    // ---- epilogue: thread = centroid row b of one tile and one half of its columns: own term, division, rounding;
     //      the centroid replaces the B token's row in the tile; an untouched row stays bit for bit
     {
       tc_fence_after();
-      const int b = 32 * (warp & 3) + lane, part = warp >> 2;
+      const int b = 32 * (warp & 3) + lane, part = (warp >> 2) & 1, ch2 = warp >> 3;  // K or V tile; columns 64 ch2 .. + 63
       const uint32_t tile_b = (part ? v_s : k_s) + 2 * kHalf;
       const int nb = degs[2 * b + 1], ns = dsum[b];
       const bool merged = ns != nb;
       const float wb = (float)nb, inv = 1.0f / (float)ns;
 #pragma unroll 1
-      for (int c4 = 0; c4 < 4; ++c4) {
+      for (int c4 = 2 * ch2; c4 < 2 * ch2 + 2; ++c4) {
         float v[32];
         tmem_ld32(tmem + ((uint32_t)(32 * (warp & 3)) << 16) + (uint32_t)(128 * (1 + part) + 32 * c4), v);
         if (merged) {
