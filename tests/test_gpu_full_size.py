@@ -83,6 +83,27 @@ def test_config2_llama8b_32k_one_round():
     torch.cuda.empty_cache()
 
 
+def test_llama8b_32k_chunk256_paper_schedule():
+    """The paper's default chunk (256) and schedule on the 32k workload, to a 25 % budget: six rounds ranked per head on
+    the tensor-memory kernel (full chunks) and the tile kernel (the shorter last chunk of every round)."""
+    need_free(12)
+    b = B()
+    s = synth.CONFIGS["llama8b_32k"]["s"]
+    p = b.Params(chunk=256, n_sink=16, n_recent=64, n_rounds_max=16, r_init=0.8, r_decay=0.2, r_min=0.2, budget=s // 4)
+    dst, rounds, _ = full_prefill("llama8b_32k", p, [(2, 3), (29, 0)])
+    assert dst.len == s // 4 and rounds >= 4
+    torch.cuda.empty_cache()
+
+
+def test_llama8b_32k_chunk256_every_edge_and_per_chunk_ranking():
+    need_free(12)
+    b = B()
+    for p in (b.Params(chunk=256, n_sink=0, n_recent=0, n_rounds_max=1, r_init=1.0, r_decay=0.0, r_min=1.0),
+              b.Params(chunk=256, n_sink=0, n_recent=0, n_rounds_max=2, r_init=0.5, r_decay=0.0, r_min=0.5, select=b.SELECT_CHUNK)):
+        dst, rounds, _ = full_prefill("llama8b_32k", p, [(9, 6)])
+        torch.cuda.empty_cache()
+
+
 def test_config3_llama8b_128k_two_rounds_ratio_one():
     """131072 tokens to 25 %: two rounds at ratio 1."""
     need_free(60)
