@@ -37,7 +37,7 @@ SELECT_CHUNK = 1   # rank inside each chunk
 @dataclass
 class Params:
     """Algorithm 1's `Require` line plus Eq. 4's schedule."""
-    chunk: int = 256          # c
+    chunk: int = 256          # c; 0 = no chunking (one chunk spans the whole middle region)
     n_sink: int = 16          # n1
     n_recent: int = 64        # n2
     n_rounds_max: int = 8
@@ -80,6 +80,8 @@ def chunk_bounds(s: int, n_sink: int, n_recent: int, c: int):
     hi = max(lo, s - n_recent)
     if hi - lo < 2:
         return lo, hi, []
+    if c == 0:  # no chunking: plain Bipartite Soft Matching over the whole middle region (Sec. 5.2, the "w/o chunk" ablation of Table 8)
+        c = hi - lo
     return lo, hi, [(b, min(b + c, hi)) for b in range(lo, hi, c)]
 
 

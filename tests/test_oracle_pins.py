@@ -97,6 +97,27 @@ def test_p1_brute_force_rounds(c, r, sink, recent, s):
         K, V, deg = Ko, Vo, do
 
 
+@pytest.mark.parametrize("r,sink,recent,s", [(1.0, 0, 0, 12), (0.5, 2, 1, 15), (0.34, 0, 3, 13)])
+def test_no_chunking_is_plain_bipartite_soft_matching(r, sink, recent, s):
+    """chunk = 0: the whole middle region is one chunk (the "w/o chunk" ablation): brute force with a chunk larger than
+    the sequence, two rounds; the similarity step then costs n^2 d / 4 multiply-adds (Table 1, BSM)."""
+    rng = np.random.default_rng(200 + s)
+    K, V = rand_cache(rng, 1, 1, s, 5, ar=0.7)
+    deg = np.ones((1, 1, s), dtype=np.int64)
+    p = O.Params(chunk=0, n_sink=sink, n_recent=recent, select=O.SELECT_GLOBAL, budget=0)
+    for _ in range(2):
+        Ko, Vo, do, _, log = O.csm_round(K, V, deg, p, r)
+        n_edges = len(log.edges[0].a_pos)
+        mid = K.shape[2] - sink - recent
+        assert n_edges == (mid + 1) // 2 and log.macs == ((mid + 1) // 2) * (mid // 2) * 5
+        M = int(math.floor(r * n_edges + 1e-9))
+        Kb, Vb, db, _ = brute_round(K[0, 0].tolist(), V[0, 0].tolist(), deg[0, 0].tolist(), sink, recent, 10 ** 9, M)
+        np.testing.assert_allclose(Ko[0, 0], Kb, rtol=1e-12, atol=1e-12)
+        np.testing.assert_allclose(Vo[0, 0], Vb, rtol=1e-12, atol=1e-12)
+        np.testing.assert_array_equal(do[0, 0], db)
+        K, V, deg = Ko, Vo, do
+
+
 def test_p1_chunk_mode_is_per_chunk_top_m():
     rng = np.random.default_rng(7)
     s, c = 24, 8
