@@ -278,6 +278,7 @@ def run_gpu(args):
     if rank == 0 and not args.skip_variants:
         extra["compress_variants"] = bench_compress_variants(b, synth, dev, K, V, peaks["hbm_gbs"], args.layers == 0)
         extra["recluster"] = bench_recluster(b, synth, dev, K, V)
+        extra["no_chunk"] = bench_no_chunk(b, dev, K, V, peaks)
 
     # end to end: inputs start in pinned host memory, the compressed cache and the decode output end there
     e2e = None
@@ -522,6 +523,34 @@ def bench_serving_mix(b, synth, dev, peak_gbs, steps=128):
                            "decode_tok_s_attention_only": Bz / (ms_att_u * L / Lu * 1e-3)}
     res["attention_speedup"] = res["uncompressed"]["ms_attention_per_step_32_layers"] / ms_att
     return res
+
+
+def bench_no_chunk(b, dev, K, V, peaks):
+    """chunk = 0 (plain Bipartite Soft Matching, the paper's "w/o chunk" ablation): every A token against every B token
+    of its head, n^2 d / 4 multiply-adds per head -- the one compute-bound variant.  One round at ratio 1 over the first
+    16384 tokens of 4 layers x 8 KV heads; the tensor-core rate counts the similarity contraction alone."""
+    import torch
+    L, H, n, D = min(4, K.shape[0]), K.shape[1], 16384, K.shape[3]
+    Ks, Vs = K[:L, :, :n].contiguous(), V[:L, :, :n].contiguous()
+    p = b.Params(chunk=0, n_sink=0, n_recent=0, n_rounds_max=1, r_init=1.0, r_decay=0.0, r_min=1.0)
+    src = b.Cache(Ks, Vs, None, None, n)
+    out_len, _, cap = b.compress_plan(n, p)
+    dst = b.Cache.empty(L, H, cap, D, Ks.dtype, dev)
+    ws = torch.empty(b.workspace_bytes(src, p), dtype=torch.uint8, device=dev)
+    b.compress_prefill(src, dst, p, ws)
+    torch.cuda.synchronize()
+    t0, t1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    t0.record()
+    iters = 3
+    for _ in range(iters):
+        b.compress_prefill(src, dst, p, ws)
+    t1.record()
+    torch.cuda.synchronize()
+    ms = t0.elapsed_time(t1) / iters
+    flops = 2.0 * L * H * (n / 2) * (n / 2) * D
+    tf = flops / (ms * 1e-3) / 1e12
+    return {"layers": L, "seq": n, "out_len": out_len, "ms": ms, "similarity_tflops": tf, "bound": "tensor",
+            "frac_of_bf16_peak": tf / peaks["bf16_tflops"], "status": b.workspace_status(ws)}
 
 
 def bench_recluster(b, synth, dev, K, V):

@@ -15,8 +15,8 @@
  *    are valid; deg and logdeg: [L, H, cap].  K and V must be 16-byte aligned.
  *  - Thread safety: calls on distinct streams with distinct workspaces and outputs do
  *    not interfere.
- *  - This version supports D = 128 and even chunk sizes 2..256; anything else returns
- *    CKV_ERR_UNSUPPORTED.
+ *  - This version supports D = 128 and even chunk sizes 2..256 (or 0 = no chunking); anything else
+ *    returns CKV_ERR_UNSUPPORTED.
  */
 #ifndef CKV_H_
 #define CKV_H_
@@ -62,7 +62,9 @@ typedef struct ckv_cache {
 
 /* Algorithm 1's inputs and Eq. 4's schedule. */
 typedef struct ckv_params {
-  int32_t chunk;        /* c: chunk size, even */
+  int32_t chunk;        /* c: chunk size, even; 0 = no chunking: every A token is matched against every B token of its
+                           (layer, head) -- plain Bipartite Soft Matching, Sec. 5.2 / Table 8 "w/o chunk"; bf16 only,
+                           ckv_compress_prefill and ckv_compress_append_recluster only */
   int32_t n_sink;       /* n1: leading tokens never merged */
   int32_t n_recent;     /* n2: trailing tokens never merged */
   int32_t n_rounds_max; /* upper bound on clustering rounds per call */

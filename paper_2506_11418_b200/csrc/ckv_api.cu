@@ -24,7 +24,7 @@ inline size_t align_up(size_t x, size_t a = 256) { return (x + a - 1) / a * a; }
 
 int check_params(const ckv_params* p) {
   if (!p) return CKV_ERR_INVALID_ARG;
-  if (p->chunk < 2 || (p->chunk & 1)) return CKV_ERR_INVALID_ARG;
+  if (p->chunk != 0 && (p->chunk < 2 || (p->chunk & 1))) return CKV_ERR_INVALID_ARG;  // 0: no chunking
   if (p->n_sink < 0 || p->n_recent < 0 || p->n_rounds_max < 0 || p->budget < 0) return CKV_ERR_INVALID_ARG;
   if (!(p->r_init >= 0.f && p->r_init <= 1.f) || !(p->r_decay >= 0.f) || !(p->r_min >= 0.f && p->r_min <= 1.f))
     return CKV_ERR_INVALID_ARG;
@@ -46,6 +46,20 @@ int plan_rounds(int64_t len, const ckv_params& p, std::vector<RoundPlan>& plan) 
     rp.lo = std::min<int64_t>(p.n_sink, s);
     rp.hi = std::max<int64_t>(rp.lo, s - p.n_recent);
     const int64_t mid = rp.hi - rp.lo;
+    if (p.chunk == 0) {
+      // no chunking (plain Bipartite Soft Matching): the middle region is one chunk; ranking per chunk and per head coincide
+      rp.n_chunks = mid >= 2 ? 1 : 0;
+      rp.n_edges = mid >= 2 ? (mid + 1) / 2 : 0;
+      rp.M = floor_ratio(r, rp.n_edges);
+      if (p.budget > 0 && p.select == CKV_SELECT_GLOBAL) rp.M = std::min<int64_t>(rp.M, s - p.budget);
+      rp.mode = rp.M == 0 ? -1 : kModeExternal;
+      rp.m_full = rp.m_tail = 0;
+      rp.s_out = s - rp.M;
+      if (rp.M == 0 && p.budget > 0) return CKV_ERR_NO_PROGRESS;
+      plan.push_back(rp);
+      s = rp.s_out;
+      continue;
+    }
     const int c = p.chunk;
     const int64_t n_full = mid >= 2 ? mid / c : 0;
     const int tail = mid >= 2 ? (int)(mid % c) : 0;
@@ -80,6 +94,7 @@ struct Workspace {
   int64_t tmp_cap;
   size_t edge_sim, edge_b, sel, chunk_off;
   int64_t edge_stride;
+  size_t bsm;  // scratch of the no-chunk rounds
   size_t assign_step;
   int64_t assign_stride;
   size_t total;
@@ -106,10 +121,17 @@ Workspace layout_workspace(int64_t LH, int D, int esize, int chunk, const std::v
   w.tmp_deg = take((size_t)LH * w.tmp_cap * 4);
   w.tmp_logdeg = take((size_t)LH * w.tmp_cap * 4);
   w.edge_stride = max_chunks * (chunk / 2);
+  int64_t bsm_mid = 0;
+  if (chunk == 0)
+    for (size_t j = 0; j < R; ++j) {
+      w.edge_stride = std::max(w.edge_stride, plan[j].n_edges);
+      bsm_mid = std::max(bsm_mid, plan[j].hi - plan[j].lo);
+    }
   w.edge_sim = take((size_t)LH * w.edge_stride * 4);
   w.edge_b = take((size_t)LH * w.edge_stride * 4);
   w.sel = take((size_t)LH * w.edge_stride);
-  w.chunk_off = take((size_t)LH * max_chunks * 4);
+  w.chunk_off = take((size_t)LH * std::max<int64_t>(max_chunks, 1) * 4);
+  w.bsm = take(chunk == 0 ? bsm_workspace_bytes(LH, bsm_mid) : 0);
   w.assign_stride = (want_assign && R >= 2) ? max_sin : 0;
   w.assign_step = take((size_t)LH * w.assign_stride * 4);
   w.total = off;
@@ -167,6 +189,23 @@ cudaError_t run_round(const RoundPlan& rp, const Buf& src, const Buf& dst, int L
   a.assign = assign; a.assign_stride = assign_stride;
   a.src_cap = src.cap; a.dst_cap = dst.cap;
   a.lo = rp.lo; a.hi = rp.hi;
+  if (chunk == 0) {
+    // no chunking: norms + tensor-core matching over all A x B pairs of a head, ranking, merge by member scan
+    if (!bsm_supported(dtype, D)) return cudaErrorInvalidValue;
+    a.LH = LH;
+    a.status = reinterpret_cast<int32_t*>(ws);
+    a.edge_stride = rp.n_edges;
+    a.edge_sim = reinterpret_cast<float*>(ws + w.edge_sim);
+    a.edge_b = reinterpret_cast<int32_t*>(ws + w.edge_b);
+    a.sel = ws + w.sel;
+    a.chunk_out_off = reinterpret_cast<int32_t*>(ws + w.chunk_off);
+    if ((e = launch_bsm_match(a, ws + w.bsm, st)) != cudaSuccess) return e;
+    SelectArgs s{};
+    s.edge_sim = a.edge_sim; s.sel = a.sel; s.chunk_out_off = a.chunk_out_off;
+    s.edge_stride = a.edge_stride; s.M = rp.M; s.lo = rp.lo; s.chunk = (int32_t)(2 * rp.n_edges); s.n_chunks = 1; s.LH = LH;
+    if ((e = launch_select(s, st)) != cudaSuccess) return e;
+    return launch_bsm_merge(a, ws + w.bsm, st);
+  }
   a.chunk = chunk; a.n_chunks = rp.n_chunks;
   a.chunk_first = 0; a.n_launch = rp.n_chunks;
   a.m_full = rp.m_full; a.m_tail = rp.m_tail;
@@ -306,7 +345,7 @@ size_t ckv_workspace_bytes(const ckv_cache* shape, const ckv_params* params) {
   }
   // append: one window of `chunk` tokens, with a tmp window for odd round counts
   const ckv_params wp = window_params(*params);
-  if (plan_rounds(params->chunk, wp, plan) == CKV_OK) {
+  if (params->chunk > 0 && plan_rounds(params->chunk, wp, plan) == CKV_OK) {
     const size_t win = align_up((size_t)LH * params->chunk * shape->D * es) * 2 + align_up((size_t)LH * params->chunk * 4) * 2;
     need = std::max(need, layout_workspace(LH, shape->D, es, params->chunk, plan, false).total + win);
   }
@@ -328,6 +367,7 @@ int ckv_compress_prefill(const ckv_cache* src, ckv_cache* dst, const ckv_params*
   if (overlaps(src->k, src_bytes, dst->k, dst_bytes) || overlaps(src->v, src_bytes, dst->v, dst_bytes) ||
       overlaps(src->k, src_bytes, dst->v, dst_bytes) || overlaps(src->v, src_bytes, dst->k, dst_bytes))
     return CKV_ERR_INVALID_ARG;
+  if (params->chunk == 0 && !bsm_supported(src->dtype, src->D)) return CKV_ERR_UNSUPPORTED;
   std::vector<RoundPlan> plan;
   if ((st = plan_rounds(src->len, *params, plan)) != CKV_OK) return st;
   if (dst->cap < dst_cap_needed(plan, src->len)) return CKV_ERR_CAPACITY;
@@ -358,6 +398,7 @@ int ckv_compress_append(ckv_cache* cache, const void* k_new, const void* v_new, 
   if (t_new < 0 || (t_new > 0 && (!k_new || !v_new))) return CKV_ERR_INVALID_ARG;
   if (!cache->k || !cache->v || !cache->deg) return CKV_ERR_INVALID_ARG;
   if (!aligned16(cache->k) || !aligned16(cache->v) || !aligned16(k_new) || !aligned16(v_new)) return CKV_ERR_ALIGNMENT;
+  if (params->chunk == 0) return CKV_ERR_INVALID_ARG;  // the append trigger is a window of `chunk` tokens
   if (cache->pending >= params->chunk) return CKV_ERR_INVALID_ARG;
   const int64_t LH = (int64_t)cache->L * cache->H;
   const int D = cache->D, es = esize_of(cache->dtype), c = params->chunk;

@@ -1,0 +1,531 @@
+// Bipartite Soft Matching without chunks (chunk = 0; Sec. 5.2, the "w/o chunk" ablation of Table 8): every A token
+// (1st, 3rd, ... of the middle region) is matched against every B token of the same (layer, head), n^2 d / 4
+// multiply-adds per head (Table 1) -- a dense contraction, compute-bound, so it runs as a tensor-core GEMM with the
+// argmax fused into the epilogue:
+//   bsm_norm_kernel     inverse key norms of the A and B tokens
+//   bsm_match_kernel    one CTA per 128 A tokens walks all B tokens in tiles of 128: a TMA warp streams B tiles
+//                       (de-interleaving tensor map, 128-byte swizzle) through a 4-stage ring, an MMA warp issues
+//                       tcgen05.mma (128 x 128 x 128 per tile) into one of two tensor-memory accumulators, eight
+//                       consumer warps read the other accumulator (tcgen05.ld), scale by 1 / |b| and keep a running
+//                       row argmax (lowest B position on ties); the edge (cosine, target) is written at the end
+//   select_kernel       the M best edges of the head (shared with the chunked path)
+//   bsm_prepare_kernel  prefix counts of the selected edges (output slots) and the number of members per B token
+//   bsm_merge_kernel    one warp per surviving token: Eq. 5 over its members, found by scanning the head's edges
+// bf16, head_dim 128.  Waits are bounded; a role whose wait gives up sets the status word and stops; the others follow.
+#include <cuda.h>
+
+#include <algorithm>
+#include <climits>
+#include <cstdint>
+
+#include "../../include/ckv.h"
+#include "ckv_common.cuh"
+#include "ckv_internal.h"
+#include "ckv_ptx.cuh"
+
+namespace ckv {
+
+namespace {
+
+using namespace ptx;
+
+constexpr int kBD = 128;          // head_dim
+constexpr int kBT = 128;          // tile: A tokens per CTA, B tokens per step
+constexpr int kBHalf = kBT * 128; // one swizzled operand tile: 128 rows x 64 columns
+constexpr int kBStages = 5;        // B tiles in flight; a stage is free again as soon as the tensor core has read it
+constexpr int kBInvSlots = 8;      // 1/|b| slices: consumers are at most three tiles behind the fetch of a slot's next use
+constexpr int kBConsumers = 8;    // warps
+constexpr int kBThreads = (kBConsumers + 2) * 32;
+// shared memory (1024-byte aligned base): A tile | B ring | 1/|b| ring | barriers | partial argmaxes | tmem address
+constexpr int oBA = 0;
+constexpr int oBB = 2 * kBHalf;
+constexpr int oBInv = oBB + kBStages * 2 * kBHalf;
+constexpr int oBBar = oBInv + kBInvSlots * 512;
+constexpr int oBPart = oBBar + 256;
+constexpr int oBTmem = oBPart + kBT * 2 * 8;
+constexpr int kBBytes = oBTmem + 16;
+
+struct BsmArgs {
+  const __nv_bfloat16* k_src;
+  int64_t src_cap, lo;
+  int32_t nA, nB;         // A and B tokens of the middle region
+  int64_t inv_stride;     // floats per head of inv_a / inv_b (multiple of 128)
+  float* inv_a;
+  float* inv_b;
+  float* edge_sim;        // [LH, edge_stride]
+  int32_t* edge_b;        // [LH, edge_stride]  local offset 2 b + 1 of the target
+  int64_t edge_stride;
+  int32_t* status;
+};
+
+__device__ __forceinline__ void mbar_arrive(uint32_t bar) { asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory"); }
+
+__host__ __device__ constexpr uint32_t bsm_idesc() {  // bf16 x bf16 -> fp32, both K-major, M = 128, N = 128
+  return (1u << 4) | (1u << 7) | (1u << 10) | ((128u >> 3) << 17) | ((128u >> 4) << 24);
+}
+
+// inverse norms: one warp per token of the middle region
+__global__ void __launch_bounds__(256) bsm_norm_kernel(const BsmArgs a) {
+  const int lh = blockIdx.y, lane = threadIdx.x & 31;
+  const int64_t mid = (int64_t)a.nA + a.nB;
+  const int64_t o = (int64_t)blockIdx.x * 8 + (threadIdx.x >> 5);
+  if (o >= mid) return;
+  const float4 x = load4(a.k_src + ((int64_t)lh * a.src_cap + a.lo + o) * kBD + lane * 4);
+  const float ss = warp_sum(fmaf(x.x, x.x, fmaf(x.y, x.y, fmaf(x.z, x.z, x.w * x.w))));
+  if (lane == 0) ((o & 1) ? a.inv_b : a.inv_a)[(int64_t)lh * a.inv_stride + (o >> 1)] = ss > 0.f ? rsqrtf(ss) : 0.f;
+}
+
+__global__ void __launch_bounds__(kBThreads, 1) bsm_match_kernel(const __grid_constant__ CUtensorMap tm_k, const BsmArgs a) {
+  extern __shared__ unsigned char smem_raw[];
+  unsigned char* smem = reinterpret_cast<unsigned char*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
+  const uint32_t s_base = smem_u32(smem);
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  const int lh = blockIdx.y, atile = blockIdx.x;
+  const int n_tiles = (a.nB + kBT - 1) / kBT;
+  auto bar_full = [&](int s) { return s_base + oBBar + 8u * s; };
+  auto bar_empty = [&](int s) { return s_base + oBBar + 8u * (kBStages + s); };
+  auto bar_tfull = [&](int b) { return s_base + oBBar + 8u * (2 * kBStages + b); };
+  auto bar_tempty = [&](int b) { return s_base + oBBar + 8u * (2 * kBStages + 2 + b); };
+  const uint32_t bar_a = s_base + oBBar + 8u * (2 * kBStages + 4);
+  auto bar_inv = [&](int i) { return s_base + oBBar + 8u * (2 * kBStages + 5 + i); };
+
+  if (tid == 0) {
+    for (int s = 0; s < kBStages; ++s) {
+      mbar_init(bar_full(s), 1);
+      mbar_init(bar_empty(s), 1);  // the MMA's commit
+    }
+    for (int b = 0; b < 2; ++b) {
+      mbar_init(bar_tfull(b), 1);
+      mbar_init(bar_tempty(b), kBConsumers);
+    }
+    mbar_init(bar_a, 1);
+    for (int i = 0; i < kBInvSlots; ++i) mbar_init(bar_inv(i), 1);
+    mbar_init_fence();
+  }
+  if (warp == 0) tmem_alloc(s_base + oBTmem, 256);
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const uint32_t tmem = *reinterpret_cast<volatile uint32_t*>(smem + oBTmem);
+  bool failed = false;
+
+  if (warp == kBConsumers) {
+    // ------------------------------------------------------------------ TMA warp: the A tile once, then the B tiles
+    if (lane == 0) {
+      mbar_arrive_expect_tx(bar_a, 2 * kBHalf);
+      tma_load_4d(s_base + oBA, &tm_k, 0, 0, atile * kBT, lh, bar_a);
+      tma_load_4d(s_base + oBA + kBHalf, &tm_k, 64, 0, atile * kBT, lh, bar_a);
+      for (int j = 0; j < n_tiles && !failed; ++j) {
+        const int s = j % kBStages;
+        if (!mbar_wait(bar_empty(s), (uint32_t)(((j / kBStages) & 1) ^ 1))) {
+          failed = true;
+          break;
+        }
+        const uint32_t dst = s_base + oBB + (uint32_t)s * 2 * kBHalf;
+        mbar_arrive_expect_tx(bar_full(s), 2 * kBHalf);
+        tma_load_4d(dst, &tm_k, 0, 1, j * kBT, lh, bar_full(s));
+        tma_load_4d(dst + kBHalf, &tm_k, 64, 1, j * kBT, lh, bar_full(s));
+        // The slice slot of tile j was last read for tile j - 8; this fetch runs after the MMA of tile j - 5 completed, which
+        // was issued after the consumers released the accumulator of tile j - 7: they are done with tile j - 8.
+        mbar_arrive_expect_tx(bar_inv(j % kBInvSlots), 512);
+        bulk_load(s_base + oBInv + (uint32_t)(j % kBInvSlots) * 512, a.inv_b + (int64_t)lh * a.inv_stride + (int64_t)j * kBT, 512,
+                  bar_inv(j % kBInvSlots));
+      }
+    }
+  } else if (warp == kBConsumers + 1) {
+    // ------------------------------------------------------------------ MMA warp: S tile = A B^T into accumulator j & 1
+    if (lane == 0) {
+      failed = !mbar_wait(bar_a, 0);
+      for (int j = 0; j < n_tiles && !failed; ++j) {
+        const int s = j % kBStages, b = j & 1;
+        if (!mbar_wait(bar_full(s), (uint32_t)((j / kBStages) & 1)) || !mbar_wait(bar_tempty(b), (uint32_t)(((j >> 1) & 1) ^ 1))) {
+          failed = true;
+          break;
+        }
+        tc_fence_after();
+        const uint32_t bt = s_base + oBB + (uint32_t)s * 2 * kBHalf;
+#pragma unroll
+        for (int ks = 0; ks < 8; ++ks) {
+          const uint32_t off = (uint32_t)(ks >> 2) * kBHalf + (uint32_t)(ks & 3) * 32u;
+          umma_bf16(tmem + (uint32_t)b * kBT, umma_desc_sw128(s_base + oBA + off, 16, 1024), umma_desc_sw128(bt + off, 16, 1024),
+                    bsm_idesc(), ks ? 1u : 0u);
+        }
+        umma_commit(bar_empty(s));  // the tensor core has read the B tile
+        umma_commit(bar_tfull(b));  // the accumulator is complete
+      }
+    }
+  } else {
+    // ------------------------------------------------------------------ consumers: running row argmax
+    const int q = warp & 3, half = warp >> 2;  // tensor-memory lanes 32 q .. + 31; columns 64 half .. + 63 of every tile
+    const int row = 32 * q + lane;
+    float bv = -INFINITY;
+    int bi = INT_MAX;
+    for (int j = 0; j < n_tiles && !failed; ++j) {
+      const int b = j & 1;
+      // (the consumers never look at the B ring: its stages may be refilled while they are still on this tile)
+      if (!mbar_wait(bar_inv(j % kBInvSlots), (uint32_t)((j / kBInvSlots) & 1)) || !mbar_wait(bar_tfull(b), (uint32_t)((j >> 1) & 1))) {
+        failed = true;
+        break;
+      }
+      tc_fence_after();
+      const float* invb = reinterpret_cast<const float*>(smem + oBInv + (j % kBInvSlots) * 512) + 64 * half;
+      const int col0 = j * kBT + 64 * half;
+      const bool ragged = col0 + 64 > a.nB;  // only the last tile can hold columns that are not B tokens
+#pragma unroll
+      for (int h = 0; h < 2; ++h) {
+        float v[32];
+        tmem_ld32(tmem + ((uint32_t)(32 * q) << 16) + (uint32_t)(b * kBT + 64 * half + 32 * h), v);
+#pragma unroll
+        for (int e4 = 0; e4 < 32; e4 += 4) {
+          const float4 ib = *reinterpret_cast<const float4*>(invb + 32 * h + e4);
+          const int col = col0 + 32 * h + e4;
+          float s0 = v[e4] * ib.x, s1 = v[e4 + 1] * ib.y, s2 = v[e4 + 2] * ib.z, s3 = v[e4 + 3] * ib.w;
+          if (ragged) {
+            s0 = col < a.nB ? s0 : -INFINITY;
+            s1 = col + 1 < a.nB ? s1 : -INFINITY;
+            s2 = col + 2 < a.nB ? s2 : -INFINITY;
+            s3 = col + 3 < a.nB ? s3 : -INFINITY;
+          }
+          // the running maximum rarely moves once a few tiles are in: one comparison per four columns, and only then
+          // the search for the first column that holds the group's maximum (lowest position wins ties)
+          const float gm = fmaxf(fmaxf(s0, s1), fmaxf(s2, s3));
+          if (gm > bv) {
+            bv = gm;
+            bi = col + (s0 == gm ? 0 : (s1 == gm ? 1 : (s2 == gm ? 2 : 3)));
+          }
+        }
+      }
+      tc_fence_before();
+      __syncwarp();
+      if (lane == 0) mbar_arrive(bar_tempty(b));
+    }
+    float* part_s = reinterpret_cast<float*>(smem + oBPart);
+    int* part_b = reinterpret_cast<int*>(smem + oBPart + kBT * 2 * 4);
+    part_s[2 * row + half] = bv;
+    part_b[2 * row + half] = bi;
+    asm volatile("bar.sync 1, %0;" ::"n"(kBConsumers * 32) : "memory");
+    if (half == 0) {
+      const int ai = atile * kBT + row;
+      if (ai < a.nA && !failed) {
+        float s0 = part_s[2 * row], s1 = part_s[2 * row + 1];
+        int b0 = part_b[2 * row], b1 = part_b[2 * row + 1];
+        if (b0 == INT_MAX || (b1 != INT_MAX && s1 > s0)) {  // the other half holds higher columns: strict >
+          s0 = s1;
+          b0 = b1;
+        }
+        const bool has = b0 != INT_MAX;
+        const float cosv = has ? s0 * a.inv_a[(int64_t)lh * a.inv_stride + ai] + 0.f : -INFINITY;
+        a.edge_sim[(int64_t)lh * a.edge_stride + ai] = cosv;
+        a.edge_b[(int64_t)lh * a.edge_stride + ai] = has ? 2 * b0 + 1 : -1;
+      }
+    }
+  }
+  if (failed && lane == 0) atomicExch(a.status, 1);
+  tc_fence_before();
+  if (__syncthreads_or(failed)) {
+    // A wait gave up: copies and MMAs issued before it may still be in flight.  They finish on their own (nothing they
+    // depend on is missing), so give them a millisecond before shared and tensor memory go back.
+    for (int i = 0; i < 1000; ++i) __nanosleep(1000);
+    __syncthreads();
+  }
+  if (warp == 0) tmem_dealloc(tmem, 256);
+}
+
+// ---- after the ranking: output slots and member counts
+
+struct BsmMergeArgs {
+  const __nv_bfloat16* k_src;
+  const __nv_bfloat16* v_src;
+  const int32_t* deg_src;  // may be null: ones
+  __nv_bfloat16* k_dst;
+  __nv_bfloat16* v_dst;
+  int32_t* deg_dst;
+  float* logdeg_dst;       // may be null
+  int32_t* assign;         // may be null
+  int64_t assign_stride;
+  int64_t src_cap, dst_cap, lo;
+  int32_t nA, nB;
+  const int32_t* edge_b;   // [LH, edge_stride]
+  const uint8_t* sel;      // [LH, edge_stride]
+  int64_t edge_stride;
+  int32_t* selpre;         // [LH, edge_stride + 1] selected edges before A token a (exclusive prefix; last = total)
+  int32_t* cnt;            // [LH, cnt_stride]     scratch of the prepare kernel (member counts, then fill cursors)
+  int32_t* off;            // [LH, cnt_stride + 1] start of each B token's member list (exclusive prefix of the counts)
+  int32_t* list;           // [LH, edge_stride]    member A indices, grouped by B token (order inside a group: arbitrary)
+  int64_t cnt_stride;
+};
+
+constexpr int kPrepThreads = 1024;
+constexpr int kPrepRun = 16;  // A tokens per thread and sweep
+
+__global__ void __launch_bounds__(kPrepThreads) bsm_prepare_kernel(const BsmMergeArgs a) {
+  __shared__ int warp_tot[kPrepThreads / 32];
+  const int lh = blockIdx.x, tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  const uint8_t* sel = a.sel + (int64_t)lh * a.edge_stride;
+  const int32_t* eb = a.edge_b + (int64_t)lh * a.edge_stride;
+  int32_t* selpre = a.selpre + (int64_t)lh * (a.edge_stride + 1);
+  int32_t* cnt = a.cnt + (int64_t)lh * a.cnt_stride;
+  for (int b = tid; b < a.nB; b += kPrepThreads) cnt[b] = 0;
+  __syncthreads();
+  int run_total = 0;
+  for (int base = 0; base < a.nA; base += kPrepThreads * kPrepRun) {
+    const int first = base + tid * kPrepRun;
+    int local = 0;
+    uint32_t bits = 0;
+    for (int j = 0; j < kPrepRun; ++j) {
+      const int ai = first + j;
+      if (ai < a.nA && sel[ai]) {
+        bits |= 1u << j;
+        ++local;
+        atomicAdd(&cnt[eb[ai] >> 1], 1);
+      }
+    }
+    // exclusive prefix of `local` over the block
+    int inc = local;
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) {
+      const int y = __shfl_up_sync(0xffffffffu, inc, o);
+      if (lane >= o) inc += y;
+    }
+    if (lane == 31) warp_tot[warp] = inc;
+    __syncthreads();
+    const int wt = warp_tot[lane];
+    int winc = wt;
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) {
+      const int y = __shfl_up_sync(0xffffffffu, winc, o);
+      if (lane >= o) winc += y;
+    }
+    int before = run_total + __shfl_sync(0xffffffffu, winc - wt, warp) + inc - local;
+    run_total += __shfl_sync(0xffffffffu, winc, 31);
+    __syncthreads();
+    for (int j = 0; j < kPrepRun; ++j) {
+      const int ai = first + j;
+      if (ai < a.nA) selpre[ai] = before;
+      before += (bits >> j) & 1u;
+    }
+  }
+  if (tid == 0) selpre[a.nA] = run_total;
+  __syncthreads();  // the counts are complete
+
+  // member lists: offsets = exclusive prefix of the counts, then every selected A token takes a place in its target's list
+  int32_t* off = a.off + (int64_t)lh * (a.cnt_stride + 1);
+  int32_t* list = a.list + (int64_t)lh * a.edge_stride;
+  int off_total = 0;
+  for (int base = 0; base < a.nB; base += kPrepThreads * kPrepRun) {
+    const int first = base + tid * kPrepRun;
+    int local = 0;
+    for (int j = 0; j < kPrepRun; ++j) local += first + j < a.nB ? cnt[first + j] : 0;
+    int inc = local;
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) {
+      const int y = __shfl_up_sync(0xffffffffu, inc, o);
+      if (lane >= o) inc += y;
+    }
+    if (lane == 31) warp_tot[warp] = inc;
+    __syncthreads();
+    const int wt = warp_tot[lane];
+    int winc = wt;
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) {
+      const int y = __shfl_up_sync(0xffffffffu, winc, o);
+      if (lane >= o) winc += y;
+    }
+    int before = off_total + __shfl_sync(0xffffffffu, winc - wt, warp) + inc - local;
+    off_total += __shfl_sync(0xffffffffu, winc, 31);
+    __syncthreads();
+    for (int j = 0; j < kPrepRun; ++j) {
+      if (first + j < a.nB) {
+        off[first + j] = before;
+        before += cnt[first + j];
+      }
+    }
+  }
+  if (tid == 0) off[a.nB] = off_total;
+  __syncthreads();
+  for (int ai = tid; ai < a.nA; ai += kPrepThreads) {
+    if (sel[ai]) {
+      const int b = eb[ai] >> 1;
+      list[off[b] + atomicSub(&cnt[b], 1) - 1] = ai;
+    }
+  }
+}
+
+// Eq. 5, one warp per token of the middle region: a merged A token writes nothing, a survivor is copied to its slot,
+// a B token with members is replaced by the degree-weighted mean of itself and its members (found by scanning the
+// head's selected edges in position order, so the summation order is fixed).
+__global__ void __launch_bounds__(256) bsm_merge_kernel(const BsmMergeArgs a) {
+  const int lh = blockIdx.y, lane = threadIdx.x & 31;
+  const int64_t mid = (int64_t)a.nA + a.nB;
+  const int64_t o = (int64_t)blockIdx.x * 8 + (threadIdx.x >> 5);
+  if (o >= mid) return;
+  const uint8_t* sel = a.sel + (int64_t)lh * a.edge_stride;
+  const int32_t* eb = a.edge_b + (int64_t)lh * a.edge_stride;
+  const int32_t* selpre = a.selpre + (int64_t)lh * (a.edge_stride + 1);
+  const int64_t src0 = (int64_t)lh * a.src_cap + a.lo;
+  const int idx = (int)(o >> 1);
+  auto slot_b = [&](int b) { return (int64_t)(2 * b + 1) - selpre[b + 1]; };  // A tokens 0 .. b come before B token b
+  int64_t slot;
+  float4 fk, fv;
+  int n_new;
+  if (!(o & 1)) {  // A token
+    if (sel[idx]) {
+      if (a.assign && lane == 0) a.assign[(int64_t)lh * a.assign_stride + a.lo + o] = (int32_t)(a.lo + slot_b(eb[idx] >> 1));
+      return;
+    }
+    slot = o - selpre[idx];
+    fk = load4(a.k_src + (src0 + o) * kBD + lane * 4);
+    fv = load4(a.v_src + (src0 + o) * kBD + lane * 4);
+    n_new = a.deg_src ? a.deg_src[src0 + o] : 1;
+  } else {
+    slot = slot_b(idx);
+    fk = load4(a.k_src + (src0 + o) * kBD + lane * 4);
+    fv = load4(a.v_src + (src0 + o) * kBD + lane * 4);
+    n_new = a.deg_src ? a.deg_src[src0 + o] : 1;
+    const int32_t* off = a.off + (int64_t)lh * (a.cnt_stride + 1);
+    const int m = off[idx + 1] - off[idx];
+    if (m > 0) {
+      const float wb = (float)n_new;
+      fk.x *= wb; fk.y *= wb; fk.z *= wb; fk.w *= wb;
+      fv.x *= wb; fv.y *= wb; fv.z *= wb; fv.w *= wb;
+      auto add_member = [&](int am) {
+        const int64_t r = src0 + 2 * (int64_t)am;
+        const float4 mk = load4(a.k_src + r * kBD + lane * 4), mv = load4(a.v_src + r * kBD + lane * 4);
+        const int wa = a.deg_src ? a.deg_src[r] : 1;
+        const float w = (float)wa;
+        n_new += wa;
+        fk.x = fmaf(w, mk.x, fk.x); fk.y = fmaf(w, mk.y, fk.y); fk.z = fmaf(w, mk.z, fk.z); fk.w = fmaf(w, mk.w, fk.w);
+        fv.x = fmaf(w, mv.x, fv.x); fv.y = fmaf(w, mv.y, fv.y); fv.z = fmaf(w, mv.z, fv.z); fv.w = fmaf(w, mv.w, fv.w);
+      };
+      if (m <= 32) {
+        // the list is in arbitrary order: add the members in increasing position, so that the sum is reproducible
+        const int mine = lane < m ? a.list[(int64_t)lh * a.edge_stride + off[idx] + lane] : INT_MAX;
+        int rank = 0;
+        for (int i = 0; i < m; ++i) rank += __shfl_sync(0xffffffffu, mine, i) < mine ? 1 : 0;
+        for (int r = 0; r < m; ++r) {
+          const int src_lane = __ffs(__ballot_sync(0xffffffffu, lane < m && rank == r)) - 1;
+          add_member(__shfl_sync(0xffffffffu, mine, src_lane));
+        }
+      } else {
+        // a crowded target: scan the head's selected edges in position order
+        const int target = 2 * idx + 1;
+        int left = m;
+        for (int g0 = 0; g0 < a.nA && left > 0; g0 += 32) {
+          const int ai = g0 + lane;
+          unsigned members = __ballot_sync(0xffffffffu, ai < a.nA && sel[ai] && eb[ai] == target);
+          left -= __popc(members);
+          while (members) {
+            add_member(g0 + __ffs(members) - 1);
+            members &= members - 1;
+          }
+        }
+      }
+      const float inv = 1.0f / (float)n_new;
+      fk.x *= inv; fk.y *= inv; fk.z *= inv; fk.w *= inv;
+      fv.x *= inv; fv.y *= inv; fv.z *= inv; fv.w *= inv;
+    }
+  }
+  const int64_t d = (int64_t)lh * a.dst_cap + a.lo + slot;
+  store4(a.k_dst + d * kBD + lane * 4, fk);  // an untouched row round-trips bit for bit
+  store4(a.v_dst + d * kBD + lane * 4, fv);
+  if (lane == 0) {
+    a.deg_dst[d] = n_new;
+    if (a.logdeg_dst) a.logdeg_dst[d] = logf((float)n_new);
+    if (a.assign) a.assign[(int64_t)lh * a.assign_stride + a.lo + o] = (int32_t)(a.lo + slot);
+  }
+}
+
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*, const cuuint64_t*,
+                                  const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave, CUtensorMapSwizzle,
+                                  CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+EncodeTiledFn bsm_encode_fn() {
+  static EncodeTiledFn fn = nullptr;
+  if (!fn) {
+    void* p = nullptr;
+    cudaDriverEntryPointQueryResult q;
+    if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &q) == cudaSuccess && q == cudaDriverEntryPointSuccess)
+      fn = reinterpret_cast<EncodeTiledFn>(p);
+  }
+  return fn;
+}
+
+}  // namespace
+
+bool bsm_supported(int dtype, int D) { return dtype == 1 && D == 128 && bsm_encode_fn() != nullptr; }
+
+// workspace of one no-chunk round, in bytes, for LH slabs whose middle region has `mid` tokens
+size_t bsm_workspace_bytes(int64_t LH, int64_t mid) {
+  const int64_t nA = (mid + 1) / 2, inv_stride = (nA + 127) / 128 * 128;
+  return (size_t)LH * (2 * inv_stride * 4 + (nA + 1) * 4 + inv_stride * 4 + (inv_stride + 1) * 4 + nA * 4) + 1024;
+}
+
+// Matching, ranking inputs and merge of one no-chunk round.  edge_sim / edge_b / sel: [LH, nA] arrays of the workspace;
+// `scratch`: bsm_workspace_bytes.  launch_select runs between match and merge (called by the driver).
+cudaError_t launch_bsm_match(const RoundArgs& r, void* scratch, cudaStream_t st) {
+  const int64_t mid = r.hi - r.lo;
+  BsmArgs a{};
+  a.k_src = static_cast<const __nv_bfloat16*>(r.k_src);
+  a.src_cap = r.src_cap;
+  a.lo = r.lo;
+  a.nA = (int32_t)((mid + 1) / 2);
+  a.nB = (int32_t)(mid / 2);
+  a.inv_stride = ((int64_t)a.nA + 127) / 128 * 128;
+  a.inv_a = static_cast<float*>(scratch);
+  a.inv_b = a.inv_a + (int64_t)r.LH * a.inv_stride;
+  a.edge_sim = r.edge_sim;
+  a.edge_b = r.edge_b;
+  a.edge_stride = r.edge_stride;
+  a.status = r.status;
+  bsm_norm_kernel<<<dim3((unsigned)((mid + 7) / 8), (unsigned)r.LH), 256, 0, st>>>(a);
+  cudaError_t e = cudaGetLastError();
+  if (e != cudaSuccess) return e;
+  // (column, parity, token pair, slab) view of the middle region; out-of-range pairs read as zeros
+  CUtensorMap tm;
+  const cuuint64_t dims[4] = {128, 2, (cuuint64_t)a.nA, (cuuint64_t)r.LH};
+  const cuuint64_t strides[3] = {256, 512, (cuuint64_t)r.src_cap * 256};
+  const cuuint32_t box[4] = {64, 1, 128, 1}, es[4] = {1, 1, 1, 1};
+  void* addr = const_cast<unsigned char*>(reinterpret_cast<const unsigned char*>(r.k_src) + r.lo * 256);
+  if (bsm_encode_fn()(&tm, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 4, addr, dims, strides, box, es, CU_TENSOR_MAP_INTERLEAVE_NONE,
+                      CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
+    return cudaErrorInvalidValue;
+  const size_t smem = kBBytes + 1024;
+  if ((e = cudaFuncSetAttribute(bsm_match_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem)) != cudaSuccess) return e;
+  bsm_match_kernel<<<dim3((unsigned)((a.nA + kBT - 1) / kBT), (unsigned)r.LH), kBThreads, smem, st>>>(tm, a);
+  return cudaGetLastError();
+}
+
+cudaError_t launch_bsm_merge(const RoundArgs& r, void* scratch, cudaStream_t st) {
+  const int64_t mid = r.hi - r.lo;
+  BsmMergeArgs a{};
+  a.k_src = static_cast<const __nv_bfloat16*>(r.k_src);
+  a.v_src = static_cast<const __nv_bfloat16*>(r.v_src);
+  a.deg_src = r.deg_src;
+  a.k_dst = static_cast<__nv_bfloat16*>(r.k_dst);
+  a.v_dst = static_cast<__nv_bfloat16*>(r.v_dst);
+  a.deg_dst = r.deg_dst;
+  a.logdeg_dst = r.logdeg_dst;
+  a.assign = r.assign;
+  a.assign_stride = r.assign_stride;
+  a.src_cap = r.src_cap;
+  a.dst_cap = r.dst_cap;
+  a.lo = r.lo;
+  a.nA = (int32_t)((mid + 1) / 2);
+  a.nB = (int32_t)(mid / 2);
+  a.edge_b = r.edge_b;
+  a.sel = r.sel;
+  a.edge_stride = r.edge_stride;
+  const int64_t inv_stride = ((int64_t)a.nA + 127) / 128 * 128;
+  a.selpre = reinterpret_cast<int32_t*>(static_cast<float*>(scratch) + 2 * (int64_t)r.LH * inv_stride);
+  a.cnt = a.selpre + (int64_t)r.LH * (a.nA + 1);
+  a.cnt_stride = inv_stride;
+  a.off = a.cnt + (int64_t)r.LH * inv_stride;
+  a.list = a.off + (int64_t)r.LH * (inv_stride + 1);
+  bsm_prepare_kernel<<<(unsigned)r.LH, kPrepThreads, 0, st>>>(a);
+  cudaError_t e = cudaGetLastError();
+  if (e != cudaSuccess) return e;
+  bsm_merge_kernel<<<dim3((unsigned)((mid + 7) / 8), (unsigned)r.LH), 256, 0, st>>>(a);
+  return cudaGetLastError();
+}
+
+}  // namespace ckv

@@ -118,6 +118,10 @@ bool round_fast_supported(const RoundArgs& a, int dtype, int D);
 cudaError_t launch_round_fast(const RoundArgs& a, int64_t n_full, cudaStream_t st);
 bool round_umma_supported(const RoundArgs& a, int dtype, int D);
 cudaError_t launch_round_umma(const RoundArgs& a, int64_t n_full, cudaStream_t st);
+bool bsm_supported(int dtype, int D);
+size_t bsm_workspace_bytes(int64_t LH, int64_t mid);
+cudaError_t launch_bsm_match(const RoundArgs& a, void* scratch, cudaStream_t st);  // a.lo, a.hi: the middle region
+cudaError_t launch_bsm_merge(const RoundArgs& a, void* scratch, cudaStream_t st);
 bool round_tile_supported(const RoundArgs& a, int dtype, int D);
 cudaError_t launch_round_tile(const RoundArgs& a, cudaStream_t st);
 

@@ -78,7 +78,7 @@ def test_plan_reports_no_progress_and_bad_arguments(b):
     with pytest.raises(b.CkvError) as e:
         b.compress_plan(1000, b.Params(chunk=64, n_sink=0, n_recent=0, r_init=0.0, r_decay=0.0, r_min=0.0, budget=10))
     assert e.value.status == 5
-    for bad in (b.Params(chunk=63), b.Params(chunk=0), b.Params(chunk=64, n_sink=-1), b.Params(chunk=64, r_init=1.5),
+    for bad in (b.Params(chunk=63), b.Params(chunk=-2), b.Params(chunk=64, n_sink=-1), b.Params(chunk=64, r_init=1.5),
                 b.Params(chunk=64, select=7)):
         with pytest.raises(b.CkvError) as e:
             b.compress_plan(1000, bad)
@@ -86,6 +86,16 @@ def test_plan_reports_no_progress_and_bad_arguments(b):
     with pytest.raises(b.CkvError) as e:
         b.compress_plan(1000, b.Params(chunk=512))
     assert e.value.status == 6
+
+
+def test_plan_without_chunks_matches_the_oracle_lengths(b):
+    """chunk = 0 (no chunking): one chunk spans the middle region; lengths after every round as the oracle counts them."""
+    for s, kw in ((1000, dict(n_sink=0, n_recent=0, r_init=1.0, r_decay=0.0, r_min=1.0, n_rounds_max=2)),
+                  (777, dict(n_sink=16, n_recent=64, r_init=0.8, r_decay=0.2, r_min=0.2, n_rounds_max=16, budget=200))):
+        out_len, rounds, _ = b.compress_plan(s, b.Params(chunk=0, **kw))
+        po = O.Params(chunk=0, **kw)
+        lens = oracle_lengths(s, po)
+        assert rounds == len(lens) and out_len == lens[-1]
 
 
 def test_argument_checks_happen_before_any_launch(b):

@@ -285,3 +285,30 @@ def test_status_codes_on_device_buffers():
     with pytest.raises(b.CkvError) as e:
         b.compress_prefill(src, dst, pb, ws)
     assert e.value.status == 5
+
+
+@pytest.mark.parametrize("s,sink,recent,r", [(300, 0, 0, 1.0), (1001, 16, 64, 0.5), (2500, 3, 0, 0.8), (130, 0, 1, 0.3), (4096, 0, 0, 1.0)])
+def test_no_chunking_single_round(s, sink, recent, r):
+    """chunk = 0: every A token against every B token of its head (plain Bipartite Soft Matching), tensor-core matching."""
+    b = B()
+    single_round_case(2, 2, s, "bf16", one_round(b, 0, r, b.SELECT_GLOBAL, sink, recent), seed=900 + s, deg_max=4)
+
+
+def test_no_chunking_paper_schedule():
+    b = B()
+    s = 3000
+    p = b.Params(chunk=0, n_sink=16, n_recent=64, n_rounds_max=16, r_init=0.8, r_decay=0.2, r_min=0.2, select=b.SELECT_GLOBAL, budget=s // 4)
+    st = multi_round_case(1, 2, s, "bf16", p, seed=37)
+    assert st["rounds"] >= 4
+
+
+def test_no_chunking_is_bf16_only():
+    b = B()
+    K, V, _ = make_inputs(1, 1, 64, "f32", seed=2)
+    p = one_round(b, 0, 1.0, b.SELECT_GLOBAL)
+    src = b.Cache(K, V, None, None, 64)
+    dst = b.Cache.empty(1, 1, 64, 128, K.dtype, DEV)
+    ws = torch.empty(max(b.workspace_bytes(src, p), 1 << 20), dtype=torch.uint8, device=DEV)
+    with pytest.raises(b.CkvError) as e:
+        b.compress_prefill(src, dst, p, ws)
+    assert e.value.status == 6
