@@ -3,14 +3,17 @@
 // multiply-adds per head (Table 1) -- a dense contraction, compute-bound, so it runs as a tensor-core GEMM with the
 // argmax fused into the epilogue:
 //   bsm_norm_kernel     inverse key norms of the A and B tokens
-//   bsm_match_kernel    one CTA per 128 A tokens walks all B tokens in tiles of 128: a TMA warp streams B tiles
-//                       (de-interleaving tensor map, 128-byte swizzle) through a 4-stage ring, an MMA warp issues
-//                       tcgen05.mma (128 x 128 x 128 per tile) into one of two tensor-memory accumulators, eight
-//                       consumer warps read the other accumulator (tcgen05.ld), scale by 1 / |b| and keep a running
-//                       row argmax (lowest B position on ties); the edge (cosine, target) is written at the end
+//   bsm_match_kernel    one CTA per 256 A tokens (two row blocks of 128) walks all B tokens in steps of 256: a TMA warp
+//                       streams B tiles (de-interleaving tensor map, 128-byte swizzle) through a ring of two steps, an MMA
+//                       warp issues tcgen05.mma 128 x 256 x 16 (the widest shape of one CTA: the least shared-memory
+//                       operand traffic per flop) for row block 0, then row block 1, each into its own 256 columns of
+//                       tensor memory; sixteen consumer warps copy an accumulator to registers (tcgen05.ld), hand it back
+//                       to the tensor core at once, scale by 1 / |b| and keep a running row argmax (lowest B position on
+//                       ties); the edge (cosine, target) is written at the end
 //   select_kernel       the M best edges of the head (shared with the chunked path)
 //   bsm_prepare_kernel  prefix counts of the selected edges (output slots) and the number of members per B token
-//   bsm_merge_kernel    one warp per surviving token: Eq. 5 over its members, found by scanning the head's edges
+//   bsm_prepare_kernel  also lists the members of every B token
+//   bsm_merge_kernel    one warp per surviving token: Eq. 5 over its members, taken from the prepared lists
 // bf16, head_dim 128.  Waits are bounded; a role whose wait gives up sets the status word and stops; the others follow.
 #include <cuda.h>
 
@@ -30,26 +33,32 @@ namespace {
 using namespace ptx;
 
 constexpr int kBD = 128;          // head_dim
-constexpr int kBT = 128;          // tile: A tokens per CTA, B tokens per step
-constexpr int kBHalf = kBT * 128; // one swizzled operand tile: 128 rows x 64 columns
-constexpr int kBStages = 5;        // B tiles in flight; a stage is free again as soon as the tensor core has read it
-constexpr int kBInvSlots = 8;      // 1/|b| slices: consumers are at most three tiles behind the fetch of a slot's next use
-constexpr int kBConsumers = 8;    // warps
+constexpr int kBT = 128;          // rows of one MMA, rows of one TMA box
+constexpr int kBM = 2 * kBT;      // A tokens per CTA: two row blocks, each with its own accumulator
+constexpr int kBN = 2 * kBT;      // B tokens per step (columns of one MMA)
+constexpr int kBHalf = kBT * 128; // one swizzled box: 128 rows x 64 columns
+constexpr int kBSteps = 2;        // steps of B in flight; a step's tiles are free again once the tensor core has read them
+constexpr int kBInvSlots = 4;     // 1/|b| slices of a step (1 KiB each)
+constexpr int kBConsumers = 16;   // warps: (quarter of the tensor-memory lanes) x (quarter of the step's columns)
+constexpr int kBTmemCols = 2 * kBN;
 constexpr int kBThreads = (kBConsumers + 2) * 32;
-// shared memory (1024-byte aligned base): A tile | B ring | 1/|b| ring | barriers | partial argmaxes | tmem address
+// Shared memory (1024-byte aligned base): A blocks | B ring | 1/|b| ring | barriers | partial argmaxes | tmem address.
+// The B ring is split by column half (dims 0..63 | 64..127), each part holding the 128-row boxes of all steps in order, so
+// that the 256 rows of a step are contiguous for the tensor core.
 constexpr int oBA = 0;
-constexpr int oBB = 2 * kBHalf;
-constexpr int oBInv = oBB + kBStages * 2 * kBHalf;
-constexpr int oBBar = oBInv + kBInvSlots * 512;
+constexpr int oBB = 4 * kBHalf;
+constexpr int kBPart = kBSteps * 2 * kBHalf;  // bytes of one column half of the ring
+constexpr int oBInv = oBB + 2 * kBPart;
+constexpr int oBBar = oBInv + kBInvSlots * kBN * 4;
 constexpr int oBPart = oBBar + 256;
-constexpr int oBTmem = oBPart + kBT * 2 * 8;
+constexpr int oBTmem = oBPart + kBM * 4 * 8;
 constexpr int kBBytes = oBTmem + 16;
 
 struct BsmArgs {
   const __nv_bfloat16* k_src;
   int64_t src_cap, lo;
   int32_t nA, nB;         // A and B tokens of the middle region
-  int64_t inv_stride;     // floats per head of inv_a / inv_b (multiple of 128)
+  int64_t inv_stride;     // floats per head of inv_a / inv_b (multiple of 256)
   float* inv_a;
   float* inv_b;
   float* edge_sim;        // [LH, edge_stride]
@@ -60,8 +69,8 @@ struct BsmArgs {
 
 __device__ __forceinline__ void mbar_arrive(uint32_t bar) { asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory"); }
 
-__host__ __device__ constexpr uint32_t bsm_idesc() {  // bf16 x bf16 -> fp32, both K-major, M = 128, N = 128
-  return (1u << 4) | (1u << 7) | (1u << 10) | ((128u >> 3) << 17) | ((128u >> 4) << 24);
+__host__ __device__ constexpr uint32_t bsm_idesc() {  // bf16 x bf16 -> fp32, both K-major, M = 128, N = 256
+  return (1u << 4) | (1u << 7) | (1u << 10) | (((uint32_t)kBN >> 3) << 17) | ((128u >> 4) << 24);
 }
 
 // inverse norms: one warp per token of the middle region
@@ -75,34 +84,108 @@ __global__ void __launch_bounds__(256) bsm_norm_kernel(const BsmArgs a) {
   if (lane == 0) ((o & 1) ? a.inv_b : a.inv_a)[(int64_t)lh * a.inv_stride + (o >> 1)] = ss > 0.f ? rsqrtf(ss) : 0.f;
 }
 
-__global__ void __launch_bounds__(kBThreads, 1) bsm_match_kernel(const __grid_constant__ CUtensorMap tm_k, const BsmArgs a) {
+// tcgen05.ld of 32 columns without the wait, and the wait with the registers as operands (so that no use moves above it)
+__device__ __forceinline__ void tmem_ld32_issue(uint32_t taddr, uint32_t (&r)[32]) {
+  asm volatile(
+      "tcgen05.ld.sync.aligned.32x32b.x32.b32 {%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15,%16,%17,%18,%19,%20,%21,%22,%23,"
+      "%24,%25,%26,%27,%28,%29,%30,%31}, [%32];"
+      : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]), "=r"(r[8]), "=r"(r[9]),
+        "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15]), "=r"(r[16]), "=r"(r[17]), "=r"(r[18]),
+        "=r"(r[19]), "=r"(r[20]), "=r"(r[21]), "=r"(r[22]), "=r"(r[23]), "=r"(r[24]), "=r"(r[25]), "=r"(r[26]), "=r"(r[27]),
+        "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
+      : "r"(taddr)
+      : "memory");
+}
+__device__ __forceinline__ void tmem_ld_wait(uint32_t (&r)[32]) {
+  asm volatile("tcgen05.wait::ld.sync.aligned;"
+               : "+r"(r[0]), "+r"(r[1]), "+r"(r[2]), "+r"(r[3]), "+r"(r[4]), "+r"(r[5]), "+r"(r[6]), "+r"(r[7]), "+r"(r[8]), "+r"(r[9]),
+                 "+r"(r[10]), "+r"(r[11]), "+r"(r[12]), "+r"(r[13]), "+r"(r[14]), "+r"(r[15]), "+r"(r[16]), "+r"(r[17]), "+r"(r[18]),
+                 "+r"(r[19]), "+r"(r[20]), "+r"(r[21]), "+r"(r[22]), "+r"(r[23]), "+r"(r[24]), "+r"(r[25]), "+r"(r[26]), "+r"(r[27]),
+                 "+r"(r[28]), "+r"(r[29]), "+r"(r[30]), "+r"(r[31])
+               :
+               : "memory");
+}
+// two fp32 products in one instruction (round to nearest even, as two scalar multiplies)
+__device__ __forceinline__ void mul2(float& x, float& y, uint32_t a0, uint32_t a1, uint64_t b) {
+  uint64_t a, d;
+  asm("mov.b64 %0, {%1, %2};" : "=l"(a) : "r"(a0), "r"(a1));
+  asm("mul.rn.f32x2 %0, %1, %2;" : "=l"(d) : "l"(a), "l"(b));
+  uint32_t lo, hi;
+  asm("mov.b64 {%0, %1}, %2;" : "=r"(lo), "=r"(hi) : "l"(d));
+  x = __uint_as_float(lo);
+  y = __uint_as_float(hi);
+}
+__device__ __forceinline__ float max3(float a, float b, float c) {
+  float d;
+  asm("max.f32 %0, %1, %2, %3;" : "=f"(d) : "f"(a), "f"(b), "f"(c));
+  return d;
+}
+
+// Running row argmax over 64 accumulator columns of one tensor-memory lane per thread: dot products scaled by 1 / |b|.
+// The running maximum rarely moves once a few tiles are in, so the common path is one maximum per sixteen columns and
+// one warp vote; only when some lane has a new maximum does the warp look for its column (the lowest one that holds the
+// maximum: the lowest B position wins ties; an equal value later on never replaces the running one).
+template <bool RAGGED>
+__device__ __forceinline__ void argmax_64(const uint32_t (&r)[2][32], const float* invb, int col0, int nB, float& bv, int& bi) {
+#pragma unroll
+  for (int h = 0; h < 2; ++h) {
+#pragma unroll
+    for (int g = 0; g < 32; g += 16) {
+      float sv[16];
+#pragma unroll
+      for (int e4 = 0; e4 < 16; e4 += 4) {
+        const ulonglong2 ib = *reinterpret_cast<const ulonglong2*>(invb + 32 * h + g + e4);
+        mul2(sv[e4], sv[e4 + 1], r[h][g + e4], r[h][g + e4 + 1], ib.x);
+        mul2(sv[e4 + 2], sv[e4 + 3], r[h][g + e4 + 2], r[h][g + e4 + 3], ib.y);
+      }
+      const int col = col0 + 32 * h + g;
+      if (RAGGED) {
+#pragma unroll
+        for (int e = 0; e < 16; ++e) sv[e] = col + e < nB ? sv[e] : -INFINITY;
+      }
+      const float gm = max3(max3(max3(sv[0], sv[1], sv[2]), max3(sv[3], sv[4], sv[5]), max3(sv[6], sv[7], sv[8])),
+                            max3(max3(sv[9], sv[10], sv[11]), max3(sv[12], sv[13], sv[14]), sv[15]), -INFINITY);
+      if (__any_sync(0xffffffffu, gm > bv)) {
+        int idx = 15;
+#pragma unroll
+        for (int e = 14; e >= 0; --e) idx = sv[e] == gm ? e : idx;
+        if (gm > bv) {
+          bv = gm;
+          bi = col + idx;
+        }
+      }
+    }
+  }
+}
+
+__global__ void __launch_bounds__(kBThreads, 1) bsm_match_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__ CUtensorMap tm_b,
+                                                                 const BsmArgs a) {
   extern __shared__ unsigned char smem_raw[];
   unsigned char* smem = reinterpret_cast<unsigned char*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
   const uint32_t s_base = smem_u32(smem);
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const int lh = blockIdx.y, atile = blockIdx.x;
-  const int n_tiles = (a.nB + kBT - 1) / kBT;
-  auto bar_full = [&](int s) { return s_base + oBBar + 8u * s; };
-  auto bar_empty = [&](int s) { return s_base + oBBar + 8u * (kBStages + s); };
-  auto bar_tfull = [&](int b) { return s_base + oBBar + 8u * (2 * kBStages + b); };
-  auto bar_tempty = [&](int b) { return s_base + oBBar + 8u * (2 * kBStages + 2 + b); };
-  const uint32_t bar_a = s_base + oBBar + 8u * (2 * kBStages + 4);
-  auto bar_inv = [&](int i) { return s_base + oBBar + 8u * (2 * kBStages + 5 + i); };
+  const int n_steps = (a.nB + kBN - 1) / kBN;
+  // barriers: full[step slot][row half of the step] | empty[step slot] | tfull[row block] | tempty[row block] | a | inv[slot]
+  auto bar_full = [&](int i) { return s_base + oBBar + 8u * i; };
+  auto bar_empty = [&](int i) { return s_base + oBBar + 8u * (2 * kBSteps + i); };
+  auto bar_tfull = [&](int m) { return s_base + oBBar + 8u * (3 * kBSteps + m); };
+  auto bar_tempty = [&](int m) { return s_base + oBBar + 8u * (3 * kBSteps + 2 + m); };
+  const uint32_t bar_a = s_base + oBBar + 8u * (3 * kBSteps + 4);
+  auto bar_inv = [&](int i) { return s_base + oBBar + 8u * (3 * kBSteps + 5 + i); };
 
   if (tid == 0) {
-    for (int s = 0; s < kBStages; ++s) {
-      mbar_init(bar_full(s), 1);
-      mbar_init(bar_empty(s), 1);  // the MMA's commit
-    }
-    for (int b = 0; b < 2; ++b) {
-      mbar_init(bar_tfull(b), 1);
-      mbar_init(bar_tempty(b), kBConsumers);
+    for (int i = 0; i < 2 * kBSteps; ++i) mbar_init(bar_full(i), 1);
+    for (int i = 0; i < kBSteps; ++i) mbar_init(bar_empty(i), 1);  // the MMA's commit
+    for (int m = 0; m < 2; ++m) {
+      mbar_init(bar_tfull(m), 1);
+      mbar_init(bar_tempty(m), kBConsumers);
     }
     mbar_init(bar_a, 1);
     for (int i = 0; i < kBInvSlots; ++i) mbar_init(bar_inv(i), 1);
     mbar_init_fence();
   }
-  if (warp == 0) tmem_alloc(s_base + oBTmem, 256);
+  if (warp == 0) tmem_alloc(s_base + oBTmem, kBTmemCols);
   tc_fence_before();
   __syncthreads();
   tc_fence_after();
@@ -110,113 +193,129 @@ __global__ void __launch_bounds__(kBThreads, 1) bsm_match_kernel(const __grid_co
   bool failed = false;
 
   if (warp == kBConsumers) {
-    // ------------------------------------------------------------------ TMA warp: the A tile once, then the B tiles
+    // ------------------------------------------------------------------ TMA warp: the A blocks once, then the B steps
     if (lane == 0) {
-      mbar_arrive_expect_tx(bar_a, 2 * kBHalf);
-      tma_load_4d(s_base + oBA, &tm_k, 0, 0, atile * kBT, lh, bar_a);
-      tma_load_4d(s_base + oBA + kBHalf, &tm_k, 64, 0, atile * kBT, lh, bar_a);
-      for (int j = 0; j < n_tiles && !failed; ++j) {
-        const int s = j % kBStages;
-        if (!mbar_wait(bar_empty(s), (uint32_t)(((j / kBStages) & 1) ^ 1))) {
+      mbar_arrive_expect_tx(bar_a, 4 * kBHalf);
+      for (int m = 0; m < 2; ++m) {  // row block m: tokens atile * 256 + 128 m .. + 127 (zero-filled past the end)
+        tma_load_4d(s_base + oBA + (uint32_t)m * 2 * kBHalf, &tm_a, 0, 0, atile * kBM + m * kBT, lh, bar_a);
+        tma_load_4d(s_base + oBA + (uint32_t)m * 2 * kBHalf + kBHalf, &tm_a, 64, 0, atile * kBM + m * kBT, lh, bar_a);
+      }
+      for (int t = 0; t < n_steps && !failed; ++t) {
+        const int slot = t % kBSteps;
+        if (!mbar_wait(bar_empty(slot), (uint32_t)(((t / kBSteps) & 1) ^ 1))) {
           failed = true;
           break;
         }
-        const uint32_t dst = s_base + oBB + (uint32_t)s * 2 * kBHalf;
-        mbar_arrive_expect_tx(bar_full(s), 2 * kBHalf);
-        tma_load_4d(dst, &tm_k, 0, 1, j * kBT, lh, bar_full(s));
-        tma_load_4d(dst + kBHalf, &tm_k, 64, 1, j * kBT, lh, bar_full(s));
-        // The slice slot of tile j was last read for tile j - 8; this fetch runs after the MMA of tile j - 5 completed, which
-        // was issued after the consumers released the accumulator of tile j - 7: they are done with tile j - 8.
-        mbar_arrive_expect_tx(bar_inv(j % kBInvSlots), 512);
-        bulk_load(s_base + oBInv + (uint32_t)(j % kBInvSlots) * 512, a.inv_b + (int64_t)lh * a.inv_stride + (int64_t)j * kBT, 512,
-                  bar_inv(j % kBInvSlots));
+        for (int hf = 0; hf < 2; ++hf) {  // B tokens t * 256 + 128 hf .. + 127 (zero-filled past the end)
+          const uint32_t dst = s_base + oBB + (uint32_t)(2 * slot + hf) * kBHalf;
+          mbar_arrive_expect_tx(bar_full(2 * slot + hf), 2 * kBHalf);
+          tma_load_4d(dst, &tm_b, 0, 0, t * kBN + hf * kBT, lh, bar_full(2 * slot + hf));
+          tma_load_4d(dst + kBPart, &tm_b, 64, 0, t * kBN + hf * kBT, lh, bar_full(2 * slot + hf));
+        }
+        // The slice slot of step t was last read for step t - 4; this fetch runs after the MMAs of step t - 2 completed,
+        // which were issued after every consumer warp had copied the accumulators of step t - 3 to registers, and a warp
+        // does that only after its argmax over step t - 4.
+        const int is = t % kBInvSlots;
+        mbar_arrive_expect_tx(bar_inv(is), kBN * 4);
+        bulk_load(s_base + oBInv + (uint32_t)is * kBN * 4, a.inv_b + (int64_t)lh * a.inv_stride + (int64_t)t * kBN, kBN * 4, bar_inv(is));
       }
     }
   } else if (warp == kBConsumers + 1) {
-    // ------------------------------------------------------------------ MMA warp: S tile = A B^T into accumulator j & 1
+    // ------------------------------------------------------------------ MMA warp: S = A_m B^T into the accumulator of row block m
     if (lane == 0) {
       failed = !mbar_wait(bar_a, 0);
-      for (int j = 0; j < n_tiles && !failed; ++j) {
-        const int s = j % kBStages, b = j & 1;
-        if (!mbar_wait(bar_full(s), (uint32_t)((j / kBStages) & 1)) || !mbar_wait(bar_tempty(b), (uint32_t)(((j >> 1) & 1) ^ 1))) {
+      for (int t = 0; t < n_steps && !failed; ++t) {
+        const int slot = t % kBSteps;
+        const uint32_t par = (uint32_t)((t / kBSteps) & 1);
+        if (!mbar_wait(bar_full(2 * slot), par) || !mbar_wait(bar_full(2 * slot + 1), par)) {
+          failed = true;
+          break;
+        }
+        const uint32_t bt = s_base + oBB + (uint32_t)(2 * slot) * kBHalf;
+        for (int m = 0; m < 2; ++m) {
+          if (!mbar_wait(bar_tempty(m), (uint32_t)((t & 1) ^ 1))) {  // the consumers are done with this block's last step
+            failed = true;
+            break;
+          }
+          tc_fence_after();
+#pragma unroll
+          for (int ks = 0; ks < 8; ++ks) {
+            const uint32_t off = (uint32_t)(ks & 3) * 32u;
+            umma_bf16(tmem + (uint32_t)m * kBN, umma_desc_sw128(s_base + oBA + (uint32_t)m * 2 * kBHalf + (uint32_t)(ks >> 2) * kBHalf + off, 16, 1024),
+                      umma_desc_sw128(bt + (uint32_t)(ks >> 2) * kBPart + off, 16, 1024), bsm_idesc(), ks ? 1u : 0u);
+          }
+          umma_commit(bar_tfull(m));  // this block's accumulator is complete
+        }
+        if (!failed) umma_commit(bar_empty(slot));  // the tensor core has read the step's B tiles
+      }
+    }
+  } else {
+    // ------------------------------------------------------------------ consumers: running row argmaxes
+    // Every warp serves both row blocks: tensor-memory lanes 32 q .. + 31, columns 64 cq .. + 63 of every step.  It copies
+    // its part of an accumulator to registers and hands the accumulator back at once, so that the tensor core refills
+    // it while the argmax runs on the registers.
+    const int q = warp & 3, cq = warp >> 2;
+    float bv[2] = {-INFINITY, -INFINITY};
+    int bi[2] = {INT_MAX, INT_MAX};
+    for (int t = 0; t < n_steps && !failed; ++t) {
+      const int is = t % kBInvSlots;
+      if (!mbar_wait(bar_inv(is), (uint32_t)((t / kBInvSlots) & 1))) {
+        failed = true;
+        break;
+      }
+      const float* invb = reinterpret_cast<const float*>(smem + oBInv + is * kBN * 4) + 64 * cq;
+      const int col0 = t * kBN + 64 * cq;
+#pragma unroll
+      for (int m = 0; m < 2; ++m) {
+        if (!mbar_wait(bar_tfull(m), (uint32_t)(t & 1))) {
           failed = true;
           break;
         }
         tc_fence_after();
-        const uint32_t bt = s_base + oBB + (uint32_t)s * 2 * kBHalf;
-#pragma unroll
-        for (int ks = 0; ks < 8; ++ks) {
-          const uint32_t off = (uint32_t)(ks >> 2) * kBHalf + (uint32_t)(ks & 3) * 32u;
-          umma_bf16(tmem + (uint32_t)b * kBT, umma_desc_sw128(s_base + oBA + off, 16, 1024), umma_desc_sw128(bt + off, 16, 1024),
-                    bsm_idesc(), ks ? 1u : 0u);
-        }
-        umma_commit(bar_empty(s));  // the tensor core has read the B tile
-        umma_commit(bar_tfull(b));  // the accumulator is complete
-      }
-    }
-  } else {
-    // ------------------------------------------------------------------ consumers: running row argmax
-    const int q = warp & 3, half = warp >> 2;  // tensor-memory lanes 32 q .. + 31; columns 64 half .. + 63 of every tile
-    const int row = 32 * q + lane;
-    float bv = -INFINITY;
-    int bi = INT_MAX;
-    for (int j = 0; j < n_tiles && !failed; ++j) {
-      const int b = j & 1;
-      // (the consumers never look at the B ring: its stages may be refilled while they are still on this tile)
-      if (!mbar_wait(bar_inv(j % kBInvSlots), (uint32_t)((j / kBInvSlots) & 1)) || !mbar_wait(bar_tfull(b), (uint32_t)((j >> 1) & 1))) {
-        failed = true;
-        break;
-      }
-      tc_fence_after();
-      const float* invb = reinterpret_cast<const float*>(smem + oBInv + (j % kBInvSlots) * 512) + 64 * half;
-      const int col0 = j * kBT + 64 * half;
-      const bool ragged = col0 + 64 > a.nB;  // only the last tile can hold columns that are not B tokens
-#pragma unroll
-      for (int h = 0; h < 2; ++h) {
-        float v[32];
-        tmem_ld32(tmem + ((uint32_t)(32 * q) << 16) + (uint32_t)(b * kBT + 64 * half + 32 * h), v);
-#pragma unroll
-        for (int e4 = 0; e4 < 32; e4 += 4) {
-          const float4 ib = *reinterpret_cast<const float4*>(invb + 32 * h + e4);
-          const int col = col0 + 32 * h + e4;
-          float s0 = v[e4] * ib.x, s1 = v[e4 + 1] * ib.y, s2 = v[e4 + 2] * ib.z, s3 = v[e4 + 3] * ib.w;
-          if (ragged) {
-            s0 = col < a.nB ? s0 : -INFINITY;
-            s1 = col + 1 < a.nB ? s1 : -INFINITY;
-            s2 = col + 2 < a.nB ? s2 : -INFINITY;
-            s3 = col + 3 < a.nB ? s3 : -INFINITY;
-          }
-          // the running maximum rarely moves once a few tiles are in: one comparison per four columns, and only then
-          // the search for the first column that holds the group's maximum (lowest position wins ties)
-          const float gm = fmaxf(fmaxf(s0, s1), fmaxf(s2, s3));
-          if (gm > bv) {
-            bv = gm;
-            bi = col + (s0 == gm ? 0 : (s1 == gm ? 1 : (s2 == gm ? 2 : 3)));
-          }
+        uint32_t r[2][32];
+        const uint32_t tcol = tmem + ((uint32_t)(32 * q) << 16) + (uint32_t)(kBN * m + 64 * cq);
+        tmem_ld32_issue(tcol, r[0]);
+        tmem_ld32_issue(tcol + 32u, r[1]);
+        tmem_ld_wait(r[0]);
+        tmem_ld_wait(r[1]);
+        tc_fence_before();
+        __syncwarp();
+        if (lane == 0) mbar_arrive(bar_tempty(m));
+        if (col0 + 64 <= a.nB) {  // only the last step can hold columns that are not B tokens
+          argmax_64<false>(r, invb, col0, a.nB, bv[m], bi[m]);
+        } else {
+          argmax_64<true>(r, invb, col0, a.nB, bv[m], bi[m]);
         }
       }
-      tc_fence_before();
-      __syncwarp();
-      if (lane == 0) mbar_arrive(bar_tempty(b));
     }
     float* part_s = reinterpret_cast<float*>(smem + oBPart);
-    int* part_b = reinterpret_cast<int*>(smem + oBPart + kBT * 2 * 4);
-    part_s[2 * row + half] = bv;
-    part_b[2 * row + half] = bi;
+    int* part_b = reinterpret_cast<int*>(smem + oBPart + kBM * 4 * 4);
+#pragma unroll
+    for (int m = 0; m < 2; ++m) {
+      part_s[4 * (kBT * m + 32 * q + lane) + cq] = bv[m];
+      part_b[4 * (kBT * m + 32 * q + lane) + cq] = bi[m];
+    }
     asm volatile("bar.sync 1, %0;" ::"n"(kBConsumers * 32) : "memory");
-    if (half == 0) {
-      const int ai = atile * kBT + row;
+    if (tid < kBM) {
+      const int row = tid, ai = atile * kBM + row;
       if (ai < a.nA && !failed) {
-        float s0 = part_s[2 * row], s1 = part_s[2 * row + 1];
-        int b0 = part_b[2 * row], b1 = part_b[2 * row + 1];
-        if (b0 == INT_MAX || (b1 != INT_MAX && s1 > s0)) {  // the other half holds higher columns: strict >
-          s0 = s1;
-          b0 = b1;
+        float s0 = part_s[4 * row];
+        int b0 = part_b[4 * row];
+#pragma unroll
+        for (int c = 1; c < 4; ++c) {  // highest similarity; the lowest B position on ties
+          const float s1 = part_s[4 * row + c];
+          const int b1 = part_b[4 * row + c];
+          if (b1 != INT_MAX && (b0 == INT_MAX || s1 > s0 || (s1 == s0 && b1 < b0))) {
+            s0 = s1;
+            b0 = b1;
+          }
         }
         const bool has = b0 != INT_MAX;
         const float cosv = has ? s0 * a.inv_a[(int64_t)lh * a.inv_stride + ai] + 0.f : -INFINITY;
         a.edge_sim[(int64_t)lh * a.edge_stride + ai] = cosv;
-        a.edge_b[(int64_t)lh * a.edge_stride + ai] = has ? 2 * b0 + 1 : -1;
+        // (no comparison ever held: not-a-number keys.  The edge still names a real B token, so that a ranking that
+        // takes every edge never hands the merge an index outside the head.)
+        a.edge_b[(int64_t)lh * a.edge_stride + ai] = has ? 2 * b0 + 1 : 1;
       }
     }
   }
@@ -228,7 +327,7 @@ __global__ void __launch_bounds__(kBThreads, 1) bsm_match_kernel(const __grid_co
     for (int i = 0; i < 1000; ++i) __nanosleep(1000);
     __syncthreads();
   }
-  if (warp == 0) tmem_dealloc(tmem, 256);
+  if (warp == 0) tmem_dealloc(tmem, kBTmemCols);
 }
 
 // ---- after the ranking: output slots and member counts
@@ -352,8 +451,9 @@ __global__ void __launch_bounds__(kPrepThreads) bsm_prepare_kernel(const BsmMerg
 }
 
 // Eq. 5, one warp per token of the middle region: a merged A token writes nothing, a survivor is copied to its slot,
-// a B token with members is replaced by the degree-weighted mean of itself and its members (found by scanning the
-// head's selected edges in position order, so the summation order is fixed).
+// a B token with members is replaced by the degree-weighted mean of itself and its members (taken from the prepared
+// list and added in position order, so the summation order is fixed; a target with more than 32 members scans the
+// head's selected edges instead).
 __global__ void __launch_bounds__(256) bsm_merge_kernel(const BsmMergeArgs a) {
   const int lh = blockIdx.y, lane = threadIdx.x & 31;
   const int64_t mid = (int64_t)a.nA + a.nB;
@@ -456,7 +556,7 @@ bool bsm_supported(int dtype, int D) { return dtype == 1 && D == 128 && bsm_enco
 
 // workspace of one no-chunk round, in bytes, for LH slabs whose middle region has `mid` tokens
 size_t bsm_workspace_bytes(int64_t LH, int64_t mid) {
-  const int64_t nA = (mid + 1) / 2, inv_stride = (nA + 127) / 128 * 128;
+  const int64_t nA = (mid + 1) / 2, inv_stride = (nA + 255) / 256 * 256;
   return (size_t)LH * (2 * inv_stride * 4 + (nA + 1) * 4 + inv_stride * 4 + (inv_stride + 1) * 4 + nA * 4) + 1024;
 }
 
@@ -470,7 +570,7 @@ cudaError_t launch_bsm_match(const RoundArgs& r, void* scratch, cudaStream_t st)
   a.lo = r.lo;
   a.nA = (int32_t)((mid + 1) / 2);
   a.nB = (int32_t)(mid / 2);
-  a.inv_stride = ((int64_t)a.nA + 127) / 128 * 128;
+  a.inv_stride = ((int64_t)a.nA + 255) / 256 * 256;
   a.inv_a = static_cast<float*>(scratch);
   a.inv_b = a.inv_a + (int64_t)r.LH * a.inv_stride;
   a.edge_sim = r.edge_sim;
@@ -480,18 +580,22 @@ cudaError_t launch_bsm_match(const RoundArgs& r, void* scratch, cudaStream_t st)
   bsm_norm_kernel<<<dim3((unsigned)((mid + 7) / 8), (unsigned)r.LH), 256, 0, st>>>(a);
   cudaError_t e = cudaGetLastError();
   if (e != cudaSuccess) return e;
-  // (column, parity, token pair, slab) view of the middle region; out-of-range pairs read as zeros
-  CUtensorMap tm;
-  const cuuint64_t dims[4] = {128, 2, (cuuint64_t)a.nA, (cuuint64_t)r.LH};
-  const cuuint64_t strides[3] = {256, 512, (cuuint64_t)r.src_cap * 256};
-  const cuuint32_t box[4] = {64, 1, 128, 1}, es[4] = {1, 1, 1, 1};
-  void* addr = const_cast<unsigned char*>(reinterpret_cast<const unsigned char*>(r.k_src) + r.lo * 256);
-  if (bsm_encode_fn()(&tm, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 4, addr, dims, strides, box, es, CU_TENSOR_MAP_INTERLEAVE_NONE,
-                      CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
-    return cudaErrorInvalidValue;
+  // (column, 1, every second token, slab) views of the middle region, one from its first token (A) and one from its second
+  // (B), each exactly as long as its side: rows past the end read as zeros and nothing outside the region is touched
+  CUtensorMap tm[2];
+  for (int side = 0; side < 2; ++side) {
+    const cuuint64_t dims[4] = {128, 1, (cuuint64_t)(side ? a.nB : a.nA), (cuuint64_t)r.LH};
+    const cuuint64_t strides[3] = {256, 512, (cuuint64_t)r.src_cap * 256};
+    const cuuint32_t box[4] = {64, 1, 128, 1}, es[4] = {1, 1, 1, 1};
+    void* addr = const_cast<unsigned char*>(reinterpret_cast<const unsigned char*>(r.k_src) + (r.lo + side) * 256);
+    if (bsm_encode_fn()(&tm[side], CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 4, addr, dims, strides, box, es, CU_TENSOR_MAP_INTERLEAVE_NONE,
+                        CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                        CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
+      return cudaErrorInvalidValue;
+  }
   const size_t smem = kBBytes + 1024;
   if ((e = cudaFuncSetAttribute(bsm_match_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem)) != cudaSuccess) return e;
-  bsm_match_kernel<<<dim3((unsigned)((a.nA + kBT - 1) / kBT), (unsigned)r.LH), kBThreads, smem, st>>>(tm, a);
+  bsm_match_kernel<<<dim3((unsigned)((a.nA + kBM - 1) / kBM), (unsigned)r.LH), kBThreads, smem, st>>>(tm[0], tm[1], a);
   return cudaGetLastError();
 }
 
@@ -515,7 +619,7 @@ cudaError_t launch_bsm_merge(const RoundArgs& r, void* scratch, cudaStream_t st)
   a.edge_b = r.edge_b;
   a.sel = r.sel;
   a.edge_stride = r.edge_stride;
-  const int64_t inv_stride = ((int64_t)a.nA + 127) / 128 * 128;
+  const int64_t inv_stride = ((int64_t)a.nA + 255) / 256 * 256;
   a.selpre = reinterpret_cast<int32_t*>(static_cast<float*>(scratch) + 2 * (int64_t)r.LH * inv_stride);
   a.cnt = a.selpre + (int64_t)r.LH * (a.nA + 1);
   a.cnt_stride = inv_stride;
