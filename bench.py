@@ -278,7 +278,7 @@ def run_gpu(args):
     if rank == 0 and not args.skip_variants:
         extra["compress_variants"] = bench_compress_variants(b, synth, dev, K, V, peaks["hbm_gbs"], args.layers == 0)
         extra["recluster"] = bench_recluster(b, synth, dev, K, V)
-        extra["no_chunk"] = bench_no_chunk(b, dev, K, V, peaks)
+        extra["no_chunk"] = bench_no_chunk(b, synth, dev, K, V, peaks, args.layers == 0)
 
     # end to end: inputs start in pinned host memory, the compressed cache and the decode output end there
     e2e = None
@@ -525,32 +525,46 @@ def bench_serving_mix(b, synth, dev, peak_gbs, steps=128):
     return res
 
 
-def bench_no_chunk(b, dev, K, V, peaks):
+def bench_no_chunk(b, synth, dev, K, V, peaks, with_128k):
     """chunk = 0 (plain Bipartite Soft Matching, the paper's "w/o chunk" ablation): every A token against every B token
-    of its head, n^2 d / 4 multiply-adds per head -- the one compute-bound variant.  One round at ratio 1 over the first
-    16384 tokens of 4 layers x 8 KV heads; the tensor-core rate counts the similarity contraction alone."""
+    of its head, n^2 d / 4 multiply-adds per head -- the one compute-bound variant.  One round at ratio 1 over (i) the
+    first 16384 tokens of 4 layers x 8 KV heads and (ii) one layer of the 131072-token workload, the length at which
+    the paper's variant runs out of memory (the similarities are never stored here).  The tensor-core rate divides the
+    flops of the similarity contraction by the time of the whole round (norms, matching, ranking, merge)."""
     import torch
-    L, H, n, D = min(4, K.shape[0]), K.shape[1], 16384, K.shape[3]
-    Ks, Vs = K[:L, :, :n].contiguous(), V[:L, :, :n].contiguous()
-    p = b.Params(chunk=0, n_sink=0, n_recent=0, n_rounds_max=1, r_init=1.0, r_decay=0.0, r_min=1.0)
-    src = b.Cache(Ks, Vs, None, None, n)
-    out_len, _, cap = b.compress_plan(n, p)
-    dst = b.Cache.empty(L, H, cap, D, Ks.dtype, dev)
-    ws = torch.empty(b.workspace_bytes(src, p), dtype=torch.uint8, device=dev)
-    b.compress_prefill(src, dst, p, ws)
-    torch.cuda.synchronize()
-    t0, t1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-    t0.record()
-    iters = 3
-    for _ in range(iters):
+
+    def time_one(Ks, Vs, iters):
+        L, H, n, D = Ks.shape
+        p = b.Params(chunk=0, n_sink=0, n_recent=0, n_rounds_max=1, r_init=1.0, r_decay=0.0, r_min=1.0)
+        src = b.Cache(Ks, Vs, None, None, n)
+        out_len, _, cap = b.compress_plan(n, p)
+        dst = b.Cache.empty(L, H, cap, D, Ks.dtype, dev)
+        ws = torch.empty(b.workspace_bytes(src, p), dtype=torch.uint8, device=dev)
         b.compress_prefill(src, dst, p, ws)
-    t1.record()
-    torch.cuda.synchronize()
-    ms = t0.elapsed_time(t1) / iters
-    flops = 2.0 * L * H * (n / 2) * (n / 2) * D
-    tf = flops / (ms * 1e-3) / 1e12
-    return {"layers": L, "seq": n, "out_len": out_len, "ms": ms, "similarity_tflops": tf, "bound": "tensor",
-            "frac_of_bf16_peak": tf / peaks["bf16_tflops"], "status": b.workspace_status(ws)}
+        torch.cuda.synchronize()
+        t0, t1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        t0.record()
+        for _ in range(iters):
+            b.compress_prefill(src, dst, p, ws)
+        t1.record()
+        torch.cuda.synchronize()
+        ms = t0.elapsed_time(t1) / iters
+        tf = 2.0 * L * H * (n / 2) * (n / 2) * D / (ms * 1e-3) / 1e12
+        return {"layers": L, "seq": n, "out_len": out_len, "ms": ms, "similarity_tflops": tf, "bound": "tensor",
+                "frac_of_bf16_peak": tf / peaks["bf16_tflops"], "workspace_mib": ws.numel() / 2**20,
+                "status": b.workspace_status(ws)}
+
+    L, n = min(4, K.shape[0]), 16384
+    res = {"16k_4_layers": time_one(K[:L, :, :n].contiguous(), V[:L, :, :n].contiguous(), 3)}
+    if with_128k:
+        cfg = synth.CONFIGS["llama8b_128k"]
+        H, D = K.shape[1], K.shape[3]
+        K3 = synth.ar1_keys(1, H, cfg["s"], D, cfg["rho"], cfg["mean_std"], seed=cfg["seed"], dtype="bf16", device=dev)
+        V3 = synth.normal_values(1, H, cfg["s"], D, seed=cfg["seed"], dtype="bf16", device=dev)
+        res["128k_1_layer"] = time_one(K3, V3, 2)
+        del K3, V3
+    torch.cuda.empty_cache()
+    return res
 
 
 def bench_recluster(b, synth, dev, K, V):

@@ -240,3 +240,54 @@ def test_config5_serving_mix_reduced_layers():
             assert np.all(np.abs(got - ref[0]) <= 2 * PU.bf16_ulp(ref[0]) * 1.0001 + 1e-30)
     del caches
     torch.cuda.empty_cache()
+
+
+def test_no_chunking_16k_four_layers():
+    """chunk = 0 (plain Bipartite Soft Matching) in the launch the benchmark's no-chunk section times: the first 16384
+    tokens of 4 layers x 8 KV heads, every edge merged.  Invariants over everything, two slabs against the oracle."""
+    need_free(8)
+    b = B()
+    cfg = synth.CONFIGS["llama8b_32k"]
+    L, H, s, D = 4, cfg["H"], 16384, cfg["d"]
+    K = synth.ar1_keys(L, H, s, D, cfg["rho"], cfg["mean_std"], seed=cfg["seed"], dtype="bf16", device=DEV)
+    V = synth.normal_values(L, H, s, D, seed=cfg["seed"], dtype="bf16", device=DEV)
+    p = b.Params(chunk=0, n_sink=0, n_recent=0, n_rounds_max=1, r_init=1.0, r_decay=0.0, r_min=1.0)
+    dst, assign, rounds = TC.run_gpu_prefill(K, V, None, p, want_assign=True, cap_extra=0)
+    assert rounds == 1 and dst.len == s // 2
+    invariants_over_everything(K, V, dst, s, rounds)
+    for l, h in ((0, 0), (3, 5)):
+        slab_matches_full_run(K, V, p, dst, assign, l, h)
+    torch.cuda.empty_cache()
+
+
+def test_no_chunking_128k_sampled_rows():
+    """chunk = 0 at 131072 tokens (the length at which the paper's un-chunked variant runs out of memory): one layer,
+    8 KV heads, ratio 1.  The n^2 / 4 similarities are never stored.  Sampled A tokens are checked one by one: the
+    oracle's cosine row against all 65536 B tokens of the head names the target; the GPU's choice must be that token
+    or one whose cosine is within 1e-5 of the best (rounding order of an fp32 contraction)."""
+    need_free(6)
+    b = B()
+    cfg = synth.CONFIGS["llama8b_128k"]
+    L, H, s, D = 1, cfg["H"], cfg["s"], cfg["d"]
+    K = synth.ar1_keys(L, H, s, D, cfg["rho"], cfg["mean_std"], seed=cfg["seed"], dtype="bf16", device=DEV)
+    V = synth.normal_values(L, H, s, D, seed=cfg["seed"], dtype="bf16", device=DEV)
+    p = b.Params(chunk=0, n_sink=0, n_recent=0, n_rounds_max=1, r_init=1.0, r_decay=0.0, r_min=1.0)
+    dst, assign, rounds = TC.run_gpu_prefill(K, V, None, p, want_assign=True, cap_extra=0)
+    assert rounds == 1 and dst.len == s // 2
+    invariants_over_everything(K, V, dst, s, rounds)
+    rng = np.random.default_rng(5)
+    for h in (0, 6):
+        Kh = K[0, h].cpu().float().numpy().astype(np.float64)
+        KB = Kh[1::2]
+        asg = assign[0, h].cpu().numpy()
+        rows = np.concatenate([[0, s // 2 - 1], rng.integers(0, s // 2, size=62)])
+        S = O.cosine_matrix(Kh[0::2][rows], KB)
+        for i, a_idx in enumerate(rows):
+            got = int(asg[2 * a_idx])  # every edge is merged: B token j survives in slot j
+            assert 0 <= got < s // 2
+            best = int(np.argmax(S[i]))
+            assert got == best or S[i, got] >= S[i, best] - 1e-5, f"head {h} A token {a_idx}: {got} vs {best}"
+        # every B token's degree is one plus the number of A tokens that chose it
+        counts = np.bincount(asg[0::2], minlength=s // 2) + 1
+        np.testing.assert_array_equal(dst.deg[0, h, :s // 2].cpu().numpy(), counts)
+    torch.cuda.empty_cache()
