@@ -73,15 +73,43 @@ __host__ __device__ constexpr uint32_t bsm_idesc() {  // bf16 x bf16 -> fp32, bo
   return (1u << 4) | (1u << 7) | (1u << 10) | (((uint32_t)kBN >> 3) << 17) | ((128u >> 4) << 24);
 }
 
-// inverse norms: one warp per token of the middle region
+__device__ __forceinline__ uint4 ld16(const __nv_bfloat16* p) { return *reinterpret_cast<const uint4*>(p); }
+__device__ __forceinline__ void unpack8(const uint4 u, float (&f)[8]) {
+  f[0] = __uint_as_float(u.x << 16); f[1] = __uint_as_float(u.x & 0xffff0000u);
+  f[2] = __uint_as_float(u.y << 16); f[3] = __uint_as_float(u.y & 0xffff0000u);
+  f[4] = __uint_as_float(u.z << 16); f[5] = __uint_as_float(u.z & 0xffff0000u);
+  f[6] = __uint_as_float(u.w << 16); f[7] = __uint_as_float(u.w & 0xffff0000u);
+}
+
+// inverse norms: a warp takes four consecutive tokens, sixteen lanes (16 bytes each) per token, two tokens per load
 __global__ void __launch_bounds__(256) bsm_norm_kernel(const BsmArgs a) {
-  const int lh = blockIdx.y, lane = threadIdx.x & 31;
+  const int lh = blockIdx.y, lane = threadIdx.x & 31, half = lane >> 4, c8 = (lane & 15) * 8;
   const int64_t mid = (int64_t)a.nA + a.nB;
-  const int64_t o = (int64_t)blockIdx.x * 8 + (threadIdx.x >> 5);
-  if (o >= mid) return;
-  const float4 x = load4(a.k_src + ((int64_t)lh * a.src_cap + a.lo + o) * kBD + lane * 4);
-  const float ss = warp_sum(fmaf(x.x, x.x, fmaf(x.y, x.y, fmaf(x.z, x.z, x.w * x.w))));
-  if (lane == 0) ((o & 1) ? a.inv_b : a.inv_a)[(int64_t)lh * a.inv_stride + (o >> 1)] = ss > 0.f ? rsqrtf(ss) : 0.f;
+  const int64_t o0 = ((int64_t)blockIdx.x * 8 + (threadIdx.x >> 5)) * 4;
+  if (o0 >= mid) return;
+  const __nv_bfloat16* base = a.k_src + ((int64_t)lh * a.src_cap + a.lo) * kBD + c8;
+  const int64_t t0 = o0 + half, t1 = o0 + 2 + half;  // half 0: the two A tokens, half 1: the two B tokens
+  const uint4 z = make_uint4(0, 0, 0, 0);
+  const uint4 u0 = t0 < mid ? ld16(base + t0 * kBD) : z, u1 = t1 < mid ? ld16(base + t1 * kBD) : z;
+  float x[8], y[8];
+  unpack8(u0, x);
+  unpack8(u1, y);
+  float s0 = 0.f, s1 = 0.f;
+#pragma unroll
+  for (int e = 0; e < 8; ++e) {
+    s0 = fmaf(x[e], x[e], s0);
+    s1 = fmaf(y[e], y[e], s1);
+  }
+#pragma unroll
+  for (int d = 8; d >= 1; d >>= 1) {
+    s0 += __shfl_xor_sync(0xffffffffu, s0, d);
+    s1 += __shfl_xor_sync(0xffffffffu, s1, d);
+  }
+  if ((lane & 15) == 0) {
+    float* out = (half ? a.inv_b : a.inv_a) + (int64_t)lh * a.inv_stride;
+    if (t0 < mid) out[t0 >> 1] = s0 > 0.f ? rsqrtf(s0) : 0.f;
+    if (t1 < mid) out[t1 >> 1] = s1 > 0.f ? rsqrtf(s1) : 0.f;
+  }
 }
 
 // tcgen05.ld of 32 columns without the wait, and the wait with the registers as operands (so that no use moves above it)
@@ -348,7 +376,8 @@ struct BsmMergeArgs {
   const uint8_t* sel;      // [LH, edge_stride]
   int64_t edge_stride;
   int32_t* selpre;         // [LH, edge_stride + 1] selected edges before A token a (exclusive prefix; last = total)
-  int32_t* cnt;            // [LH, cnt_stride]     scratch of the prepare kernel (member counts, then fill cursors)
+  int32_t* cnt;            // [LH, cnt_stride]     prepare kernel: member counts, then fill cursors; at the end the member
+                           //                      of a B token that has exactly one (else -1)
   int32_t* off;            // [LH, cnt_stride + 1] start of each B token's member list (exclusive prefix of the counts)
   int32_t* list;           // [LH, edge_stride]    member A indices, grouped by B token (order inside a group: arbitrary)
   int64_t cnt_stride;
@@ -448,91 +477,107 @@ __global__ void __launch_bounds__(kPrepThreads) bsm_prepare_kernel(const BsmMerg
       list[off[b] + atomicSub(&cnt[b], 1) - 1] = ai;
     }
   }
+  __syncthreads();
+  // the counters are back at zero: reuse them for "the member of a B token that has exactly one" (the common case of
+  // the merge, which then needs no look-up in the list)
+  for (int b = tid; b < a.nB; b += kPrepThreads) cnt[b] = off[b + 1] - off[b] == 1 ? list[off[b]] : -1;
 }
 
-// Eq. 5, one warp per token of the middle region: a merged A token writes nothing, a survivor is copied to its slot,
-// a B token with members is replaced by the degree-weighted mean of itself and its members (taken from the prepared
-// list and added in position order, so the summation order is fixed; a target with more than 32 members scans the
-// head's selected edges instead).
-__global__ void __launch_bounds__(256) bsm_merge_kernel(const BsmMergeArgs a) {
-  const int lh = blockIdx.y, lane = threadIdx.x & 31;
-  const int64_t mid = (int64_t)a.nA + a.nB;
-  const int64_t o = (int64_t)blockIdx.x * 8 + (threadIdx.x >> 5);
-  if (o >= mid) return;
+// Eq. 5, one warp per pair (A token 2i, B token 2i + 1) of the middle region; lanes 0-15 carry the K row and lanes
+// 16-31 the V row (16 bytes each), so one load or store instruction moves both.  A merged A token writes nothing, a
+// survivor is copied to its slot (the raw bits), a B token with members is replaced by the degree-weighted mean of itself
+// and its members (taken from the prepared list and added in position order, so the summation order is fixed; a target
+// with more than 32 members scans the head's selected edges instead).
+__global__ void __launch_bounds__(128, 16) bsm_merge_kernel(const BsmMergeArgs a) {
+  const int lh = blockIdx.y, lane = threadIdx.x & 31, half = lane >> 4, c8 = (lane & 15) * 8;
+  const int idx = blockIdx.x * 4 + (threadIdx.x >> 5);
+  if (idx >= a.nA) return;
   const uint8_t* sel = a.sel + (int64_t)lh * a.edge_stride;
   const int32_t* eb = a.edge_b + (int64_t)lh * a.edge_stride;
   const int32_t* selpre = a.selpre + (int64_t)lh * (a.edge_stride + 1);
-  const int64_t src0 = (int64_t)lh * a.src_cap + a.lo;
-  const int idx = (int)(o >> 1);
+  const int64_t src0 = (int64_t)lh * a.src_cap + a.lo, dst0 = (int64_t)lh * a.dst_cap + a.lo;
+  const __nv_bfloat16* src = (half ? a.v_src : a.k_src) + c8;
+  __nv_bfloat16* dst = (half ? a.v_dst : a.k_dst) + c8;
   auto slot_b = [&](int b) { return (int64_t)(2 * b + 1) - selpre[b + 1]; };  // A tokens 0 .. b come before B token b
-  int64_t slot;
-  float4 fk, fv;
-  int n_new;
-  if (!(o & 1)) {  // A token
-    if (sel[idx]) {
-      if (a.assign && lane == 0) a.assign[(int64_t)lh * a.assign_stride + a.lo + o] = (int32_t)(a.lo + slot_b(eb[idx] >> 1));
-      return;
+  auto finish = [&](int64_t o, int64_t slot, int n_new) {
+    if (lane == 0) {
+      a.deg_dst[dst0 + slot] = n_new;
+      if (a.logdeg_dst) a.logdeg_dst[dst0 + slot] = logf((float)n_new);
+      if (a.assign) a.assign[(int64_t)lh * a.assign_stride + a.lo + o] = (int32_t)(a.lo + slot);
     }
-    slot = o - selpre[idx];
-    fk = load4(a.k_src + (src0 + o) * kBD + lane * 4);
-    fv = load4(a.v_src + (src0 + o) * kBD + lane * 4);
-    n_new = a.deg_src ? a.deg_src[src0 + o] : 1;
+  };
+  const int64_t oa = 2 * (int64_t)idx, ob = oa + 1;
+  const bool has_b = idx < a.nB;
+  const int32_t* off = a.off + (int64_t)lh * (a.cnt_stride + 1);
+  // everything that depends on nothing is requested first: flags, slots, list bounds, degree, the B row
+  const bool a_merged = sel[idx] != 0;
+  const int sp0 = selpre[idx], sp1 = selpre[idx + 1];
+  const int l0 = has_b ? off[idx] : 0, l1 = has_b ? off[idx + 1] : 0;
+  const int single = has_b ? a.cnt[(int64_t)lh * a.cnt_stride + idx] : -1;
+  int n_new = has_b && a.deg_src ? a.deg_src[src0 + ob] : 1;
+  const uint4 z = make_uint4(0, 0, 0, 0);
+  const uint4 rb = has_b ? ld16(src + (src0 + ob) * kBD) : z;
+  const uint4 ra = a_merged ? z : ld16(src + (src0 + oa) * kBD);
+  if (a_merged) {
+    if (a.assign && lane == 0) a.assign[(int64_t)lh * a.assign_stride + a.lo + oa] = (int32_t)(a.lo + slot_b(eb[idx] >> 1));
   } else {
-    slot = slot_b(idx);
-    fk = load4(a.k_src + (src0 + o) * kBD + lane * 4);
-    fv = load4(a.v_src + (src0 + o) * kBD + lane * 4);
-    n_new = a.deg_src ? a.deg_src[src0 + o] : 1;
-    const int32_t* off = a.off + (int64_t)lh * (a.cnt_stride + 1);
-    const int m = off[idx + 1] - off[idx];
-    if (m > 0) {
-      const float wb = (float)n_new;
-      fk.x *= wb; fk.y *= wb; fk.z *= wb; fk.w *= wb;
-      fv.x *= wb; fv.y *= wb; fv.z *= wb; fv.w *= wb;
-      auto add_member = [&](int am) {
-        const int64_t r = src0 + 2 * (int64_t)am;
-        const float4 mk = load4(a.k_src + r * kBD + lane * 4), mv = load4(a.v_src + r * kBD + lane * 4);
-        const int wa = a.deg_src ? a.deg_src[r] : 1;
-        const float w = (float)wa;
-        n_new += wa;
-        fk.x = fmaf(w, mk.x, fk.x); fk.y = fmaf(w, mk.y, fk.y); fk.z = fmaf(w, mk.z, fk.z); fk.w = fmaf(w, mk.w, fk.w);
-        fv.x = fmaf(w, mv.x, fv.x); fv.y = fmaf(w, mv.y, fv.y); fv.z = fmaf(w, mv.z, fv.z); fv.w = fmaf(w, mv.w, fv.w);
-      };
-      if (m <= 32) {
-        // the list is in arbitrary order: add the members in increasing position, so that the sum is reproducible
-        const int mine = lane < m ? a.list[(int64_t)lh * a.edge_stride + off[idx] + lane] : INT_MAX;
-        int rank = 0;
-        for (int i = 0; i < m; ++i) rank += __shfl_sync(0xffffffffu, mine, i) < mine ? 1 : 0;
-        for (int r = 0; r < m; ++r) {
-          const int src_lane = __ffs(__ballot_sync(0xffffffffu, lane < m && rank == r)) - 1;
-          add_member(__shfl_sync(0xffffffffu, mine, src_lane));
-        }
-      } else {
-        // a crowded target: scan the head's selected edges in position order
-        const int target = 2 * idx + 1;
-        int left = m;
-        for (int g0 = 0; g0 < a.nA && left > 0; g0 += 32) {
-          const int ai = g0 + lane;
-          unsigned members = __ballot_sync(0xffffffffu, ai < a.nA && sel[ai] && eb[ai] == target);
-          left -= __popc(members);
-          while (members) {
-            add_member(g0 + __ffs(members) - 1);
-            members &= members - 1;
-          }
+    const int64_t slot = oa - sp0;
+    *reinterpret_cast<uint4*>(dst + (dst0 + slot) * kBD) = ra;
+    finish(oa, slot, a.deg_src ? a.deg_src[src0 + oa] : 1);
+  }
+  if (!has_b) return;
+  const int64_t slot = ob - sp1;  // A tokens 0 .. idx come before this B token
+  const int m = l1 - l0;
+  uint4 out = rb;  // an untouched row keeps its bits
+  if (m > 0) {
+    float f[8];
+    unpack8(rb, f);
+    const float wb = (float)n_new;
+#pragma unroll
+    for (int e = 0; e < 8; ++e) f[e] *= wb;
+    auto add_member = [&](int am) {
+      const int64_t r = src0 + 2 * (int64_t)am;
+      float g[8];
+      unpack8(ld16(src + r * kBD), g);
+      const int wa = a.deg_src ? a.deg_src[r] : 1;
+      const float w = (float)wa;
+      n_new += wa;
+#pragma unroll
+      for (int e = 0; e < 8; ++e) f[e] = fmaf(w, g[e], f[e]);
+    };
+    if (m == 1) {
+      add_member(single);
+    } else if (m <= 32) {
+      // the list is in arbitrary order: add the members in increasing position, so that the sum is reproducible
+      const int mine = lane < m ? a.list[(int64_t)lh * a.edge_stride + l0 + lane] : INT_MAX;
+      int rank = 0;
+      for (int i = 0; i < m; ++i) rank += __shfl_sync(0xffffffffu, mine, i) < mine ? 1 : 0;
+      for (int r = 0; r < m; ++r) {
+        const int src_lane = __ffs(__ballot_sync(0xffffffffu, lane < m && rank == r)) - 1;
+        add_member(__shfl_sync(0xffffffffu, mine, src_lane));
+      }
+    } else {
+      // a crowded target: scan the head's selected edges in position order
+      const int target = 2 * idx + 1;
+      int left = m;
+      for (int g0 = 0; g0 < a.nA && left > 0; g0 += 32) {
+        const int ai = g0 + lane;
+        unsigned members = __ballot_sync(0xffffffffu, ai < a.nA && sel[ai] && eb[ai] == target);
+        left -= __popc(members);
+        while (members) {
+          add_member(g0 + __ffs(members) - 1);
+          members &= members - 1;
         }
       }
-      const float inv = 1.0f / (float)n_new;
-      fk.x *= inv; fk.y *= inv; fk.z *= inv; fk.w *= inv;
-      fv.x *= inv; fv.y *= inv; fv.z *= inv; fv.w *= inv;
     }
+    const float inv = 1.0f / (float)n_new;
+    out.x = pack_bf16x2(f[0] * inv, f[1] * inv);
+    out.y = pack_bf16x2(f[2] * inv, f[3] * inv);
+    out.z = pack_bf16x2(f[4] * inv, f[5] * inv);
+    out.w = pack_bf16x2(f[6] * inv, f[7] * inv);
   }
-  const int64_t d = (int64_t)lh * a.dst_cap + a.lo + slot;
-  store4(a.k_dst + d * kBD + lane * 4, fk);  // an untouched row round-trips bit for bit
-  store4(a.v_dst + d * kBD + lane * 4, fv);
-  if (lane == 0) {
-    a.deg_dst[d] = n_new;
-    if (a.logdeg_dst) a.logdeg_dst[d] = logf((float)n_new);
-    if (a.assign) a.assign[(int64_t)lh * a.assign_stride + a.lo + o] = (int32_t)(a.lo + slot);
-  }
+  *reinterpret_cast<uint4*>(dst + (dst0 + slot) * kBD) = out;
+  finish(ob, slot, n_new);
 }
 
 typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*, const cuuint64_t*,
@@ -577,7 +622,7 @@ cudaError_t launch_bsm_match(const RoundArgs& r, void* scratch, cudaStream_t st)
   a.edge_b = r.edge_b;
   a.edge_stride = r.edge_stride;
   a.status = r.status;
-  bsm_norm_kernel<<<dim3((unsigned)((mid + 7) / 8), (unsigned)r.LH), 256, 0, st>>>(a);
+  bsm_norm_kernel<<<dim3((unsigned)((mid + 31) / 32), (unsigned)r.LH), 256, 0, st>>>(a);
   cudaError_t e = cudaGetLastError();
   if (e != cudaSuccess) return e;
   // (column, 1, every second token, slab) views of the middle region, one from its first token (A) and one from its second
@@ -628,7 +673,7 @@ cudaError_t launch_bsm_merge(const RoundArgs& r, void* scratch, cudaStream_t st)
   bsm_prepare_kernel<<<(unsigned)r.LH, kPrepThreads, 0, st>>>(a);
   cudaError_t e = cudaGetLastError();
   if (e != cudaSuccess) return e;
-  bsm_merge_kernel<<<dim3((unsigned)((mid + 7) / 8), (unsigned)r.LH), 256, 0, st>>>(a);
+  bsm_merge_kernel<<<dim3((unsigned)((a.nA + 3) / 4), (unsigned)r.LH), 128, 0, st>>>(a);
   return cudaGetLastError();
 }
 
