@@ -568,6 +568,7 @@ int ckv_decode_attn(const ckv_layer_view* views_dev, int32_t Bz, int32_t H, int3
   a.partial = static_cast<float*>(workspace);
   a.Bz = Bz; a.H = H; a.G = G;
   decode_plan(Bz, H, dtype, max_len, 0, G, D, &a.n_splits, &a.span);
+  a.max_len = max_len;
   a.scale = scale;
   return launch_decode(a, dtype, D, static_cast<cudaStream_t>(cuda_stream)) == cudaSuccess ? CKV_OK : CKV_ERR_CUDA;
 }

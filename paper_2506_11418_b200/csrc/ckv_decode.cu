@@ -290,6 +290,11 @@ namespace {
 //   O^T[d, head]    += V^T P      mma.sync, V through ldmatrix.trans; P is the score accumulator re-packed
 //                                 to bf16, already in the layout the B operand needs
 // No CTA-wide barrier is used; a warp whose split is empty leaves at once.
+//
+// Small batches (CL = 8 or 16): the CTAs of one (sequence, KV head) form a thread-block cluster, every warp of the
+// cluster is one split, and the partials never leave the chip: each warp parks its partial in its CTA's shared memory,
+// and after a cluster barrier every CTA combines 128 / CL output columns of every query head by reading all CTAs'
+// partials through distributed shared memory.  One launch per call, no workspace traffic, no combine kernel.
 
 constexpr int kFT = 32;                         // tokens per tile
 constexpr int kFStages = 3;
@@ -324,10 +329,22 @@ __device__ __forceinline__ void mma_bf16_16816(float (&d)[4], uint32_t a0, uint3
       : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1));
 }
 
+__device__ __forceinline__ void cluster_sync_all() {
+  asm volatile("barrier.cluster.arrive.release.aligned;\n\tbarrier.cluster.wait.acquire.aligned;" ::: "memory");
+}
+// a float of the shared memory of CTA `rank` of this cluster, at the offset `local_addr` has in this CTA's window
+__device__ __forceinline__ float ld_cluster_f32(uint32_t local_addr, uint32_t rank) {
+  uint32_t ra;
+  float v;
+  asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(ra) : "r"(local_addr), "r"(rank));
+  asm volatile("ld.shared::cluster.f32 %0, [%1];" : "=f"(v) : "r"(ra) : "memory");
+  return v;
+}
+
 // PAGED: the cache lives in fixed-size pages, [n_pages, H, page_tokens, D], and a per-sequence block table maps
 // logical block i (tokens i * page_tokens ...) to its page; page_tokens is a multiple of the tile, so a tile never
 // straddles pages.  Each lane keeps one entry of the table (32 blocks per refill), handed out by shuffle.
-template <bool PAGED>
+template <bool PAGED, int CL>
 __global__ void __launch_bounds__(kFWarps * 32, 1) decode_fast_kernel(const DecodeArgs a) {
   constexpr int D = 128;
   extern __shared__ __align__(128) unsigned char smem_raw[];
@@ -336,7 +353,7 @@ __global__ void __launch_bounds__(kFWarps * 32, 1) decode_fast_kernel(const Deco
   const int split = blockIdx.x * kFWarps + warp;
   griddep_wait();    // the views, the queries and the partial buffer may belong to the kernel ahead in the stream
   griddep_launch();  // the combine kernel may become resident; it waits for this grid before it reads
-  if (split >= a.n_splits) return;
+  if (CL == 0 && split >= a.n_splits) return;  // (in a cluster every warp is a split, and all reach the barriers)
   const int h = blockIdx.y, b = blockIdx.z, G = a.G;
   ckv_layer_view view{};
   const int32_t* table = nullptr;
@@ -497,6 +514,65 @@ __global__ void __launch_bounds__(kFWarps * 32, 1) decode_fast_kernel(const Deco
   // ---- this split's partial: out[D], max, sum per query head
   l_run += __shfl_xor_sync(0xffffffffu, l_run, 1);
   l_run += __shfl_xor_sync(0xffffffffu, l_run, 2);
+  if constexpr (CL > 0) {
+    constexpr int P = D + 4, NP = kFWarps * CL, ND = D / CL, NPG = 32 / ND, PER = NP / NPG;
+    __syncthreads();  // every warp of the CTA is done with its ring: the partials take its place
+    float* part = reinterpret_cast<float*>(smem_raw);  // [warp][8 heads][P]
+    float* scl = part + kFWarps * 8 * P;               // [warp][NP] weights 2^(m_p - m)
+    if (t == 0) {
+      part[(warp * 8 + g) * P + D] = m_run;
+      part[(warp * 8 + g) * P + D + 1] = l_run;
+    }
+#pragma unroll
+    for (int e = 0; e < 2; ++e) {
+      float* dst = part + (warp * 8 + 2 * t + e) * P;
+#pragma unroll
+      for (int i = 0; i < 8; ++i) {
+        dst[16 * i + g] = oacc[i][e];
+        dst[16 * i + 8 + g] = oacc[i][2 + e];
+      }
+    }
+    cluster_sync_all();
+    const uint32_t part_s = (uint32_t)__cvta_generic_to_shared(smem_raw);
+    const int d = lane % ND, pg = lane / ND, d0 = (int)blockIdx.x * ND;  // this CTA's columns d0 .. d0 + ND - 1
+    for (int head = warp; head < G; head += kFWarps) {
+      float mp[NP / 32], lp[NP / 32], mm = -INFINITY;
+#pragma unroll
+      for (int k = 0; k < NP / 32; ++k) {
+        const int pi = lane + 32 * k;  // partial of warp (pi & 3) of CTA (pi >> 2)
+        const uint32_t addr = part_s + (uint32_t)((((pi & 3) * 8 + head) * P + D) * 4);
+        mp[k] = ld_cluster_f32(addr, (uint32_t)(pi >> 2));
+        lp[k] = ld_cluster_f32(addr + 4u, (uint32_t)(pi >> 2));
+        mm = fmaxf(mm, mp[k]);
+      }
+      mm = warp_max(mm);
+      float ll = 0.f;
+#pragma unroll
+      for (int k = 0; k < NP / 32; ++k) {
+        const float f = mp[k] == -INFINITY ? 0.f : exp2f(mp[k] - mm);
+        scl[warp * NP + lane + 32 * k] = f;
+        ll = fmaf(f, lp[k], ll);
+      }
+      ll = warp_sum(ll);
+      __syncwarp();
+      float acc = 0.f;
+#pragma unroll 4
+      for (int j = 0; j < PER; ++j) {
+        const int pi = pg * PER + j;
+        acc = fmaf(scl[warp * NP + pi], ld_cluster_f32(part_s + (uint32_t)((((pi & 3) * 8 + head) * P + d0 + d) * 4), (uint32_t)(pi >> 2)),
+                   acc);
+      }
+#pragma unroll
+      for (int sft = ND; sft < 32; sft <<= 1) acc += __shfl_xor_sync(0xffffffffu, acc, sft);
+      if (pg == 0) {
+        const float inv = ll > 0.f ? 1.f / ll : 0.f;
+        reinterpret_cast<__nv_bfloat16*>(a.out)[(((int64_t)b * a.H + h) * G + head) * D + d0 + d] = __float2bfloat16_rn(acc * inv);
+      }
+      __syncwarp();
+    }
+    cluster_sync_all();  // nobody leaves while its shared memory may still be read
+    return;
+  }
   float* pbase = a.partial + ((((int64_t)b * a.H + h) * G) * a.n_splits + split) * (D + 4);
   const int64_t hstride = (int64_t)a.n_splits * (D + 4);
   if (t == 0 && g < G) {
@@ -517,12 +593,77 @@ __global__ void __launch_bounds__(kFWarps * 32, 1) decode_fast_kernel(const Deco
   }
 }
 
+template <bool PAGED, int CL>
+cudaError_t launch_decode_cluster(DecodeArgs a, cudaStream_t st) {
+  auto kern = decode_fast_kernel<PAGED, CL>;
+  cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kFSmemBytes);
+  if (e != cudaSuccess) return e;
+  if (CL > 8 && (e = cudaFuncSetAttribute(kern, cudaFuncAttributeNonPortableClusterSizeAllowed, 1)) != cudaSuccess) return e;
+  a.n_splits = kFWarps * CL;
+  cudaLaunchConfig_t cfg{};
+  cfg.gridDim = dim3(CL, (unsigned)a.H, (unsigned)a.Bz);
+  cfg.blockDim = dim3(kFWarps * 32);
+  cfg.dynamicSmemBytes = kFSmemBytes;
+  cfg.stream = st;
+  cudaLaunchAttribute attr[2];
+  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[0].val.programmaticStreamSerializationAllowed = 1;
+  attr[1].id = cudaLaunchAttributeClusterDimension;
+  attr[1].val.clusterDim.x = CL;
+  attr[1].val.clusterDim.y = 1;
+  attr[1].val.clusterDim.z = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = 2;
+  return cudaLaunchKernelEx(&cfg, kern, a);
+}
+
+// How many clusters of CL CTAs of the decode kernel the device can hold at once (0: this cluster size cannot be
+// scheduled here); asked once per device and kernel.
+template <bool PAGED, int CL>
+int max_active_clusters() {
+  constexpr int kMaxDev = 64;
+  static int cached[kMaxDev];  // 0 = not asked yet, else the answer + 1
+  int dev = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDev) return 0;
+  if (cached[dev] == 0) {
+    auto kern = decode_fast_kernel<PAGED, CL>;
+    int n = 0;
+    bool ok = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kFSmemBytes) == cudaSuccess;
+    if (ok && CL > 8) ok = cudaFuncSetAttribute(kern, cudaFuncAttributeNonPortableClusterSizeAllowed, 1) == cudaSuccess;
+    if (ok) {
+      cudaLaunchConfig_t cfg{};
+      cfg.gridDim = dim3(CL, 1, 1);
+      cfg.blockDim = dim3(kFWarps * 32);
+      cfg.dynamicSmemBytes = kFSmemBytes;
+      cudaLaunchAttribute attr[1];
+      attr[0].id = cudaLaunchAttributeClusterDimension;
+      attr[0].val.clusterDim.x = CL;
+      attr[0].val.clusterDim.y = 1;
+      attr[0].val.clusterDim.z = 1;
+      cfg.attrs = attr;
+      cfg.numAttrs = 1;
+      if (cudaOccupancyMaxActiveClusters(&n, kern, &cfg) != cudaSuccess) {
+        n = 0;
+        cudaGetLastError();  // a refusal here only means "not this cluster size"
+      }
+    }
+    cached[dev] = n + 1;
+  }
+  return cached[dev] - 1;
+}
+
 template <bool PAGED>
 cudaError_t launch_decode_fast(const DecodeArgs& a, cudaStream_t st) {
-  cudaError_t e = cudaFuncSetAttribute(decode_fast_kernel<PAGED>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kFSmemBytes);
+  // Few (sequence, head) pairs: one cluster per pair in a single wave, when every warp still gets two tiles or more.
+  const int64_t pairs = (int64_t)a.Bz * a.H, tiles = (a.max_len + kFT - 1) / kFT;
+  if (pairs * 16 <= 148 && tiles >= 2 * 16 * kFWarps && max_active_clusters<PAGED, 16>() >= pairs)
+    return launch_decode_cluster<PAGED, 16>(a, st);
+  if (pairs * 8 <= 148 && tiles >= 2 * 8 * kFWarps && max_active_clusters<PAGED, 8>() >= pairs)
+    return launch_decode_cluster<PAGED, 8>(a, st);
+  cudaError_t e = cudaFuncSetAttribute(decode_fast_kernel<PAGED, 0>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kFSmemBytes);
   if (e != cudaSuccess) return e;
   const dim3 grid((unsigned)((a.n_splits + kFWarps - 1) / kFWarps), (unsigned)a.H, (unsigned)a.Bz);
-  if ((e = launch_dependent(decode_fast_kernel<PAGED>, grid, dim3(kFWarps * 32), kFSmemBytes, st, a)) != cudaSuccess) return e;
+  if ((e = launch_dependent(decode_fast_kernel<PAGED, 0>, grid, dim3(kFWarps * 32), kFSmemBytes, st, a)) != cudaSuccess) return e;
   return launch_dependent(decode_combine_kernel<__nv_bfloat16, 128>, dim3((unsigned)(a.Bz * a.H * a.G)), dim3(kCombThreads), 0,
                           st, a);
 }

@@ -77,6 +77,7 @@ struct DecodeArgs {
   int32_t Bz, H, G;
   int32_t n_splits;
   int64_t span;       // tokens per split
+  int64_t max_len;    // longest sequence of the batch (host's bound; chooses the launch shape)
   float scale;
   // paged cache (bf16 kernel only): pages of `page_tokens` tokens, [n_pages, H, page_tokens, D]
   const void* k_pages;

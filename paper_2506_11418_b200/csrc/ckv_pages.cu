@@ -141,6 +141,7 @@ int ckv_decode_attn_paged(const ckv_paged_view* views_dev, const void* k_pages, 
   a.partial = static_cast<float*>(workspace);
   a.Bz = Bz; a.H = H; a.G = G;
   decode_plan(Bz, H, dtype, max_len, 0, G, D, &a.n_splits, &a.span);
+  a.max_len = max_len;
   a.scale = scale;
   a.k_pages = k_pages; a.v_pages = v_pages; a.logdeg_pages = logdeg_pages; a.page_shift = shift;
   return launch_decode_paged(a, static_cast<cudaStream_t>(cuda_stream)) == cudaSuccess ? CKV_OK : CKV_ERR_CUDA;

@@ -116,3 +116,13 @@ def test_decode_config4_shape_small_batch():
     caches = build_batch([8192, 8192], [8448, 8448], 8, "bf16", seed=90, total_factor=4)
     worst = check_decode(caches, 8, 4, "bf16", seed=91)
     assert worst < 2e-2
+
+
+@pytest.mark.parametrize("lens,H,G", [([16416], 8, 4), ([5000], 2, 8), ([4096, 9000, 130], 1, 4), ([20000], 1, 1)])
+def test_decode_small_batch_cluster_path(lens, H, G):
+    """Few (sequence, head) pairs and long caches: the launch where the CTAs of a pair form a thread-block cluster and
+    combine their partials through distributed shared memory (16 CTAs per pair here; the ragged batches above take
+    the 8-CTA shape, large batches the two-kernel path).  The first case is the decode leg of the benchmark's step."""
+    caches = build_batch(lens, [n + 7 for n in lens], H, "bf16", seed=300 + H, total_factor=4)
+    worst = check_decode(caches, H, G, "bf16", seed=310 + G)
+    assert worst < 2e-2
