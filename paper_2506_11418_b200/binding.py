@@ -162,7 +162,14 @@ class Cache:
                         L, H, D, dtype_code(self.k.dtype), cap, self.len, self.pending)
 
 
+_raw_stream = getattr(torch._C, "_cuda_getCurrentRawStream", None)
+
+
 def _stream_ptr():
+    """The current CUDA stream as a pointer (the raw-handle query is several times cheaper than building a Stream object,
+    which matters for calls that take ten microseconds on the GPU)."""
+    if _raw_stream is not None:
+        return C.c_void_p(_raw_stream(torch.cuda.current_device()))
     return C.c_void_p(torch.cuda.current_stream().cuda_stream)
 
 

@@ -296,12 +296,18 @@ namespace {
 // and after a cluster barrier every CTA combines 128 / CL output columns of every query head by reading all CTAs'
 // partials through distributed shared memory.  One launch per call, no workspace traffic, no combine kernel.
 
-constexpr int kFT = 32;                         // tokens per tile
+constexpr int kFT = 32;                         // tokens per tile (large batches)
 constexpr int kFStages = 3;
 constexpr int kFWarps = 4;
 constexpr int kFTileBytes = kFT * 256;          // one bf16 tile of K or V
 constexpr int kFStageBytes = 2 * kFTileBytes + kFT * 4;
 constexpr size_t kFSmemBytes = (size_t)kFWarps * kFStages * kFStageBytes;
+// Small batches (cluster launch).  Measured on batch 1 x 8 KV heads x 16416 tokens: 4 warps x 3 stages x 32-token tiles
+// 18.5 us per call, 6 warps x 2 stages 20.0 us, 8 warps x 3 stages x 16-token tiles 20.1 us.
+constexpr int kCT = 32;
+constexpr int kCWarps = 4;
+constexpr int kCStages = 3;
+constexpr size_t kCSmemBytes = (size_t)kCWarps * kCStages * (2 * kCT * 256 + kCT * 4);
 
 __device__ __forceinline__ void cp_async16(uint32_t dst, const void* src, uint32_t src_bytes) {
   asm volatile("cp.async.cg.shared.global [%0], [%1], 16, %2;" ::"r"(dst), "l"(src), "r"(src_bytes) : "memory");
@@ -344,13 +350,15 @@ __device__ __forceinline__ float ld_cluster_f32(uint32_t local_addr, uint32_t ra
 // PAGED: the cache lives in fixed-size pages, [n_pages, H, page_tokens, D], and a per-sequence block table maps
 // logical block i (tokens i * page_tokens ...) to its page; page_tokens is a multiple of the tile, so a tile never
 // straddles pages.  Each lane keeps one entry of the table (32 blocks per refill), handed out by shuffle.
-template <bool PAGED, int CL>
-__global__ void __launch_bounds__(kFWarps * 32, 1) decode_fast_kernel(const DecodeArgs a) {
+template <bool PAGED, int CL, int TT, int NW, int ST>
+__global__ void __launch_bounds__(NW * 32, 1) decode_fast_kernel(const DecodeArgs a) {
   constexpr int D = 128;
+  constexpr int kTileBytes = TT * 256;                  // one bf16 tile of K or V
+  constexpr int kStageBytes = 2 * kTileBytes + TT * 4;  // K tile, V tile, log-degrees
   extern __shared__ __align__(128) unsigned char smem_raw[];
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
   const int g = lane >> 2, t = lane & 3;
-  const int split = blockIdx.x * kFWarps + warp;
+  const int split = blockIdx.x * NW + warp;
   griddep_wait();    // the views, the queries and the partial buffer may belong to the kernel ahead in the stream
   griddep_launch();  // the combine kernel may become resident; it waits for this grid before it reads
   if (CL == 0 && split >= a.n_splits) return;  // (in a cluster every warp is a split, and all reach the barriers)
@@ -366,10 +374,10 @@ __global__ void __launch_bounds__(kFWarps * 32, 1) decode_fast_kernel(const Deco
   }
   const int64_t len = view.len;
   // the sequence's own tiles are dealt evenly to the splits (a ragged batch stays balanced)
-  const int64_t seq_tiles = (len + kFT - 1) / kFT;
-  const int64_t t_begin = kFT * (seq_tiles * split / a.n_splits);
-  const int64_t t_end = min(len, kFT * (seq_tiles * (split + 1) / a.n_splits));
-  const int ntiles = (int)((t_end - t_begin + kFT - 1) / kFT);
+  const int64_t seq_tiles = (len + TT - 1) / TT;
+  const int64_t t_begin = TT * (seq_tiles * split / a.n_splits);
+  const int64_t t_end = min(len, TT * (seq_tiles * (split + 1) / a.n_splits));
+  const int ntiles = (int)((t_end - t_begin + TT - 1) / TT);
   const __nv_bfloat16* kbase = PAGED ? reinterpret_cast<const __nv_bfloat16*>(a.k_pages)
                                      : reinterpret_cast<const __nv_bfloat16*>(view.k) + (int64_t)h * view.cap * D;
   const __nv_bfloat16* vbase = PAGED ? reinterpret_cast<const __nv_bfloat16*>(a.v_pages)
@@ -379,8 +387,8 @@ __global__ void __launch_bounds__(kFWarps * 32, 1) decode_fast_kernel(const Deco
   const int64_t n_blocks = PAGED ? (len + ((int64_t)1 << a.page_shift) - 1) >> a.page_shift : 0;
   int64_t blk0 = PAGED ? t_begin >> a.page_shift : 0;
   int my_page = (PAGED && ntiles > 0 && blk0 + lane < n_blocks) ? table[blk0 + lane] : 0;
-  const uint32_t ring = (uint32_t)__cvta_generic_to_shared(smem_raw) + (uint32_t)warp * kFStages * kFStageBytes;
-  const float* ring_ld = reinterpret_cast<const float*>(smem_raw + (size_t)warp * kFStages * kFStageBytes);
+  const uint32_t ring = (uint32_t)__cvta_generic_to_shared(smem_raw) + (uint32_t)warp * ST * kStageBytes;
+  const float* ring_ld = reinterpret_cast<const float*>(smem_raw + (size_t)warp * ST * kStageBytes);
 
   // query fragments (A operand, rows = heads; rows >= G are zero)
   uint32_t qa[8][2];
@@ -396,8 +404,8 @@ __global__ void __launch_bounds__(kFWarps * 32, 1) decode_fast_kernel(const Deco
   const float sc = a.scale * kLog2e;
 
   auto issue = [&](int tile) {
-    const int64_t t0 = t_begin + (int64_t)tile * kFT;
-    const uint32_t st = ring + (uint32_t)(tile % kFStages) * kFStageBytes;
+    const int64_t t0 = t_begin + (int64_t)tile * TT;
+    const uint32_t st = ring + (uint32_t)(tile % ST) * kStageBytes;
     const int c = lane & 15;
     // row0: where the tile's first token sits in the K / V / log-degree arrays; rows of a tile are contiguous
     int64_t row0 = t0;
@@ -411,17 +419,17 @@ __global__ void __launch_bounds__(kFWarps * 32, 1) decode_fast_kernel(const Deco
       row0 = (((int64_t)page * a.H + h) << a.page_shift) + (t0 & (((int64_t)1 << a.page_shift) - 1));
     }
 #pragma unroll
-    for (int i = 0; i < 16; ++i) {
+    for (int i = 0; i < TT / 2; ++i) {
       const int r = (lane >> 4) + 2 * i;
       const bool ok = t0 + r < t_end;
       const int64_t row = ok ? row0 + r : row0;  // clamped address, zero-filled when out of range
       const uint32_t off = (uint32_t)r * 256u + (uint32_t)((c ^ (r & 7)) << 4);
       cp_async16(st + off, kbase + row * D + c * 8, ok ? 16u : 0u);
-      cp_async16(st + kFTileBytes + off, vbase + row * D + c * 8, ok ? 16u : 0u);
+      cp_async16(st + kTileBytes + off, vbase + row * D + c * 8, ok ? 16u : 0u);
     }
     if (ldbase) {  // one log-degree per lane; 4-byte copies have no alignment demands on the slab
-      const bool ok = t0 + lane < t_end;
-      cp_async4(st + 2 * kFTileBytes + lane * 4, ldbase + (ok ? row0 + lane : row0), ok ? 4u : 0u);
+      const bool ok = lane < TT && t0 + lane < t_end;
+      if (TT == 32 || lane < TT) cp_async4(st + 2 * kTileBytes + lane * 4, ldbase + (ok ? row0 + lane : row0), ok ? 4u : 0u);
     }
   };
 
@@ -431,28 +439,29 @@ __global__ void __launch_bounds__(kFWarps * 32, 1) decode_fast_kernel(const Deco
   float m_run = -INFINITY, l_run = 0.f;  // for head g (this thread's share of the tokens)
 
 #pragma unroll
-  for (int i = 0; i < kFStages - 1; ++i) {
+  for (int i = 0; i < ST - 1; ++i) {
     if (i < ntiles) issue(i);
     cp_async_commit();
   }
   for (int tile = 0; tile < ntiles; ++tile) {
-    cp_async_wait<kFStages - 2>();
+    cp_async_wait<ST - 2>();
     __syncwarp();
-    if (tile + kFStages - 1 < ntiles) issue(tile + kFStages - 1);
+    if (tile + ST - 1 < ntiles) issue(tile + ST - 1);
     cp_async_commit();
-    const int stage = tile % kFStages;
-    const uint32_t ks_ = ring + (uint32_t)stage * kFStageBytes, vs_ = ks_ + kFTileBytes;
-    const float* lds = ring_ld + (size_t)stage * (kFStageBytes / 4) + 2 * kFTileBytes / 4;
-    const int nt = (int)min((int64_t)kFT, t_end - (t_begin + (int64_t)tile * kFT));
+    const int stage = tile % ST;
+    const uint32_t ks_ = ring + (uint32_t)stage * kStageBytes, vs_ = ks_ + kTileBytes;
+    const float* lds = ring_ld + (size_t)stage * (kStageBytes / 4) + 2 * kTileBytes / 4;
+    const int nt = (int)min((int64_t)TT, t_end - (t_begin + (int64_t)tile * TT));
 
     // ---- S = Q K^T for 32 tokens: n tile j covers tokens 8j .. 8j+7
-    float sacc[4][4];
+    constexpr int NT = TT / 8;  // n tiles of 8 tokens
+    float sacc[NT][4];
 #pragma unroll
-    for (int j = 0; j < 4; ++j) sacc[j][0] = sacc[j][1] = sacc[j][2] = sacc[j][3] = 0.f;
+    for (int j = 0; j < NT; ++j) sacc[j][0] = sacc[j][1] = sacc[j][2] = sacc[j][3] = 0.f;
 #pragma unroll
     for (int kq = 0; kq < 4; ++kq) {
 #pragma unroll
-      for (int j = 0; j < 4; ++j) {
+      for (int j = 0; j < NT; ++j) {
         const int tok = 8 * j + (lane & 7);
         const int chunk = 4 * kq + (lane >> 3);
         uint32_t r[4];
@@ -462,10 +471,10 @@ __global__ void __launch_bounds__(kFWarps * 32, 1) decode_fast_kernel(const Deco
       }
     }
     // ---- bias, mask, online softmax (thread holds head g, tokens 8j + 2t, 8j + 2t + 1)
-    float p[4][2];
+    float p[NT][2];
     float tmax = -INFINITY;
 #pragma unroll
-    for (int j = 0; j < 4; ++j) {
+    for (int j = 0; j < NT; ++j) {
 #pragma unroll
       for (int e = 0; e < 2; ++e) {
         const int tok = 8 * j + 2 * t + e;
@@ -481,9 +490,9 @@ __global__ void __launch_bounds__(kFWarps * 32, 1) decode_fast_kernel(const Deco
     const float corr = exp2f(m_run - m_new);
     m_run = m_new;
     float psum = 0.f;
-    uint32_t pb[4];
+    uint32_t pb[NT];
 #pragma unroll
-    for (int j = 0; j < 4; ++j) {
+    for (int j = 0; j < NT; ++j) {
       const float p0 = exp2f(p[j][0] - m_new), p1 = exp2f(p[j][1] - m_new);
       psum += p0 + p1;
       pb[j] = pack_bf16x2(p0, p1);
@@ -497,7 +506,7 @@ __global__ void __launch_bounds__(kFWarps * 32, 1) decode_fast_kernel(const Deco
     }
     // ---- O^T += V^T P: m tile i covers d = 16 i .. 16 i + 15, k step s covers tokens 16 s .. 16 s + 15
 #pragma unroll
-    for (int s = 0; s < 2; ++s) {
+    for (int s = 0; s < TT / 16; ++s) {
 #pragma unroll
       for (int i = 0; i < 8; ++i) {
         const int mi = lane >> 3;
@@ -515,10 +524,11 @@ __global__ void __launch_bounds__(kFWarps * 32, 1) decode_fast_kernel(const Deco
   l_run += __shfl_xor_sync(0xffffffffu, l_run, 1);
   l_run += __shfl_xor_sync(0xffffffffu, l_run, 2);
   if constexpr (CL > 0) {
-    constexpr int P = D + 4, NP = kFWarps * CL, ND = D / CL, NPG = 32 / ND, PER = NP / NPG;
+    // ND output columns per combining CTA (a divisor of 32); with 10 CTAs the first 8 combine 16 columns each
+    constexpr int P = D + 4, NP = NW * CL, ND = (D % CL == 0 && 32 % (D / CL) == 0) ? D / CL : 16, NPG = 32 / ND, PER = NP / NPG;
     __syncthreads();  // every warp of the CTA is done with its ring: the partials take its place
     float* part = reinterpret_cast<float*>(smem_raw);  // [warp][8 heads][P]
-    float* scl = part + kFWarps * 8 * P;               // [warp][NP] weights 2^(m_p - m)
+    float* scl = part + NW * 8 * P;               // [warp][NP] weights 2^(m_p - m)
     if (t == 0) {
       part[(warp * 8 + g) * P + D] = m_run;
       part[(warp * 8 + g) * P + D + 1] = l_run;
@@ -535,22 +545,24 @@ __global__ void __launch_bounds__(kFWarps * 32, 1) decode_fast_kernel(const Deco
     cluster_sync_all();
     const uint32_t part_s = (uint32_t)__cvta_generic_to_shared(smem_raw);
     const int d = lane % ND, pg = lane / ND, d0 = (int)blockIdx.x * ND;  // this CTA's columns d0 .. d0 + ND - 1
-    for (int head = warp; head < G; head += kFWarps) {
-      float mp[NP / 32], lp[NP / 32], mm = -INFINITY;
+    for (int head = warp; head < G && (int)blockIdx.x * ND < D; head += NW) {
+      constexpr int NK = (NP + 31) / 32;
+      static_assert(NP % NPG == 0, "the partials split evenly over the lane groups");
+      float mp[NK], lp[NK], mm = -INFINITY;
 #pragma unroll
-      for (int k = 0; k < NP / 32; ++k) {
-        const int pi = lane + 32 * k;  // partial of warp (pi & 3) of CTA (pi >> 2)
-        const uint32_t addr = part_s + (uint32_t)((((pi & 3) * 8 + head) * P + D) * 4);
-        mp[k] = ld_cluster_f32(addr, (uint32_t)(pi >> 2));
-        lp[k] = ld_cluster_f32(addr + 4u, (uint32_t)(pi >> 2));
+      for (int k = 0; k < NK; ++k) {
+        const int pi = lane + 32 * k;  // partial of warp (pi % NW) of CTA (pi / NW)
+        const uint32_t addr = part_s + (uint32_t)((((pi % NW) * 8 + head) * P + D) * 4);
+        mp[k] = pi < NP ? ld_cluster_f32(addr, (uint32_t)(pi / NW)) : -INFINITY;
+        lp[k] = pi < NP ? ld_cluster_f32(addr + 4u, (uint32_t)(pi / NW)) : 0.f;
         mm = fmaxf(mm, mp[k]);
       }
       mm = warp_max(mm);
       float ll = 0.f;
 #pragma unroll
-      for (int k = 0; k < NP / 32; ++k) {
+      for (int k = 0; k < NK; ++k) {
         const float f = mp[k] == -INFINITY ? 0.f : exp2f(mp[k] - mm);
-        scl[warp * NP + lane + 32 * k] = f;
+        if (lane + 32 * k < NP) scl[warp * NP + lane + 32 * k] = f;
         ll = fmaf(f, lp[k], ll);
       }
       ll = warp_sum(ll);
@@ -559,7 +571,7 @@ __global__ void __launch_bounds__(kFWarps * 32, 1) decode_fast_kernel(const Deco
 #pragma unroll 4
       for (int j = 0; j < PER; ++j) {
         const int pi = pg * PER + j;
-        acc = fmaf(scl[warp * NP + pi], ld_cluster_f32(part_s + (uint32_t)((((pi & 3) * 8 + head) * P + d0 + d) * 4), (uint32_t)(pi >> 2)),
+        acc = fmaf(scl[warp * NP + pi], ld_cluster_f32(part_s + (uint32_t)((((pi % NW) * 8 + head) * P + d0 + d) * 4), (uint32_t)(pi / NW)),
                    acc);
       }
 #pragma unroll
@@ -595,15 +607,13 @@ __global__ void __launch_bounds__(kFWarps * 32, 1) decode_fast_kernel(const Deco
 
 template <bool PAGED, int CL>
 cudaError_t launch_decode_cluster(DecodeArgs a, cudaStream_t st) {
-  auto kern = decode_fast_kernel<PAGED, CL>;
-  cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kFSmemBytes);
-  if (e != cudaSuccess) return e;
-  if (CL > 8 && (e = cudaFuncSetAttribute(kern, cudaFuncAttributeNonPortableClusterSizeAllowed, 1)) != cudaSuccess) return e;
-  a.n_splits = kFWarps * CL;
+  // (the kernel's attributes were set by max_active_clusters, which every caller asks first)
+  auto kern = decode_fast_kernel<PAGED, CL, kCT, kCWarps, kCStages>;
+  a.n_splits = kCWarps * CL;
   cudaLaunchConfig_t cfg{};
   cfg.gridDim = dim3(CL, (unsigned)a.H, (unsigned)a.Bz);
-  cfg.blockDim = dim3(kFWarps * 32);
-  cfg.dynamicSmemBytes = kFSmemBytes;
+  cfg.blockDim = dim3(kCWarps * 32);
+  cfg.dynamicSmemBytes = kCSmemBytes;
   cfg.stream = st;
   cudaLaunchAttribute attr[2];
   attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
@@ -626,15 +636,15 @@ int max_active_clusters() {
   int dev = 0;
   if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDev) return 0;
   if (cached[dev] == 0) {
-    auto kern = decode_fast_kernel<PAGED, CL>;
+    auto kern = decode_fast_kernel<PAGED, CL, kCT, kCWarps, kCStages>;
     int n = 0;
-    bool ok = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kFSmemBytes) == cudaSuccess;
+    bool ok = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kCSmemBytes) == cudaSuccess;
     if (ok && CL > 8) ok = cudaFuncSetAttribute(kern, cudaFuncAttributeNonPortableClusterSizeAllowed, 1) == cudaSuccess;
     if (ok) {
       cudaLaunchConfig_t cfg{};
       cfg.gridDim = dim3(CL, 1, 1);
-      cfg.blockDim = dim3(kFWarps * 32);
-      cfg.dynamicSmemBytes = kFSmemBytes;
+      cfg.blockDim = dim3(kCWarps * 32);
+      cfg.dynamicSmemBytes = kCSmemBytes;
       cudaLaunchAttribute attr[1];
       attr[0].id = cudaLaunchAttributeClusterDimension;
       attr[0].val.clusterDim.x = CL;
@@ -654,16 +664,27 @@ int max_active_clusters() {
 
 template <bool PAGED>
 cudaError_t launch_decode_fast(const DecodeArgs& a, cudaStream_t st) {
-  // Few (sequence, head) pairs: one cluster per pair in a single wave, when every warp still gets two tiles or more.
-  const int64_t pairs = (int64_t)a.Bz * a.H, tiles = (a.max_len + kFT - 1) / kFT;
-  if (pairs * 16 <= 148 && tiles >= 2 * 16 * kFWarps && max_active_clusters<PAGED, 16>() >= pairs)
-    return launch_decode_cluster<PAGED, 16>(a, st);
-  if (pairs * 8 <= 148 && tiles >= 2 * 8 * kFWarps && max_active_clusters<PAGED, 8>() >= pairs)
-    return launch_decode_cluster<PAGED, 8>(a, st);
-  cudaError_t e = cudaFuncSetAttribute(decode_fast_kernel<PAGED, 0>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kFSmemBytes);
+  // Few (sequence, head) pairs: one cluster per pair in a single wave.
+  // (short caches too: a call costs about 9 us this way against 18 us for the two dependent kernels below)
+  const int64_t pairs = (int64_t)a.Bz * a.H, tiles = (a.max_len + kCT - 1) / kCT;
+  // The largest cluster of which `pairs` fit at once (on a B200: 7 of 16 CTAs, 11 of 10, 15 of 8); a short cache does
+  // not need more than 8 CTAs.
+  if (tiles >= 8 * 8 * kCWarps) {
+    if (max_active_clusters<PAGED, 16>() >= pairs) return launch_decode_cluster<PAGED, 16>(a, st);
+    if (max_active_clusters<PAGED, 10>() >= pairs) return launch_decode_cluster<PAGED, 10>(a, st);
+  }
+  if (max_active_clusters<PAGED, 8>() >= pairs) return launch_decode_cluster<PAGED, 8>(a, st);
+  static bool attr_set[64];  // per device
+  int dev = 0;
+  cudaError_t e = cudaGetDevice(&dev);
   if (e != cudaSuccess) return e;
+  if (dev < 0 || dev >= 64 || !attr_set[dev]) {
+    e = cudaFuncSetAttribute(decode_fast_kernel<PAGED, 0, kFT, kFWarps, kFStages>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kFSmemBytes);
+    if (e != cudaSuccess) return e;
+    if (dev >= 0 && dev < 64) attr_set[dev] = true;
+  }
   const dim3 grid((unsigned)((a.n_splits + kFWarps - 1) / kFWarps), (unsigned)a.H, (unsigned)a.Bz);
-  if ((e = launch_dependent(decode_fast_kernel<PAGED, 0>, grid, dim3(kFWarps * 32), kFSmemBytes, st, a)) != cudaSuccess) return e;
+  if ((e = launch_dependent(decode_fast_kernel<PAGED, 0, kFT, kFWarps, kFStages>, grid, dim3(kFWarps * 32), kFSmemBytes, st, a)) != cudaSuccess) return e;
   return launch_dependent(decode_combine_kernel<__nv_bfloat16, 128>, dim3((unsigned)(a.Bz * a.H * a.G)), dim3(kCombThreads), 0,
                           st, a);
 }
