@@ -215,7 +215,9 @@ def run_gpu(args):
     # the lengths a step produces are a function of shapes only, so the decode views can be built once
     dst.len = final_len
     views = [b.layer_views([dst], l, dev) for l in range(L)]
-    launches_per_step = 1 + 3 + 2 * L
+    # prefill round, append (copy, window round, copy), and one cluster launch per layer for batch-1 decode (the split
+    # and combine kernels of larger batches are one kernel here)
+    launches_per_step = 1 + 3 + L
 
     ev = lambda: torch.cuda.Event(enable_timing=True)
     comp_ev, dec_ev = [], []
