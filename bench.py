@@ -272,6 +272,21 @@ def run_gpu(args):
     extra = {"compress_ms": comp_ms, "compress_tokens_per_s": s / (comp_ms * 1e-3), "decode_ms_all_layers": dec_ms,
              "decode_gbs_batch1": dec_achieved}
 
+    if rank == 0:
+        # the same step captured once into a CUDA graph and replayed: what the GPU needs when the host issues nothing
+        graph = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(graph):
+            step(False)
+        graph.replay()
+        torch.cuda.synchronize()
+        g0, g1 = ev(), ev()
+        g0.record()
+        for _ in range(args.steps):
+            graph.replay()
+        g1.record()
+        torch.cuda.synchronize()
+        extra["step_from_cuda_graph_ms"] = g0.elapsed_time(g1) / args.steps
+        del graph
     if rank == 0 and not args.skip_decode_cfg4:
         extra["decode_cfg4"] = bench_decode_cfg4(b, synth, dev, peaks["hbm_gbs"])
         extra["decode_cfg4_paged"] = bench_decode_paged(b, synth, dev, peaks["hbm_gbs"])
