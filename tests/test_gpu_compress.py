@@ -294,6 +294,15 @@ def test_no_chunking_single_round(s, sink, recent, r):
     single_round_case(2, 2, s, "bf16", one_round(b, 0, r, b.SELECT_GLOBAL, sink, recent), seed=900 + s, deg_max=4)
 
 
+def test_no_chunking_ranked_per_chunk_is_the_same_thing():
+    """With one chunk per head the two ranking scopes coincide; a budget is only trimmed to in the per-head scope."""
+    b = B()
+    single_round_case(1, 3, 1500, "bf16", one_round(b, 0, 0.5, b.SELECT_CHUNK, 4, 8), seed=77, deg_max=3)
+    p = b.Params(chunk=0, n_sink=4, n_recent=8, n_rounds_max=16, r_init=0.6, r_decay=0.2, r_min=0.2, select=b.SELECT_CHUNK, budget=500)
+    st = multi_round_case(1, 2, 1500, "bf16", p, seed=78)
+    assert st["rounds"] >= 3 and st["dst"].len <= 500
+
+
 def test_no_chunking_paper_schedule():
     b = B()
     s = 3000
