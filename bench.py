@@ -700,7 +700,7 @@ def bench_decode_cfg4(b, synth, dev, peak_gbs):
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=20)
+    ap.add_argument("--steps", type=int, default=None, help="timed steps (default: 200; 3 for --impl reference, whose step is seconds of CPU work)")
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="ckv", choices=["ckv", "reference"])
     ap.add_argument("--layers", type=int, default=0, help="use only this many layers of the workload (profiling a small case)")
@@ -710,6 +710,8 @@ def main():
     ap.add_argument("--skip-variants", action="store_true")
     ap.add_argument("--skip-serving", action="store_true")
     args = ap.parse_args()
+    if args.steps is None:
+        args.steps = 3 if args.impl == "reference" else 200
     if args.impl == "reference":
         run_reference(args)
     else:

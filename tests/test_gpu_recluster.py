@@ -12,7 +12,7 @@ pytestmark = pytest.mark.gpu
 DEV = "cuda"
 
 
-@pytest.mark.parametrize("dtype,chunk,select", [("bf16", 64, 0), ("f32", 64, 0), ("bf16", 256, 0), ("bf16", 64, 1), ("bf16", 8, 0)])
+@pytest.mark.parametrize("dtype,chunk,select", [("bf16", 64, 0), ("f32", 64, 0), ("bf16", 256, 0), ("bf16", 64, 1), ("bf16", 8, 0), ("bf16", 0, 0)])
 def test_fixed_budget_trigger(dtype, chunk, select):
     from paper_2506_11418_b200 import binding as b
     L, H, D, s0, g = 2, 2, 128, 700, 48
