@@ -793,6 +793,7 @@ extern "C" int ckv_decode_attn_static(const ckv_layer_view* views_dev, int32_t B
   a.G = G;
   a.n_splits = n_splits;
   a.span = span;
+  a.max_len = max_len;
   a.scale = scale;
   return ckv::launch_decode(a, dtype, D, static_cast<cudaStream_t>(cuda_stream)) == cudaSuccess ? CKV_OK : CKV_ERR_CUDA;
 }
