@@ -302,7 +302,7 @@ __device__ __forceinline__ int block_exscan(int x, int* total, int* warp_tot) {
   return before + inc - x;
 }
 
-__global__ void __launch_bounds__(kSelThreads) select_kernel(const SelectArgs a) {
+__global__ void __launch_bounds__(kSelThreads, 2) select_kernel(const SelectArgs a) {
   static_assert(kSelThreads == 1024, "one warp total per lane in block_exscan");
   __shared__ uint32_t hist[256];
   __shared__ uint32_t s_prefix, s_rem;
@@ -325,10 +325,14 @@ __global__ void __launch_bounds__(kSelThreads) select_kernel(const SelectArgs a)
       for (int64_t i = tid; i < n_up; i += kSelThreads) {
         const uint32_t key = i < n ? sim_key(sim[i]) : 0u;
         const bool in = i < n && (key & mask) == prefix;
-        // similarities cluster, so most lanes hit the same bin: one atomic per distinct bin of the warp
         const uint32_t bin = in ? ((key >> shift) & 255u) : 256u;
-        const unsigned peers = __match_any_sync(0xffffffffu, bin);
-        if (in && lane == __ffs(peers) - 1) atomicAdd(&hist[bin], (uint32_t)__popc(peers));
+        if (pass == 3) {
+          // sign and exponent: similarities cluster, most lanes hit the same bin: one atomic per distinct bin of the warp
+          const unsigned peers = __match_any_sync(0xffffffffu, bin);
+          if (in && lane == __ffs(peers) - 1) atomicAdd(&hist[bin], (uint32_t)__popc(peers));
+        } else if (in) {
+          atomicAdd(&hist[bin], 1u);  // mantissa bytes of the few remaining candidates: spread over the bins
+        }
       }
       __syncthreads();
       if (tid < 32) {
@@ -366,11 +370,15 @@ __global__ void __launch_bounds__(kSelThreads) select_kernel(const SelectArgs a)
   const uint32_t T = prefix;   // key of the M-th best edge
   const int quota = (int)rem;  // how many edges equal to T are merged: the earliest ones
 
-  // ---- one pass in position order: every thread owns a run of consecutive edges
+  // ---- one pass in position order: every thread owns a run of consecutive edges (all threads busy when the head has
+  //      at least 1024 edges; at most 64 per thread and sweep, one bit each in a 64-bit mask)
+  const int run = (int)min((int64_t)kSelRun, max((int64_t)1, (n + kSelThreads - 1) / kSelThreads));
+  uint8_t* selp = a.sel + (int64_t)lh * n;
+  int32_t* offp = a.chunk_out_off + (int64_t)lh * a.n_chunks;
   int sel_run = 0, eq_run = 0;  // totals of the sweeps before this one
-  for (int64_t base = 0; base < n; base += (int64_t)kSelThreads * kSelRun) {
-    const int64_t first = base + (int64_t)tid * kSelRun;
-    const int len = (int)max((int64_t)0, min((int64_t)kSelRun, n - first));
+  for (int64_t base = 0; base < n; base += (int64_t)kSelThreads * run) {
+    const int64_t first = base + (int64_t)tid * run;
+    const int len = (int)max((int64_t)0, min((int64_t)run, n - first));
     unsigned long long gt_bits = 0ull, eq_bits = 0ull;
     for (int j = 0; j < len; ++j) {
       const uint32_t key = sim_key(sim[first + j]);
@@ -384,16 +392,23 @@ __global__ void __launch_bounds__(kSelThreads) select_kernel(const SelectArgs a)
     unsigned long long sel_bits = gt_bits;
     for (unsigned long long e = eq_bits, k = 0; e && (int)k < take; e &= e - 1, ++k) sel_bits |= e & (~e + 1ull);
     const int s_ex = sel_run + block_exscan(__popcll(sel_bits), &s_tot, warp_tot);
-    int before = s_ex;
-    for (int j = 0; j < len; ++j) {
-      const int64_t i = first + j;
-      const int sbit = (int)((sel_bits >> j) & 1ull);
-      a.sel[(int64_t)lh * n + i] = (uint8_t)sbit;
-      if (i % hc == 0) {
-        const int64_t ch = i / hc;
-        a.chunk_out_off[(int64_t)lh * a.n_chunks + ch] = (int32_t)(a.lo + ch * a.chunk - before);
+    if (len > 0) {
+      // flags: four at a time where the run allows it
+      if ((len & 3) == 0 && ((reinterpret_cast<uintptr_t>(selp) + (uintptr_t)first) & 3u) == 0) {
+        for (int j = 0; j < len; j += 4) {
+          const uint32_t nib = (uint32_t)(sel_bits >> j) & 15u;
+          *reinterpret_cast<uint32_t*>(selp + first + j) = (nib & 1u) | ((nib & 2u) << 7) | ((nib & 4u) << 14) | ((nib & 8u) << 21);
+        }
+      } else {
+        for (int j = 0; j < len; ++j) selp[first + j] = (uint8_t)((sel_bits >> j) & 1ull);
       }
-      before += sbit;
+      // output offset of every chunk that starts inside the run: chunk start minus the edges selected before it
+      int64_t ch = (first + hc - 1) / hc;
+      for (int64_t at = ch * hc; at < first + len; at += hc, ++ch) {
+        const int j = (int)(at - first);
+        const int before = s_ex + __popcll(sel_bits & ((1ull << j) - 1ull));
+        offp[ch] = (int32_t)(a.lo + ch * a.chunk - before);
+      }
     }
     eq_run += eq_tot;
     sel_run += s_tot;
