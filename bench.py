@@ -59,9 +59,9 @@ def decode_bytes(rows, D, es):
 # profiles/round_fast_kernel_llama8b_4layers.md (1 048 576 token-vectors per launch; traffic grows in proportion to
 # the token-vectors processed, so it is scaled to the launch timed here).  Valid only for the kernel source it
 # was taken from: the digest below is of ckv_compress_fast.cu at that time.
-NCU_TRAFFIC = {"bytes_per_token_vector": (536905728 + 239911168) / 1048576,
+NCU_TRAFFIC = {"bytes_per_token_vector": (536905472 + 238534912) / 1048576,
                "source": "paper_2506_11418_b200/csrc/ckv_compress_fast.cu",
-               "sha256": "b96ba7869f546928105c380bd1f9a43bde79e7911966ff761b457233a26960bf"}
+               "sha256": "cac8149dd5cca459a65579e8f4920999a6aab09152ec97f72602ed07318a0b1a"}
 
 
 def ncu_traffic(token_vectors: int):

@@ -118,8 +118,9 @@ __global__ void __launch_bounds__(NW * 32, 1) round_fast_kernel(const FastArgs a
   extern __shared__ __align__(128) unsigned char smem[];
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
   const int g = lane >> 2, t = lane & 3;
-  unsigned char* stage = smem + (size_t)warp * kStageBytes;
-  unsigned char* extra = smem + (size_t)NW * kStageBytes + (size_t)warp * kExtraBytes;
+  constexpr int kStage = KIND == kFastMatch ? kTileBytes : kStageBytes;  // the matching alone stages no V tile
+  unsigned char* stage = smem + (size_t)warp * kStage;
+  unsigned char* extra = smem + (size_t)NW * kStage + (size_t)warp * kExtraBytes;
   int* degs = reinterpret_cast<int*>(extra);             // [64]
   const uint32_t bar = smem_u32(extra + 384);
   const uint32_t k_s = smem_u32(stage), v_s = k_s + kTileBytes;
@@ -426,7 +427,7 @@ int sm_count() {
 
 template <int NW, bool HAS_DEG, int KIND>
 cudaError_t launch_fast_inst(const FastArgs& a, cudaStream_t st) {
-  const size_t smem = (size_t)NW * (kStageBytes + kExtraBytes);
+  const size_t smem = (size_t)NW * ((KIND == kFastMatch ? kTileBytes : kStageBytes) + kExtraBytes);
   const int64_t ctas = std::min<int64_t>(sm_count(), (a.n_items + NW - 1) / NW);
   cudaError_t e = cudaFuncSetAttribute(round_fast_kernel<NW, HAS_DEG, KIND>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
   if (e != cudaSuccess) return e;
@@ -477,7 +478,7 @@ cudaError_t launch_round_fast(const RoundArgs& r, int64_t n_full, cudaStream_t s
   a.chunk_out_off = r.chunk_out_off;
   switch (r.mode) {
     case kModeAll: return launch_fast_kind<7, kFastAll>(a, st);
-    case kModeMatchOnly: return launch_fast_kind<7, kFastMatch>(a, st);
+    case kModeMatchOnly: return launch_fast_kind<13, kFastMatch>(a, st);  // half the bytes per warp: twice the warps
     default: return launch_fast_kind<7, kFastSelect>(a, st);
   }
 }
