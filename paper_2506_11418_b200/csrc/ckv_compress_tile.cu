@@ -312,8 +312,9 @@ __global__ void __launch_bounds__(TileCfg<C>::T, TileCfg<C>::kCtasPerSm) round_t
     }
     cp_async_wait<2 * PV + 1>();  // V(n) was committed 2 PV + 1 groups ago
     // S2: the V tile has landed, the partial argmaxes are visible; do the weights need more than one bf16 piece?
-    const int deg_bits = __syncthreads_or(my_deg > 255 ? (my_deg > 65535 ? 2 : 1) : 0);
-    const int n_pieces = deg_bits >= 2 ? 3 : deg_bits + 1;
+    // (the barrier's reduction is a predicate, not a bitwise OR: ask for the third piece only when a second is needed)
+    int n_pieces = 1;
+    if (__syncthreads_or(my_deg > 255)) n_pieces = __syncthreads_or(my_deg > 65535) ? 3 : 2;
 
     // ---- one edge per A token
     if (tid < M) {

@@ -330,8 +330,9 @@ round_umma_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constan
       if (lane == 0) selmask[warp] = bits;
     }
     // do the weights need more than one bf16 piece?  (also: tables visible)
-    const int deg_bits = __syncthreads_or(my_deg > 255 ? (my_deg > 65535 ? 2 : 1) : 0);
-    const int n_pieces = deg_bits >= 2 ? 3 : deg_bits + 1;
+    // (the barrier's reduction is a predicate, not a bitwise OR: ask for the third piece only when a second is needed)
+    int n_pieces = 1;
+    if (__syncthreads_or(my_deg > 255)) n_pieces = __syncthreads_or(my_deg > 65535) ? 3 : 2;
 
     // ---- output order: survivors keep their order, a merged A token shares its B token's slot
     auto sel_bit = [&](int ai) { return (selmask[ai >> 5] >> (ai & 31)) & 1u; };
