@@ -51,7 +51,11 @@ def compare_values(gpu: np.ndarray, ref: np.ndarray, dtype: str, what: str):
     ref_b = O.bf16_round(ref)
     diff = np.abs(gpu - ref_b)
     ulp = bf16_ulp(ref_b)
-    assert np.all(diff <= ulp * 1.0001), f"{what}: more than one bf16 ulp off, max {np.max(diff / ulp):.2f} ulp"
+    # One bf16 step, except where the members of a cluster cancel: Eq. 5 in fp32 carries an absolute error of a few
+    # 2^-24 * sum n_i |x_i| / n' <= a few 2^-24 * max |x|, which exceeds the ulp of a centroid much smaller than its members.
+    cancel = np.abs(gpu - ref) <= 1e-6 * (np.abs(ref).max() if ref.size else 0.0)
+    bad = (diff > ulp * 1.0001) & ~cancel
+    assert not bad.any(), f"{what}: more than one bf16 ulp off, max {np.max((diff / ulp)[bad]):.2f} ulp"
     within = np.abs(gpu - ref) <= 2e-2
     frac = float(np.mean(within)) if gpu.size else 1.0
     assert np.all(within | (np.abs(ref) >= 2.0)), f"{what}: an element below 2 in magnitude is more than 2e-2 off"

@@ -169,19 +169,23 @@ def multi_round_check(K, V, dtype, p):
     stats = dict(rounds=rounds, dst=dst, assign=assign)
     if np.array_equal(g["assign"], asg):
         np.testing.assert_array_equal(g["deg"], do)
+        close = True
         for l in range(L):
             for h in range(H):
-                # bf16 storage between rounds can flip a rounding in an earlier round: allow one ulp per round
+                # bf16 storage between rounds can flip a rounding in an earlier round: allow one ulp per round.  Where a
+                # flipped centroid later meets members that cancel it, its one ulp is many ulps of the small result:
+                # such a run is not accepted here but checked round by round below.
                 if dtype == "bf16":
                     diff = np.abs(g["K"][l, h] - Ko[l, h])
-                    assert np.all(diff <= rounds * PU.bf16_ulp(Ko[l, h]) * 1.0001)
+                    close &= bool(np.all(diff <= rounds * PU.bf16_ulp(Ko[l, h]) * 1.0001))
                     diff = np.abs(g["V"][l, h] - Vo[l, h])
-                    assert np.all(diff <= rounds * PU.bf16_ulp(Vo[l, h]) * 1.0001 + 1e-30)
+                    close &= bool(np.all(diff <= rounds * PU.bf16_ulp(Vo[l, h]) * 1.0001 + 1e-30))
                 else:
                     PU.compare_values(g["K"][l, h], Ko[l, h], dtype, "K")
                     PU.compare_values(g["V"][l, h], Vo[l, h], dtype, "V")
-        stats["end_to_end"] = True
-        return stats
+        if close:
+            stats["end_to_end"] = True
+            return stats
     # round by round on the GPU's own intermediates
     stats["end_to_end"] = False
     cur = b.Cache(K, V, None, None, s)
