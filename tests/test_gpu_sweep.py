@@ -52,3 +52,26 @@ def test_schedule_sweep(chunk, s, select, r_init, decay, budget, rounds, seed):
     p = b.Params(chunk=chunk, n_sink=16, n_recent=64, n_rounds_max=rounds, r_init=r_init, r_decay=decay,
                  r_min=max(decay, 0.2), select=select, budget=budget)
     TC.multi_round_case(1, 2, s, "bf16", p, seed=seed)
+
+
+def decode_cases(n, seed):
+    rng = random.Random(seed)
+    out = []
+    for i in range(n):
+        H = rng.choice([1, 2, 4, 8])
+        G = rng.choice([1, 2, 4, 7, 8])
+        Bz = rng.choice([1, 1, 2, 3, 5, 12, 40])
+        top = rng.choice([40, 300, 3000, 9000, 20000]) if Bz * H <= 16 else rng.choice([40, 300, 2000])
+        lens = [rng.choice([0, 1, rng.randint(1, top), top]) for _ in range(Bz)]
+        dtype = rng.choice(["bf16", "bf16", "bf16", "f32"])
+        out.append(pytest.param(lens, H, G, dtype, rng.random() < 0.8, 5000 + i, id=f"{i}-B{Bz}-H{H}-G{G}-{dtype}-top{top}"))
+    return out
+
+
+@pytest.mark.parametrize("lens,H,G,dtype,with_deg,seed", decode_cases(24, 11))
+def test_decode_sweep(lens, H, G, dtype, with_deg, seed):
+    """Batch sizes and lengths on both sides of every launch choice of the decode path (thread-block clusters of 16, 10
+    and 8 CTAs, split kernel + combine), empty and one-token sequences included."""
+    import test_gpu_decode as TD
+    caches = TD.build_batch(lens, [n + 5 for n in lens], H, dtype, seed=seed, with_deg=with_deg)
+    TD.check_decode(caches, H, G, dtype, seed=seed + 1)
