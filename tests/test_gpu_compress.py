@@ -100,18 +100,20 @@ def test_round_global_top_m(dtype, chunk, s, r, budget):
     single_round_case(2, 2, s, dtype, one_round(b, chunk, r, b.SELECT_GLOBAL, 16, 64, budget), seed=3 * chunk + s, deg_max=3)
 
 
-@pytest.mark.parametrize("dtype", ["f32", "bf16"])
-def test_identical_keys_tie_to_lowest_index(dtype):
-    """All keys of a chunk equal: every similarity ties at 1, the first B token must win, the centroid key is that key."""
+@pytest.mark.parametrize("dtype,c", [("f32", 64), ("bf16", 64), ("bf16", 128), ("bf16", 256), ("f32", 6), ("bf16", 0)])
+def test_identical_keys_tie_to_lowest_index(dtype, c):
+    """All keys of a chunk equal: every similarity ties at 1, the first B token must win, the centroid key is that key.
+    Without chunks (c = 0) the whole head is one chunk and its first B token collects every A token."""
     b = B()
-    L, H, s, c = 1, 2, 256, 64
-    base = synth.normal_values(L, H, s // c, 128, seed=3, dtype=dtype, device=DEV)
-    K = base.repeat_interleave(c, dim=2).contiguous()
+    L, H, s = 1, 2, 768
+    cc = c if c else s
+    base = synth.normal_values(L, H, s // cc, 128, seed=3, dtype=dtype, device=DEV)
+    K = base.repeat_interleave(cc, dim=2).contiguous()
     V = synth.normal_values(L, H, s, 128, seed=4, dtype=dtype, device=DEV)
     p = one_round(b, c, 1.0, b.SELECT_GLOBAL)
     dst, assign, _ = run_gpu_prefill(K, V, None, p)
     a = assign.cpu().numpy()
-    expect = (np.arange(s) // c) * (c // 2)              # every A token of chunk i lands in slot of B token 1 of chunk i
+    expect = (np.arange(s) // cc) * (cc // 2)            # every A token of chunk i lands in slot of B token 1 of chunk i
     pos = np.arange(s)
     is_a = pos % 2 == 0
     np.testing.assert_array_equal(a[0, 0][is_a], expect[is_a])
