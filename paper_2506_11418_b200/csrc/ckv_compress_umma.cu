@@ -483,6 +483,224 @@ round_umma_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constan
   if (warp == 0) tmem_dealloc(tmem, kTmemCols);
 }
 
+// ---- the matching alone (first pass of a round ranked per head): a pipeline instead of a chain -------------------
+// Nothing but the K tile is needed, so three chunks fit: a TMA warp streams K tiles through a ring of three stages, an
+// MMA warp issues S = A B^T for up to four chunks ahead (four tensor-memory slots of 128 columns), and two groups of
+// eight consumer warps follow, each on every other chunk: inverse norms from the staged tile (the stage goes back to the
+// ring once the group and the MMA have read it), then Eq. 2 and the row argmax from tensor memory, (cosine, target) out.
+// Loads, contraction and the two groups' epilogues overlap; the chunk-at-a-time kernel above needs 2.7 us per chunk for
+// this, its bytes 1.5 us.
+constexpr int kMStages = 3;
+constexpr int kMSlots = 4;
+constexpr int kMConsumers = 16;
+constexpr int kMThreads = (kMConsumers + 2) * 32;
+constexpr int oMInv = kMStages * kTileU;             // float [kMSlots][256]: A tokens [0,128), B tokens [128,256)
+constexpr int oMPartS = oMInv + kMSlots * 1024;      // float [2 groups][128][2]
+constexpr int oMPartB = oMPartS + 2048;              // int   [2 groups][128][2]
+constexpr int oMBar = oMPartB + 2048;                // full[3], empty[3], tfull[4], tempty[4]
+constexpr int oMFlag = oMBar + 128;                  // int: a consumer's wait gave up
+constexpr int oMTmem = oMFlag + 16;
+constexpr int kMBytes = oMTmem + 16;
+
+__device__ __forceinline__ void mbar_arrive_one(uint32_t bar) {
+  asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
+}
+
+__global__ void __launch_bounds__(kMThreads, 1)
+match_umma_kernel(const __grid_constant__ CUtensorMap tm_k, const RoundArgs a, const int n_full) {
+  extern __shared__ unsigned char smem_raw[];
+  unsigned char* smem = reinterpret_cast<unsigned char*>((reinterpret_cast<uintptr_t>(smem_raw) + kUAlign - 1) & ~(uintptr_t)(kUAlign - 1));
+  const uint32_t s_base = smem_u32(smem);
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  float* inv_all = reinterpret_cast<float*>(smem + oMInv);
+  float* part_s = reinterpret_cast<float*>(smem + oMPartS);
+  int* part_b = reinterpret_cast<int*>(smem + oMPartB);
+  volatile int* s_failed = reinterpret_cast<volatile int*>(smem + oMFlag);
+  auto bar_full = [&](int i) { return s_base + oMBar + 8u * i; };
+  auto bar_empty = [&](int i) { return s_base + oMBar + 8u * (kMStages + i); };
+  auto bar_tfull = [&](int i) { return s_base + oMBar + 8u * (2 * kMStages + i); };
+  auto bar_tempty = [&](int i) { return s_base + oMBar + 8u * (2 * kMStages + kMSlots + i); };
+  const int64_t n_items = (int64_t)n_full * a.LH;
+  // this CTA's k-th chunk is item blockIdx.x + k gridDim.x
+  const int64_t my_items = n_items > (int64_t)blockIdx.x ? (n_items - blockIdx.x + gridDim.x - 1) / gridDim.x : 0;
+
+  if (tid == 0) {
+    for (int i = 0; i < kMStages; ++i) {
+      mbar_init(bar_full(i), 1);
+      mbar_init(bar_empty(i), 1 + kMConsumers / 2);  // the MMA's commit and every warp of the chunk's group (norms read)
+    }
+    for (int i = 0; i < kMSlots; ++i) {
+      mbar_init(bar_tfull(i), 1);
+      mbar_init(bar_tempty(i), kMConsumers / 2);
+    }
+    *s_failed = 0;
+    mbar_init_fence();
+  }
+  if (warp == 0) tmem_alloc(s_base + oMTmem, 512);
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const uint32_t tmem = *reinterpret_cast<volatile uint32_t*>(smem + oMTmem);
+  bool failed = false;
+
+  if (warp == kMConsumers) {
+    // ------------------------------------------------------------------ TMA warp
+    if (lane == 0) {
+      for (int64_t k = 0; k < my_items && !failed; ++k) {
+        const int64_t item = blockIdx.x + k * gridDim.x;
+        const int lh = (int)(item / n_full), ch = (int)(item % n_full);
+        const int st = (int)(k % kMStages);
+        if (!mbar_wait(bar_empty(st), (uint32_t)(((k / kMStages) & 1) ^ 1))) {
+          failed = true;
+          break;
+        }
+        const uint32_t dst = s_base + (uint32_t)st * kTileU;
+        mbar_arrive_expect_tx(bar_full(st), kTileU);
+        tma_load_4d(dst, &tm_k, 0, 0, ch * kUM, lh, bar_full(st));
+        tma_load_4d(dst + kHalf, &tm_k, 64, 0, ch * kUM, lh, bar_full(st));
+        tma_load_4d(dst + 2 * kHalf, &tm_k, 0, 1, ch * kUM, lh, bar_full(st));
+        tma_load_4d(dst + 3 * kHalf, &tm_k, 64, 1, ch * kUM, lh, bar_full(st));
+      }
+    }
+  } else if (warp == kMConsumers + 1) {
+    // ------------------------------------------------------------------ MMA warp
+    if (lane == 0) {
+      for (int64_t k = 0; k < my_items && !failed; ++k) {
+        const int st = (int)(k % kMStages), sl = (int)(k % kMSlots);
+        if (!mbar_wait(bar_full(st), (uint32_t)((k / kMStages) & 1)) || !mbar_wait(bar_tempty(sl), (uint32_t)(((k / kMSlots) & 1) ^ 1))) {
+          failed = true;
+          break;
+        }
+        tc_fence_after();
+        const uint32_t k_s = s_base + (uint32_t)st * kTileU;
+#pragma unroll
+        for (int ks = 0; ks < 8; ++ks) {
+          const uint32_t off = (uint32_t)(ks >> 2) * kHalf + (uint32_t)(ks & 3) * 32u;
+          umma_bf16(tmem + (uint32_t)sl * kUM, umma_desc_sw128(k_s + off, 16, 1024), umma_desc_sw128(k_s + 2 * kHalf + off, 16, 1024),
+                    umma_idesc(false), ks ? 1u : 0u);
+        }
+        umma_commit(bar_empty(st));
+        umma_commit(bar_tfull(sl));
+      }
+    }
+  } else {
+    // ------------------------------------------------------------------ consumers: group 0 takes the even chunks of
+    // this CTA, group 1 the odd ones
+    const int g = lane >> 2, t = lane & 3;
+    const int grp = warp >> 3, wg = warp & 7, gtid = tid & 255;
+    const int q = wg & 3, ch2 = wg >> 2;  // tensor-memory lanes 32 q .. + 31 (A tokens); columns 64 ch2 .. + 63 (B tokens)
+    float* gpart_s = part_s + grp * 256;
+    int* gpart_b = part_b + grp * 256;
+    auto group_sync = [&]() {
+      if (grp == 0) {
+        asm volatile("bar.sync 1, 256;" ::: "memory");
+      } else {
+        asm volatile("bar.sync 2, 256;" ::: "memory");
+      }
+    };
+    for (int64_t k = grp; k < my_items; k += 2) {
+      const int64_t item = blockIdx.x + k * gridDim.x;
+      const int lh = (int)(item / n_full), ch = (int)(item % n_full);
+      const int st = (int)(k % kMStages), sl = (int)(k % kMSlots);
+      float* inv_nrm = inv_all + sl * 256;
+      // ---- inverse norms from the staged tile: a warp takes two blocks of 16 tokens (blocks 0-7: A tokens, 8-15: B)
+      if (!failed && !mbar_wait(bar_full(st), (uint32_t)((k / kMStages) & 1))) failed = true;
+      if (!failed) {
+        const uint32_t k_s = s_base + (uint32_t)st * kTileU;
+#pragma unroll
+        for (int half = 0; half < 2; ++half) {
+          const int blk = 2 * wg + half, w8 = blk & 7;
+          const bool for_a = blk < 8;
+          float n0[4] = {0.f, 0.f, 0.f, 0.f}, n1[4] = {0.f, 0.f, 0.f, 0.f};
+          const uint32_t part = k_s + (for_a ? 0u : 2u * kHalf);
+          const int r0 = 16 * w8 + (lane & 7);
+#pragma unroll
+          for (int kq = 0; kq < 4; ++kq) {
+            uint32_t p[4], qq[4];
+            ldsm_x4(part + sw_off(r0, 4 * kq + (lane >> 3)), p);
+            ldsm_x4(part + sw_off(r0 + 8, 4 * kq + (lane >> 3)), qq);
+            mma_bf16(n0, p[0], qq[0], p[1], qq[1], p[0], p[1]);
+            mma_bf16(n0, p[2], qq[2], p[3], qq[3], p[2], p[3]);
+            mma_bf16(n1, p[0], qq[0], p[1], qq[1], qq[0], qq[1]);
+            mma_bf16(n1, p[2], qq[2], p[3], qq[3], qq[2], qq[3]);
+          }
+          if (t == (g >> 1)) {  // the diagonal entries (see the kernel above)
+            const float s0 = (g & 1) ? n0[1] : n0[0], s1 = (g & 1) ? n1[3] : n1[2];
+            const int base = (for_a ? 0 : kUM) + 16 * w8;
+            inv_nrm[base + g] = s0 > 0.f ? rsqrtf(s0) : 0.f;
+            inv_nrm[base + 8 + g] = s1 > 0.f ? rsqrtf(s1) : 0.f;
+          }
+        }
+        __syncwarp();
+        if (lane == 0) mbar_arrive_one(bar_empty(st));  // this warp is done with the stage
+      }
+      if (!failed && !mbar_wait(bar_tfull(sl), (uint32_t)((k / kMSlots) & 1))) failed = true;
+      if (failed) *s_failed = 1;
+      group_sync();  // every warp's norms are visible
+      const int ai = 32 * q + lane;
+      if (!failed) {
+        tc_fence_after();
+        const float inva = inv_nrm[ai];
+        float bv = -INFINITY;
+        int bi = INT_MAX;
+#pragma unroll
+        for (int h = 0; h < 2; ++h) {
+          const int c0 = 64 * ch2 + 32 * h;
+          float v[32];
+          tmem_ld32(tmem + ((uint32_t)(32 * q) << 16) + (uint32_t)(sl * kUM + c0), v);
+          if (h == 1) {
+            tc_fence_before();
+            __syncwarp();
+            if (lane == 0) mbar_arrive_one(bar_tempty(sl));  // this warp has copied its part of the accumulator
+          }
+#pragma unroll
+          for (int j = 0; j < 32; j += 4) {
+            const float4 ib = *reinterpret_cast<const float4*>(inv_nrm + kUM + c0 + j);
+            const float ibs[4] = {ib.x, ib.y, ib.z, ib.w};
+#pragma unroll
+            for (int e = 0; e < 4; ++e) {
+              float sim = v[j + e] * ibs[e] * inva;
+              sim += 0.f;  // -0 -> +0, so that the ranking orders zeros as equal
+              if (sim > bv) {  // columns in increasing order: the lowest index wins ties
+                bv = sim;
+                bi = c0 + j + e;
+              }
+            }
+          }
+        }
+        gpart_s[ai * 2 + ch2] = bv;
+        gpart_b[ai * 2 + ch2] = bi;
+      }
+      group_sync();  // the partial argmaxes are visible
+      if (*s_failed) {
+        failed = true;
+        break;
+      }
+      if (gtid < kUM) {
+        float bv = gpart_s[2 * gtid];
+        int bi = gpart_b[2 * gtid];
+        const float ps = gpart_s[2 * gtid + 1];
+        const int pb = gpart_b[2 * gtid + 1];
+        if (pb != INT_MAX && (bi == INT_MAX || ps > bv)) {  // the upper column half: strict > keeps the lowest index
+          bv = ps;
+          bi = pb;
+        }
+        const int64_t eslot = (int64_t)lh * a.edge_stride + (int64_t)ch * kUM + gtid;
+        a.edge_sim[eslot] = bi == INT_MAX ? -INFINITY : bv;
+        a.edge_b[eslot] = bi == INT_MAX ? -1 : 2 * bi + 1;
+      }
+    }
+  }
+  if (failed && lane == 0) atomicExch(a.status, 1);
+  tc_fence_before();
+  if (__syncthreads_or(failed)) {
+    // copies and MMAs issued before the wait that gave up may still be in flight: they end on their own
+    for (int i = 0; i < 1000; ++i) __nanosleep(1000);
+    __syncthreads();
+  }
+  if (warp == 0) tmem_dealloc(tmem, 512);
+}
+
 // ---- host side: tensor maps and launch
 
 typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*, const cuuint64_t*,
@@ -552,6 +770,14 @@ cudaError_t launch_round_umma(const RoundArgs& a, int64_t n_full, cudaStream_t s
     if (!make_dst_map(&tm_ko, a.k_dst, a.dst_cap, a.LH) || !make_dst_map(&tm_vo, a.v_dst, a.dst_cap, a.LH)) return cudaErrorInvalidValue;
   } else {
     tm_v = tm_ko = tm_vo = tm_k;  // never used by the matching alone
+  }
+  if (a.mode == kModeMatchOnly) {
+    const size_t msmem = kMBytes + kUAlign;
+    cudaError_t em = cudaFuncSetAttribute(match_umma_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)msmem);
+    if (em != cudaSuccess) return em;
+    const int64_t mctas = std::min<int64_t>(umma_sm_count(), n_full * a.LH);
+    match_umma_kernel<<<(unsigned)mctas, kMThreads, msmem, st>>>(tm_k, a, (int)n_full);
+    return cudaGetLastError();
   }
   const size_t smem = kUBytes + kUAlign;
   cudaError_t e = cudaFuncSetAttribute(round_umma_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
