@@ -23,11 +23,9 @@ def make_pool(n_pages, H, P, D, seed):
     return kp, vp, dp, lp
 
 
-@pytest.mark.parametrize("P,G,with_deg", [(64, 4, True), (32, 1, True), (128, 8, False), (64, 4, False)])
-def test_paged_decode_ragged_batch(P, G, with_deg):
+def paged_decode_case(P, G, with_deg, lens, H):
     from paper_2506_11418_b200 import binding as b
-    H, D = 2, 128
-    lens = [1, 63, 64, 65, 1000, 0, 4100, 2500, 96]
+    D = 128
     n_blocks = [(n + P - 1) // P for n in lens]
     pool = sum(n_blocks) + 7
     kp, vp, dp, lp = make_pool(pool, H, P, D, seed=5)
@@ -60,6 +58,18 @@ def test_paged_decode_ragged_batch(P, G, with_deg):
         ref = O.app_attn_paged(PU.to_np64(q[i]), kpn, vpn, dpn if with_deg else None, tables[i].cpu().numpy(), n, scale)
         err = np.abs(got - ref).max()
         assert err <= 2e-2, f"sequence {i} (len {n}): max abs error {err:.3e}"
+
+
+@pytest.mark.parametrize("P,G,with_deg", [(64, 4, True), (32, 1, True), (128, 8, False), (64, 4, False)])
+def test_paged_decode_ragged_batch(P, G, with_deg):
+    paged_decode_case(P, G, with_deg, [1, 63, 64, 65, 1000, 0, 4100, 2500, 96], 2)
+
+
+@pytest.mark.parametrize("P,G,lens,H", [(64, 4, [20000], 1), (32, 8, [9000, 8200, 8500, 8300], 2), (128, 2, [1000, 64, 0], 2),
+                                        (256, 4, [16416], 8)])
+def test_paged_decode_small_batch(P, G, lens, H):
+    """Few (sequence, head) pairs: the paged kernel in its thread-block-cluster forms (16, 10 and 8 CTAs per pair)."""
+    paged_decode_case(P, G, True, lens, H)
 
 
 def test_pages_compress_write_back_attend():
