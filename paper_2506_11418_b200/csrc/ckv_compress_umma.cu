@@ -506,8 +506,14 @@ __device__ __forceinline__ void mbar_arrive_one(uint32_t bar) {
   asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
 }
 
+// C = 256: an item is one chunk.  C = 128: an item is two consecutive chunks (256 tokens, the same tiles and the same
+// 128 x 128 contraction); a row then only looks at the 64 columns of its own chunk, the other half of S is ignored (a
+// second chunk past the end of the region reads as zeros and is not written).
+template <int C>
 __global__ void __launch_bounds__(kMThreads, 1)
 match_umma_kernel(const __grid_constant__ CUtensorMap tm_k, const RoundArgs a, const int n_full) {
+  static_assert(C == 256 || C == 128, "chunk 256, or pairs of chunks of 128");
+  const int n_blk = C == 256 ? n_full : (n_full + 1) / 2;  // items per slab
   extern __shared__ unsigned char smem_raw[];
   unsigned char* smem = reinterpret_cast<unsigned char*>((reinterpret_cast<uintptr_t>(smem_raw) + kUAlign - 1) & ~(uintptr_t)(kUAlign - 1));
   const uint32_t s_base = smem_u32(smem);
@@ -520,8 +526,8 @@ match_umma_kernel(const __grid_constant__ CUtensorMap tm_k, const RoundArgs a, c
   auto bar_empty = [&](int i) { return s_base + oMBar + 8u * (kMStages + i); };
   auto bar_tfull = [&](int i) { return s_base + oMBar + 8u * (2 * kMStages + i); };
   auto bar_tempty = [&](int i) { return s_base + oMBar + 8u * (2 * kMStages + kMSlots + i); };
-  const int64_t n_items = (int64_t)n_full * a.LH;
-  // this CTA's k-th chunk is item blockIdx.x + k gridDim.x
+  const int64_t n_items = (int64_t)n_blk * a.LH;
+  // this CTA's k-th item is item blockIdx.x + k gridDim.x
   const int64_t my_items = n_items > (int64_t)blockIdx.x ? (n_items - blockIdx.x + gridDim.x - 1) / gridDim.x : 0;
 
   if (tid == 0) {
@@ -548,7 +554,7 @@ match_umma_kernel(const __grid_constant__ CUtensorMap tm_k, const RoundArgs a, c
     if (lane == 0) {
       for (int64_t k = 0; k < my_items && !failed; ++k) {
         const int64_t item = blockIdx.x + k * gridDim.x;
-        const int lh = (int)(item / n_full), ch = (int)(item % n_full);
+        const int lh = (int)(item / n_blk), ch = (int)(item % n_blk);
         const int st = (int)(k % kMStages);
         if (!mbar_wait(bar_empty(st), (uint32_t)(((k / kMStages) & 1) ^ 1))) {
           failed = true;
@@ -600,7 +606,7 @@ match_umma_kernel(const __grid_constant__ CUtensorMap tm_k, const RoundArgs a, c
     };
     for (int64_t k = grp; k < my_items; k += 2) {
       const int64_t item = blockIdx.x + k * gridDim.x;
-      const int lh = (int)(item / n_full), ch = (int)(item % n_full);
+      const int lh = (int)(item / n_blk), ch = (int)(item % n_blk);
       const int st = (int)(k % kMStages), sl = (int)(k % kMSlots);
       float* inv_nrm = inv_all + sl * 256;
       // ---- inverse norms from the staged tile: a warp takes two blocks of 16 tokens (blocks 0-7: A tokens, 8-15: B)
@@ -643,12 +649,14 @@ match_umma_kernel(const __grid_constant__ CUtensorMap tm_k, const RoundArgs a, c
         const float inva = inv_nrm[ai];
         float bv = -INFINITY;
         int bi = INT_MAX;
+        // columns of this thread: 64 (two loads) at chunk 256; at chunk 128 the 32 columns ch2 of the row's own chunk
+        constexpr int NH = C == 256 ? 2 : 1;
 #pragma unroll
-        for (int h = 0; h < 2; ++h) {
-          const int c0 = 64 * ch2 + 32 * h;
+        for (int h = 0; h < NH; ++h) {
+          const int c0 = C == 256 ? 64 * ch2 + 32 * h : 64 * (q >> 1) + 32 * ch2;
           float v[32];
           tmem_ld32(tmem + ((uint32_t)(32 * q) << 16) + (uint32_t)(sl * kUM + c0), v);
-          if (h == 1) {
+          if (h == NH - 1) {
             tc_fence_before();
             __syncwarp();
             if (lane == 0) mbar_arrive_one(bar_tempty(sl));  // this warp has copied its part of the accumulator
@@ -685,9 +693,18 @@ match_umma_kernel(const __grid_constant__ CUtensorMap tm_k, const RoundArgs a, c
           bv = ps;
           bi = pb;
         }
-        const int64_t eslot = (int64_t)lh * a.edge_stride + (int64_t)ch * kUM + gtid;
-        a.edge_sim[eslot] = bi == INT_MAX ? -INFINITY : bv;
-        a.edge_b[eslot] = bi == INT_MAX ? -1 : 2 * bi + 1;
+        if (C == 256) {
+          const int64_t eslot = (int64_t)lh * a.edge_stride + (int64_t)ch * kUM + gtid;
+          a.edge_sim[eslot] = bi == INT_MAX ? -INFINITY : bv;
+          a.edge_b[eslot] = bi == INT_MAX ? -1 : 2 * bi + 1;
+        } else {
+          const int hb = gtid >> 6, chunk = 2 * ch + hb;  // the row's chunk; B indices are local to it
+          if (chunk < n_full) {
+            const int64_t eslot = (int64_t)lh * a.edge_stride + (int64_t)chunk * 64 + (gtid & 63);
+            a.edge_sim[eslot] = bi == INT_MAX ? -INFINITY : bv;
+            a.edge_b[eslot] = bi == INT_MAX ? -1 : 2 * (bi - 64 * hb) + 1;
+          }
+        }
       }
     }
   }
@@ -757,14 +774,16 @@ int umma_sm_count() {
 }  // namespace
 
 bool round_umma_supported(const RoundArgs& a, int dtype, int D) {
-  return dtype == 1 && D == 128 && a.chunk == kUC && a.status != nullptr && encode_tiled_fn() != nullptr;
+  // chunk 256 in every mode; chunk 128 for the matching pass of a round ranked per head
+  const bool shape = a.chunk == kUC || (a.chunk == 128 && a.mode == kModeMatchOnly);
+  return dtype == 1 && D == 128 && shape && a.status != nullptr && encode_tiled_fn() != nullptr;
 }
 
 // The full chunks of a round at chunk 256.  A shorter last chunk, if any, is left to the tile kernel.
 cudaError_t launch_round_umma(const RoundArgs& a, int64_t n_full, cudaStream_t st) {
   if (n_full <= 0) return cudaSuccess;
   CUtensorMap tm_k, tm_v, tm_ko, tm_vo;
-  if (!make_src_map(&tm_k, a.k_src, a.lo, n_full * kUM, a.src_cap, a.LH)) return cudaErrorInvalidValue;
+  if (!make_src_map(&tm_k, a.k_src, a.lo, n_full * (a.chunk / 2), a.src_cap, a.LH)) return cudaErrorInvalidValue;
   if (a.mode != kModeMatchOnly) {
     if (!make_src_map(&tm_v, a.v_src, a.lo, n_full * kUM, a.src_cap, a.LH)) return cudaErrorInvalidValue;
     if (!make_dst_map(&tm_ko, a.k_dst, a.dst_cap, a.LH) || !make_dst_map(&tm_vo, a.v_dst, a.dst_cap, a.LH)) return cudaErrorInvalidValue;
@@ -773,10 +792,11 @@ cudaError_t launch_round_umma(const RoundArgs& a, int64_t n_full, cudaStream_t s
   }
   if (a.mode == kModeMatchOnly) {
     const size_t msmem = kMBytes + kUAlign;
-    cudaError_t em = cudaFuncSetAttribute(match_umma_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)msmem);
+    auto kern = a.chunk == kUC ? match_umma_kernel<256> : match_umma_kernel<128>;
+    cudaError_t em = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)msmem);
     if (em != cudaSuccess) return em;
-    const int64_t mctas = std::min<int64_t>(umma_sm_count(), n_full * a.LH);
-    match_umma_kernel<<<(unsigned)mctas, kMThreads, msmem, st>>>(tm_k, a, (int)n_full);
+    const int64_t items = (a.chunk == kUC ? n_full : (n_full + 1) / 2) * a.LH;
+    kern<<<(unsigned)std::min<int64_t>(umma_sm_count(), items), kMThreads, msmem, st>>>(tm_k, a, (int)n_full);
     return cudaGetLastError();
   }
   const size_t smem = kUBytes + kUAlign;
