@@ -418,6 +418,9 @@ def bench_compress_variants(b, synth, dev, K, V, peak_gbs, with_128k):
         ("chunk256 ratio1", P(chunk=256, n_sink=0, n_recent=0, n_rounds_max=1, r_init=1.0, r_decay=0.0, r_min=1.0)),
         ("chunk64 paper schedule to 25%", P(chunk=64, budget=s // 4, **paper)),
         ("chunk256 paper schedule to 25%", P(chunk=256, budget=s // 4, **paper)),
+        ("chunk128 ratio0.8 ranked per head", P(chunk=128, n_sink=16, n_recent=64, n_rounds_max=1, r_init=0.8, r_decay=0.0, r_min=0.8)),
+        ("chunk256 ratio0.8 ranked per head", P(chunk=256, n_sink=16, n_recent=64, n_rounds_max=1, r_init=0.8, r_decay=0.0, r_min=0.8)),
+        ("chunk128 paper schedule to 25%", P(chunk=128, budget=s // 4, **paper)),
     ]
     res = {}
 
