@@ -166,8 +166,10 @@ struct Buf {  // one cache buffer a round reads or writes
 };
 
 // One clustering round src -> dst (Sec. 5.2, Sec. 5.3, Eq. 5), sinks and recent tokens copied verbatim.
+// first_chunk > 0 (chunked rounds that merge every edge only): the chunks before it are someone else's work.
 cudaError_t run_round(const RoundPlan& rp, const Buf& src, const Buf& dst, int LH, int D, int dtype, int chunk,
-                      int32_t* assign, int64_t assign_stride, const Workspace& w, unsigned char* ws, cudaStream_t st) {
+                      int32_t* assign, int64_t assign_stride, const Workspace& w, unsigned char* ws, cudaStream_t st,
+                      int32_t first_chunk = 0) {
   cudaError_t e;
   CopyArgs c{};
   c.k_src = src.k; c.v_src = src.v; c.deg_src = src.deg;
@@ -207,7 +209,8 @@ cudaError_t run_round(const RoundPlan& rp, const Buf& src, const Buf& dst, int L
     return launch_bsm_merge(a, ws + w.bsm, st);
   }
   a.chunk = chunk; a.n_chunks = rp.n_chunks;
-  a.chunk_first = 0; a.n_launch = rp.n_chunks;
+  a.chunk_first = first_chunk; a.n_launch = rp.n_chunks - first_chunk;
+  if (a.n_launch <= 0) return cudaSuccess;
   a.m_full = rp.m_full; a.m_tail = rp.m_tail;
   a.out_stride = chunk - rp.m_full;
   a.out_lo = rp.lo;
@@ -220,6 +223,7 @@ cudaError_t run_round(const RoundPlan& rp, const Buf& src, const Buf& dst, int L
     const bool fast = round_fast_supported(x, dtype, D), umma = !fast && round_umma_supported(x, dtype, D);
     if (fast || umma) {
       const int64_t n_full = (rp.hi - rp.lo) / chunk;
+      if (!fast && first_chunk > 0) return cudaErrorInvalidValue;
       cudaError_t err = fast ? launch_round_fast(x, n_full, st) : launch_round_umma(x, n_full, st);
       if (err != cudaSuccess || rp.n_chunks == n_full) return err;
       x.chunk_first = (int32_t)n_full;
@@ -259,6 +263,35 @@ int run_plan(const std::vector<RoundPlan>& plan, const Buf& src, const Buf& dst,
           reinterpret_cast<float*>(ws + w.tmp_logdeg), w.tmp_cap};
   Buf cur = src;
   for (size_t j = 0; j < R; ++j) {
+    // Two rounds in one pass: rounds j and j + 1 both merge every edge at chunk 64 and the source degrees are all
+    // one.  Pairs of full round-1 chunks are exactly the full round-2 chunks they feed; those go through the fused
+    // kernel straight into the second round's target.  What is left (an odd chunk, the shorter last chunk, sinks and
+    // recent tokens) takes the two rounds one after the other.
+    if (j + 1 < R && cur.deg == nullptr && plan[j].mode == kModeAll && plan[j + 1].mode == kModeAll &&
+        plan[j].lo == plan[j + 1].lo && round_fused2_supported(dtype, D, chunk)) {
+      const int64_t units = (plan[j].hi - plan[j].lo) / chunk / 2;
+      if (units > 0) {
+        const Buf& t1 = round_targets_dst(j, R) ? dst : tmp;
+        const Buf& t2 = round_targets_dst(j + 1, R) ? dst : tmp;
+        int32_t* step2 = assign ? reinterpret_cast<int32_t*>(ws + w.assign_step) : nullptr;
+        RoundArgs f{};
+        f.k_src = cur.k; f.v_src = cur.v;
+        f.k_dst = t2.k; f.v_dst = t2.v; f.deg_dst = t2.deg; f.logdeg_dst = t2.logdeg;
+        f.assign = assign; f.assign_stride = src_len;  // j == 0 here: only the caller's source has no degrees
+        f.src_cap = cur.cap; f.dst_cap = t2.cap;
+        f.lo = plan[j].lo; f.LH = LH;
+        f.status = reinterpret_cast<int32_t*>(ws);
+        if (launch_round_fused2(f, units, step2, w.assign_stride, st) != cudaSuccess) return CKV_ERR_CUDA;
+        e = run_round(plan[j], cur, t1, LH, D, dtype, chunk, assign, src_len, w, ws, st, (int32_t)(2 * units));
+        if (e != cudaSuccess) return CKV_ERR_CUDA;
+        e = run_round(plan[j + 1], t1, t2, LH, D, dtype, chunk, step2, w.assign_stride, w, ws, st, (int32_t)units);
+        if (e != cudaSuccess) return CKV_ERR_CUDA;
+        if (assign && launch_compose_assign(assign, step2, src_len, w.assign_stride, LH, st) != cudaSuccess) return CKV_ERR_CUDA;
+        cur = t2;
+        ++j;
+        continue;
+      }
+    }
     const Buf& target = round_targets_dst(j, R) ? dst : tmp;
     int32_t* step = nullptr;
     int64_t step_stride = 0;

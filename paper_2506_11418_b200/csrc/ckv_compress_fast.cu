@@ -449,7 +449,11 @@ bool round_fast_supported(const RoundArgs& a, int dtype, int D) {
 
 // The full chunks of a round in any mode.  The shorter last chunk, if any, is left to the tile kernel.
 cudaError_t launch_round_fast(const RoundArgs& r, int64_t n_full, cudaStream_t st) {
+  // r.chunk_first > 0: only the full chunks from that one on (modes whose output offsets are a multiple of the chunk index)
+  const int64_t first = r.chunk_first;
+  n_full -= first;
   if (n_full <= 0) return cudaSuccess;
+  if (first > 0 && r.mode != kModeAll && r.mode != kModeChunkTopM) return cudaErrorInvalidValue;
   FastArgs a{};
   a.k_src = static_cast<const __nv_bfloat16*>(r.k_src);
   a.v_src = static_cast<const __nv_bfloat16*>(r.v_src);
@@ -462,8 +466,8 @@ cudaError_t launch_round_fast(const RoundArgs& r, int64_t n_full, cudaStream_t s
   a.assign_stride = r.assign_stride;
   a.src_cap = r.src_cap;
   a.dst_cap = r.dst_cap;
-  a.lo = r.lo;
-  a.out_lo = r.out_lo;
+  a.lo = r.lo + first * kC;
+  a.out_lo = r.out_lo + first * r.out_stride;
   a.n_full = n_full;
   a.n_items = n_full * r.LH;
   a.status = r.status;

@@ -123,6 +123,10 @@ bool bsm_supported(int dtype, int D);
 size_t bsm_workspace_bytes(int64_t LH, int64_t mid);
 cudaError_t launch_bsm_match(const RoundArgs& a, void* scratch, cudaStream_t st);  // a.lo, a.hi: the middle region
 cudaError_t launch_bsm_merge(const RoundArgs& a, void* scratch, cudaStream_t st);
+// two consecutive ratio-1 rounds at chunk 64 in one pass (source degrees all one): rounds j, j + 1 on the first
+// 2 * units chunks of every slab; assign2 / stride2: the second round's slot map when a.assign is given
+bool round_fused2_supported(int dtype, int D, int chunk);
+cudaError_t launch_round_fused2(const RoundArgs& a, int64_t units, int32_t* assign2, int64_t stride2, cudaStream_t st);
 bool round_tile_supported(const RoundArgs& a, int dtype, int D);
 cudaError_t launch_round_tile(const RoundArgs& a, cudaStream_t st);
 

@@ -215,6 +215,29 @@ def test_two_rounds_ratio_one(dtype):
     assert st["rounds"] == 2
 
 
+@pytest.mark.parametrize("s,sink,recent,rounds", [(4096 + 64, 0, 0, 2), (4096 + 64 + 37, 0, 0, 2), (3000, 16, 64, 2), (130, 0, 0, 2),
+                                                 (127, 0, 0, 2), (256 + 5, 3, 0, 2), (8192 + 192, 16, 64, 3), (20000, 0, 7, 4)])
+def test_rounds_in_one_pass_edges(s, sink, recent, rounds):
+    """Two ratio-1 rounds at chunk 64 on a cache without degrees run as one pass over pairs of chunks; an odd chunk, a
+    shorter last chunk, sinks and recent tokens take the two rounds one after the other, later rounds follow."""
+    b = B()
+    p = b.Params(chunk=64, n_sink=sink, n_recent=recent, n_rounds_max=rounds, r_init=1.0, r_decay=0.0, r_min=1.0, select=b.SELECT_CHUNK)
+    st = multi_round_case(2, 3, s, "bf16", p, seed=77 + s)
+    assert st["rounds"] == rounds
+
+
+def test_rounds_in_one_pass_without_slot_map():
+    """The same call with and without the optional slot map gives the same cache, bit for bit."""
+    b = B()
+    p = b.Params(chunk=64, n_sink=5, n_recent=9, n_rounds_max=2, r_init=1.0, r_decay=0.0, r_min=1.0, select=b.SELECT_GLOBAL)
+    K, V, _ = make_inputs(2, 2, 5000, "bf16", seed=91)
+    d1, _, _ = run_gpu_prefill(K, V, None, p, want_assign=True)
+    d2, _, _ = run_gpu_prefill(K, V, None, p, want_assign=False)
+    n = d1.len
+    assert d2.len == n and torch.equal(d1.k[:, :, :n], d2.k[:, :, :n]) and torch.equal(d1.v[:, :, :n], d2.v[:, :, :n])
+    assert torch.equal(d1.deg[:, :, :n], d2.deg[:, :, :n]) and torch.equal(d1.logdeg[:, :, :n], d2.logdeg[:, :, :n])
+
+
 @pytest.mark.parametrize("dtype", ["f32", "bf16"])
 @pytest.mark.parametrize("select", [0, 1])
 def test_paper_schedule_to_quarter_budget(dtype, select):
