@@ -59,57 +59,43 @@ __device__ __forceinline__ uint32_t f_addr(uint32_t tile, int row, int c16) {
   return tile + (uint32_t)(c16 >> 3) * kFHalf + (uint32_t)row * 128u + (uint32_t)(((c16 & 7) ^ (row & 7)) << 4);
 }
 
-// Sec. 5.2 on one chunk (rows row0 .. row0 + 63 of the tile; A = even rows, B = odd rows): returns, in lane i, the
-// B index (0..31) that A token i is matched to.
-__device__ __forceinline__ int match64(uint32_t tile, int row0, int lane) {
+// Sec. 5.2 on one chunk: A tokens in rows row_a .. + 31 of the tile, B tokens in rows row_b .. + 31.  Returns, in lane
+// i, the B index (0..31) that A token i is matched to.
+__device__ __forceinline__ int match64(uint32_t tile, int row_a, int row_b, int lane) {
   const int g = lane >> 2, t = lane & 3;
   float acc[2][4][4];   // [m tile][n tile][c]: A token 16 mt + g (+8), B index 8 nt + 2t (+1)
   float nacc[2][2][4];  // B B^T diagonals
+  // lane l supplies the address of row l % 8 of matrix l / 8.  A operand (16 tokens x 16 columns): matrices = (tokens
+  // 0-7, 8-15) x (columns 0-7, 8-15) in the order a0 a1 a2 a3.  B operand of two n tiles: (tokens 0-7 | columns 0-7,
+  // 8-15), then the next eight tokens: b0, b1 of n tile 2p, then of 2p + 1.
+  const int a_row = row_a + (lane & 7) + ((lane >> 3) & 1) * 8, a_c = lane >> 4;
+  const int b_row = row_b + (lane & 7) + (lane >> 4) * 8, b_c = (lane >> 3) & 1;
 #pragma unroll
-  for (int i = 0; i < 2; ++i)
+  for (int kk = 0; kk < 8; ++kk) {  // 16 columns per step
+    uint32_t fa[2][4], fb[2][4];
 #pragma unroll
-    for (int j = 0; j < 4; ++j)
+    for (int mt = 0; mt < 2; ++mt) ldsm_x4(f_addr(tile, a_row + 16 * mt, 2 * kk + a_c), fa[mt]);
 #pragma unroll
-      for (int c = 0; c < 4; ++c) acc[i][j][c] = 0.f;
-#pragma unroll
-  for (int i = 0; i < 2; ++i)
-#pragma unroll
-    for (int j = 0; j < 2; ++j)
-#pragma unroll
-      for (int c = 0; c < 4; ++c) nacc[i][j][c] = 0.f;
-
-#pragma unroll
-  for (int kp = 0; kp < 4; ++kp) {
-    // each lane reads 16 contiguous bytes of a row (elements 32 kp + 8 t .. + 7); the same permutation of the
-    // contraction index on both operands leaves the dot products unchanged
-    const int c16 = 4 * kp + t;
-    uint4 ra[2][2], rb[4];
+    for (int p = 0; p < 2; ++p) ldsm_x4(f_addr(tile, b_row + 16 * p, 2 * kk + b_c), fb[p]);
 #pragma unroll
     for (int mt = 0; mt < 2; ++mt)
 #pragma unroll
-      for (int hi = 0; hi < 2; ++hi) ld_shared_v4(f_addr(tile, row0 + 2 * (16 * mt + 8 * hi + g), c16), ra[mt][hi]);
-#pragma unroll
-    for (int nt = 0; nt < 4; ++nt) ld_shared_v4(f_addr(tile, row0 + 2 * (8 * nt + g) + 1, c16), rb[nt]);
-#pragma unroll
-    for (int ks = 0; ks < 2; ++ks) {
-      uint32_t b0[4], b1[4];
-#pragma unroll
       for (int nt = 0; nt < 4; ++nt) {
-        b0[nt] = ks ? rb[nt].z : rb[nt].x;
-        b1[nt] = ks ? rb[nt].w : rb[nt].y;
+        const uint32_t b0 = fb[nt >> 1][2 * (nt & 1)], b1 = fb[nt >> 1][2 * (nt & 1) + 1];
+        if (kk == 0)
+          mma_bf16_first(acc[mt][nt], fa[mt][0], fa[mt][1], fa[mt][2], fa[mt][3], b0, b1);
+        else
+          mma_bf16(acc[mt][nt], fa[mt][0], fa[mt][1], fa[mt][2], fa[mt][3], b0, b1);
       }
+    // B B^T on pairs of n tiles: rows = B indices 16 p + g (+8); the diagonal holds the squared norms
 #pragma unroll
-      for (int mt = 0; mt < 2; ++mt) {
-        const uint32_t a0 = ks ? ra[mt][0].z : ra[mt][0].x, a1 = ks ? ra[mt][1].z : ra[mt][1].x;
-        const uint32_t a2 = ks ? ra[mt][0].w : ra[mt][0].y, a3 = ks ? ra[mt][1].w : ra[mt][1].y;
-#pragma unroll
-        for (int nt = 0; nt < 4; ++nt) mma_bf16(acc[mt][nt], a0, a1, a2, a3, b0[nt], b1[nt]);
-      }
-      // B B^T on pairs of n tiles: rows = B indices 16 p + g (+8); the diagonal holds the squared norms
-#pragma unroll
-      for (int p = 0; p < 2; ++p) {
-        mma_bf16(nacc[p][0], b0[2 * p], b0[2 * p + 1], b1[2 * p], b1[2 * p + 1], b0[2 * p], b1[2 * p]);
-        mma_bf16(nacc[p][1], b0[2 * p], b0[2 * p + 1], b1[2 * p], b1[2 * p + 1], b0[2 * p + 1], b1[2 * p + 1]);
+    for (int p = 0; p < 2; ++p) {
+      if (kk == 0) {
+        mma_bf16_first(nacc[p][0], fb[p][0], fb[p][2], fb[p][1], fb[p][3], fb[p][0], fb[p][1]);
+        mma_bf16_first(nacc[p][1], fb[p][0], fb[p][2], fb[p][1], fb[p][3], fb[p][2], fb[p][3]);
+      } else {
+        mma_bf16(nacc[p][0], fb[p][0], fb[p][2], fb[p][1], fb[p][3], fb[p][0], fb[p][1]);
+        mma_bf16(nacc[p][1], fb[p][0], fb[p][2], fb[p][1], fb[p][3], fb[p][2], fb[p][3]);
       }
     }
   }
@@ -124,7 +110,7 @@ __device__ __forceinline__ int match64(uint32_t tile, int row0, int lane) {
     inv1[nt] = __shfl_sync(0xffffffffu, inv, 9 * t + 4);    // B index 8 nt + 2t + 1 lives in lane 4 (2t + 1) + t
   }
   // row argmax; dividing a row by |a| > 0 cannot change it
-  int row_b[2][2];
+  int row_best[2][2];
 #pragma unroll
   for (int mt = 0; mt < 2; ++mt)
 #pragma unroll
@@ -143,7 +129,7 @@ __device__ __forceinline__ int match64(uint32_t tile, int row0, int lane) {
         const int oi = __shfl_xor_sync(0xffffffffu, bi, o);
         if (ov > bv || (ov == bv && oi < bi)) { bv = ov; bi = oi; }
       }
-      row_b[mt][hi] = bi;
+      row_best[mt][hi] = bi;
     }
   // lane = A index i takes row i = 16 mt + 8 hi + g from the quad of g = i & 7
   int my_best = 0;
@@ -152,102 +138,110 @@ __device__ __forceinline__ int match64(uint32_t tile, int row0, int lane) {
   for (int mt = 0; mt < 2; ++mt)
 #pragma unroll
     for (int hi = 0; hi < 2; ++hi) {
-      const int vb = __shfl_sync(0xffffffffu, row_b[mt][hi], src);
+      const int vb = __shfl_sync(0xffffffffu, row_best[mt][hi], src);
       if (which == 2 * mt + hi) my_best = vb;
     }
   return my_best & 31;  // a row of NaNs has no maximum: stay inside the chunk
 }
 
-// Eq. 5 on one chunk of one tensor, in place: tokens = rows src_row0 .. + 63 of the tile (A = even, B = odd), lane i
-// holds the B index A token i merges into; the 32 centroids go to rows dst_row0 .. + 31.  deg_in: the 64 tokens'
-// degrees (null: all one); deg_out: the 32 summed degrees.
-__device__ __forceinline__ void merge64(uint32_t tile, int src_row0, int dst_row0, int my_best, const int* deg_in,
-                                        const int* deg_out, int lane) {
+// Eq. 5 on one chunk of one tensor, in place.  A tokens in rows row_a .. + 31, B tokens in rows row_b .. + 31; lane i
+// holds the B index A token i merges into, lane j the summed degree n' of B token j's cluster.  deg_a / deg_b: degrees
+// of the A and B tokens, element stride 2 (null: all one).  Centroid j goes to row dst0 + j (dst_split false) or, split
+// by parity for the next round, to row dst0 + j / 2 (j even) / dst0 + 64 + j / 2 (j odd).
+__device__ __forceinline__ void merge64(uint32_t tile, int row_a, int row_b, int dst0, bool dst_split, int my_best, int my_n,
+                                        const int* deg_a, const int* deg_b, int lane) {
   const int g = lane >> 2, t = lane & 3;
-  // which 16 x 16 blocks (m tile, k step) of W hold an entry: the B tokens' own terms, and the edges
-  const unsigned need = __reduce_or_sync(0xffffffffu, 1u << (((my_best >> 4) << 2) + (lane >> 3))) | 0xc3u;
-  // W as the row-major A operand: rows = B index, columns = token of the chunk
-  uint32_t wf[2][4][4];
+  // W as the row-major A operand: rows = B index, columns = the chunk's tokens, A tokens first (k steps 0, 1), then B
+  // tokens (k steps 2, 3).  The B tokens' own terms are the diagonal of blocks (m tile 0, step 2) and (1, 3); which
+  // blocks of the A part hold an edge is found by a vote.
+  const unsigned need = __reduce_or_sync(0xffffffffu, 1u << (((my_best >> 4) << 1) + (lane >> 4)));
+  uint32_t wa[2][2][4];  // [m tile][k step][register]
 #pragma unroll
-  for (int ks = 0; ks < 4; ++ks) {
-    const int i0 = 8 * ks + t, i1 = i0 + 4;  // A token i (token 2i) and B token i (token 2i + 1) share a register
-    const int tg0 = __shfl_sync(0xffffffffu, my_best, i0), tg1 = __shfl_sync(0xffffffffu, my_best, i1);
-    uint32_t wa0 = kOneBf16, wb0 = kOneBf16 << 16, wa1 = kOneBf16, wb1 = kOneBf16 << 16;
-    if (deg_in) {
-      wa0 = __float_as_uint((float)deg_in[2 * i0]) >> 16;
-      wb0 = __float_as_uint((float)deg_in[2 * i0 + 1]) & 0xffff0000u;
-      wa1 = __float_as_uint((float)deg_in[2 * i1]) >> 16;
-      wb1 = __float_as_uint((float)deg_in[2 * i1 + 1]) & 0xffff0000u;
+  for (int ks = 0; ks < 2; ++ks) {
+    const int i0 = 16 * ks + 2 * t;  // A tokens i0, i0 + 1 (columns 2t, 2t + 1) and i0 + 8, i0 + 9
+    const int tg0 = __shfl_sync(0xffffffffu, my_best, i0), tg1 = __shfl_sync(0xffffffffu, my_best, i0 + 1);
+    const int tg2 = __shfl_sync(0xffffffffu, my_best, i0 + 8), tg3 = __shfl_sync(0xffffffffu, my_best, i0 + 9);
+    uint32_t w0 = kOneBf16, w1 = kOneBf16 << 16, w2 = kOneBf16, w3 = kOneBf16 << 16;
+    if (deg_a) {  // degrees up to 256 are exact in bf16
+      w0 = __float_as_uint((float)deg_a[2 * i0]) >> 16;
+      w1 = __float_as_uint((float)deg_a[2 * i0 + 2]) & 0xffff0000u;
+      w2 = __float_as_uint((float)deg_a[2 * i0 + 16]) >> 16;
+      w3 = __float_as_uint((float)deg_a[2 * i0 + 18]) & 0xffff0000u;
     }
 #pragma unroll
     for (int mt = 0; mt < 2; ++mt) {
       const int r = 16 * mt + g;
-      wf[mt][ks][0] = (tg0 == r ? wa0 : 0u) | (i0 == r ? wb0 : 0u);
-      wf[mt][ks][1] = (tg0 == r + 8 ? wa0 : 0u) | (i0 == r + 8 ? wb0 : 0u);
-      wf[mt][ks][2] = (tg1 == r ? wa1 : 0u) | (i1 == r ? wb1 : 0u);
-      wf[mt][ks][3] = (tg1 == r + 8 ? wa1 : 0u) | (i1 == r + 8 ? wb1 : 0u);
+      wa[mt][ks][0] = (tg0 == r ? w0 : 0u) | (tg1 == r ? w1 : 0u);
+      wa[mt][ks][1] = (tg0 == r + 8 ? w0 : 0u) | (tg1 == r + 8 ? w1 : 0u);
+      wa[mt][ks][2] = (tg2 == r ? w2 : 0u) | (tg3 == r ? w3 : 0u);
+      wa[mt][ks][3] = (tg2 == r + 8 ? w2 : 0u) | (tg3 == r + 8 ? w3 : 0u);
     }
   }
+  // own terms: row g of the diagonal block has its entry in column g: register 0 (rows 0-7) and 3 (rows 8-15) of the
+  // lane with 2t == g (low half) or 2t + 1 == g (high half)
+  uint32_t wd[2][2];  // [m tile][rows 0-7 / 8-15]
+#pragma unroll
+  for (int mt = 0; mt < 2; ++mt)
+#pragma unroll
+    for (int hi = 0; hi < 2; ++hi) {
+      uint32_t w = kOneBf16;
+      if (deg_b) w = __float_as_uint((float)deg_b[2 * (16 * mt + 8 * hi + g)]) >> 16;
+      wd[mt][hi] = (g == 2 * t) ? w : ((g == 2 * t + 1) ? (w << 16) : 0u);
+    }
+  const float my_inv = 1.0f / (float)my_n;
   float inv[2][2];
 #pragma unroll
   for (int mt = 0; mt < 2; ++mt)
 #pragma unroll
-    for (int hi = 0; hi < 2; ++hi) inv[mt][hi] = 1.0f / (float)deg_out[16 * mt + 8 * hi + g];
+    for (int hi = 0; hi < 2; ++hi) inv[mt][hi] = __shfl_sync(0xffffffffu, my_inv, 16 * mt + 8 * hi + g);
 
+  // ldmatrix.trans: lane l supplies row l % 8 (+8 for odd l / 8) of the sixteen tokens of a k step, 16-byte piece
+  // 2 jp + l / 16 -> b0, b1 of n tile 2 jp, then of 2 jp + 1.  stmatrix: row l % 8 of the eight output rows, piece l / 8.
+  const int k_row = (lane & 7) + ((lane >> 3) & 1) * 8, k_c = lane >> 4;
 #pragma unroll 1
-  for (int h = 0; h < 2; ++h) {
-    // columns 64 h .. + 63.  n tile j, column n = g  <->  tile column 64 h + 8 g + j: a lane's 16-byte piece feeds
-    // eight n tiles, and an accumulator row ends up with 16 contiguous columns per lane
+  for (int h = 0; h < 2; ++h) {  // columns 64 h .. + 63: n tile j = columns 8 j .. + 7 of the half
     float acc[2][8][4];
 #pragma unroll
-    for (int mt = 0; mt < 2; ++mt)
-#pragma unroll
-      for (int j = 0; j < 8; ++j)
-#pragma unroll
-        for (int c = 0; c < 4; ++c) acc[mt][j][c] = 0.f;
-#pragma unroll
     for (int ks = 0; ks < 4; ++ks) {
-      const int r0 = src_row0 + 16 * ks + 2 * t;
-      uint4 x[4];
-      ld_shared_v4(f_addr(tile, r0, 8 * h + g), x[0]);
-      ld_shared_v4(f_addr(tile, r0 + 1, 8 * h + g), x[1]);
-      ld_shared_v4(f_addr(tile, r0 + 8, 8 * h + g), x[2]);
-      ld_shared_v4(f_addr(tile, r0 + 9, 8 * h + g), x[3]);
-      const uint32_t x0[4] = {x[0].x, x[0].y, x[0].z, x[0].w}, x1[4] = {x[1].x, x[1].y, x[1].z, x[1].w};
-      const uint32_t x2[4] = {x[2].x, x[2].y, x[2].z, x[2].w}, x3[4] = {x[3].x, x[3].y, x[3].z, x[3].w};
-      uint32_t b0[8], b1[8];  // (token 2t, token 2t + 1) and (token 2t + 8, token 2t + 9) of column 8 g + j
+      const int step = (ks + 2) & 3;  // the B tokens first (steps 2, 3): their blocks are always there and start the sums
+      if (step < 2 && !((need >> step) & 5u)) continue;
+      const int base = step < 2 ? row_a + 16 * step : row_b + 16 * (step - 2);
+      uint32_t fb[4][4];
 #pragma unroll
-      for (int w = 0; w < 4; ++w) {
-        b0[2 * w] = __byte_perm(x0[w], x1[w], 0x5410);
-        b0[2 * w + 1] = __byte_perm(x0[w], x1[w], 0x7632);
-        b1[2 * w] = __byte_perm(x2[w], x3[w], 0x5410);
-        b1[2 * w + 1] = __byte_perm(x2[w], x3[w], 0x7632);
+      for (int jp = 0; jp < 4; ++jp) ldsm_x4_trans(f_addr(tile, base + k_row, 8 * h + 2 * jp + k_c), fb[jp]);
+      if (step >= 2) {
+        const int mt = step - 2;
+#pragma unroll
+        for (int j = 0; j < 8; ++j)
+          mma_bf16_first(acc[mt][j], wd[mt][0], 0u, 0u, wd[mt][1], fb[j >> 1][2 * (j & 1)], fb[j >> 1][2 * (j & 1) + 1]);
+      } else {
+#pragma unroll
+        for (int mt = 0; mt < 2; ++mt)
+          if ((need >> (2 * mt + step)) & 1u) {
+#pragma unroll
+            for (int j = 0; j < 8; ++j)
+              mma_bf16(acc[mt][j], wa[mt][step][0], wa[mt][step][1], wa[mt][step][2], wa[mt][step][3], fb[j >> 1][2 * (j & 1)],
+                       fb[j >> 1][2 * (j & 1) + 1]);
+          }
       }
-#pragma unroll
-      for (int mt = 0; mt < 2; ++mt)
-        if ((need >> (4 * mt + ks)) & 1u) {
-#pragma unroll
-          for (int j = 0; j < 8; ++j) mma_bf16(acc[mt][j], wf[mt][ks][0], wf[mt][ks][1], wf[mt][ks][2], wf[mt][ks][3], b0[j], b1[j]);
-        }
     }
     __syncwarp();  // every lane has read this half's rows: they may be overwritten
 #pragma unroll
     for (int mt = 0; mt < 2; ++mt)
 #pragma unroll
       for (int hi = 0; hi < 2; ++hi) {
-        const int row = dst_row0 + 16 * mt + 8 * hi + g;
         const float s = inv[mt][hi];
-        uint4 o0, o1;  // columns 16 t .. + 7 and 16 t + 8 .. + 15 of this half
-        o0.x = pack_bf16x2(acc[mt][0][2 * hi] * s, acc[mt][1][2 * hi] * s);
-        o0.y = pack_bf16x2(acc[mt][2][2 * hi] * s, acc[mt][3][2 * hi] * s);
-        o0.z = pack_bf16x2(acc[mt][4][2 * hi] * s, acc[mt][5][2 * hi] * s);
-        o0.w = pack_bf16x2(acc[mt][6][2 * hi] * s, acc[mt][7][2 * hi] * s);
-        o1.x = pack_bf16x2(acc[mt][0][2 * hi + 1] * s, acc[mt][1][2 * hi + 1] * s);
-        o1.y = pack_bf16x2(acc[mt][2][2 * hi + 1] * s, acc[mt][3][2 * hi + 1] * s);
-        o1.z = pack_bf16x2(acc[mt][4][2 * hi + 1] * s, acc[mt][5][2 * hi + 1] * s);
-        o1.w = pack_bf16x2(acc[mt][6][2 * hi + 1] * s, acc[mt][7][2 * hi + 1] * s);
-        st_shared_v4(f_addr(tile, row, 8 * h + 2 * t), o0);
-        st_shared_v4(f_addr(tile, row, 8 * h + 2 * t + 1), o1);
+        uint32_t o[8];
+#pragma unroll
+        for (int j = 0; j < 8; ++j) {
+          float x, y;
+          mul_f32x2(x, y, acc[mt][j][2 * hi], acc[mt][j][2 * hi + 1], s);
+          o[j] = pack_bf16x2(x, y);
+        }
+        const int j_out = 16 * mt + 8 * hi + (lane & 7);
+        const int row = dst_split ? dst0 + ((j_out & 1) << 6) + (j_out >> 1) : dst0 + j_out;
+        stsm_x4(f_addr(tile, row, 8 * h + (lane >> 3)), o[0], o[1], o[2], o[3]);
+        stsm_x4(f_addr(tile, row, 8 * h + 4 + (lane >> 3)), o[4], o[5], o[6], o[7]);
       }
   }
   __syncwarp();
@@ -276,12 +270,15 @@ round_fused2_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_const
 
   const int64_t stride = (int64_t)gridDim.x * kFWarps;
   int64_t item = (int64_t)blockIdx.x * kFWarps + warp;
+  // a tile: per half of the columns, the unit's 64 A tokens (1st, 3rd, ... token) in rows 0-63, its B tokens in 64-127
   auto fetch = [&](const CUtensorMap* tm, int64_t it) {
     const uint32_t lh = (uint32_t)it / a.units, u = (uint32_t)it - lh * a.units;
-    const int tok = (int)(a.lo + (int64_t)u * kFUnit);
+    const int pair = (int)(u * (kFUnit / 2));
     mbar_arrive_expect_tx(bar, kFStage);
-    tma_load_3d(tile, tm, 0, tok, (int)lh, bar);
-    tma_load_3d(tile + kFHalf, tm, 64, tok, (int)lh, bar);
+#pragma unroll
+    for (int h = 0; h < 2; ++h)
+#pragma unroll
+      for (int par = 0; par < 2; ++par) tma_load_4d(tile + h * kFHalf + par * (kFHalf / 2), tm, 64 * h, par, pair, (int)lh, bar);
   };
   if (item < a.n_items && lane == 0) fetch(&tm_k, item);
 
@@ -300,20 +297,16 @@ round_fused2_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_const
       parity ^= 1;
       __syncwarp();
 #pragma unroll 1
-      for (int it = 0; it < 3; ++it) {  // round 1 on rows 0-63 and 64-127, then round 2 on the 64 centroids
-        const int row0 = it == 1 ? 64 : 0, dst0 = it == 1 ? 32 : 0;
-        int best;
+      for (int it = 0; it < 3; ++it) {  // round 1 on the unit's first and second chunk, then round 2 on the 64 centroids
+        // round 1 leaves centroid j of chunk q where round 2 finds it: position 32 q + j of the 64, split by parity
+        const int row_a = it == 1 ? 32 : 0, row_b = 64 + row_a, dst0 = it == 0 ? 0 : (it == 1 ? 16 : 0);
+        int best, n;
         if (ph == 0) {
-          best = match64(tile, row0, lane);
-          if (it < 2) {
-            d1[32 * it + lane] = 1;
-            __syncwarp();
-            atomicAdd(&d1[32 * it + best], 1);
-          } else {
-            d2[lane] = d1[2 * lane + 1];
-            __syncwarp();
-            atomicAdd(&d2[best], d1[2 * lane]);
-          }
+          best = match64(tile, row_a, row_b, lane);
+          int* d = it < 2 ? d1 + 32 * it : d2;
+          d[lane] = it < 2 ? 1 : d1[2 * lane + 1];
+          __syncwarp();
+          atomicAdd(&d[best], it < 2 ? 1 : d1[2 * lane]);
           __syncwarp();
           if (it == 0) best_q0 = best;
           if (it == 1) best_q1 = best;
@@ -321,7 +314,8 @@ round_fused2_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_const
         } else {
           best = it == 0 ? best_q0 : (it == 1 ? best_q1 : best_r2);
         }
-        merge64(tile, row0, dst0, best, it < 2 ? nullptr : d1, it < 2 ? d1 + 32 * it : d2, lane);
+        n = it < 2 ? d1[32 * it + lane] : d2[lane];
+        merge64(tile, row_a, row_b, dst0, it < 2, best, n, it < 2 ? nullptr : d1, it < 2 ? nullptr : d1 + 1, lane);
       }
       fence_async_smem();  // the TMA store reads the rows through the asynchronous proxy
       __syncwarp();
@@ -377,6 +371,19 @@ EncodeTiledFn fused_encode_fn() {
   return fn;
 }
 
+// source view: (column 128, parity 2, token pair, slab) from token `lo` on; box = 64 columns of one parity for 64
+// pairs, 128-byte swizzle: the A tokens and the B tokens of a unit land in separate runs of rows
+bool make_src_map(CUtensorMap* tm, const void* base, int64_t lo, int64_t pairs, int64_t cap, int LH) {
+  EncodeTiledFn fn = fused_encode_fn();
+  if (!fn) return false;
+  const cuuint64_t dims[4] = {128, 2, (cuuint64_t)pairs, (cuuint64_t)LH};
+  const cuuint64_t strides[3] = {256, 512, (cuuint64_t)cap * 256};
+  const cuuint32_t box[4] = {64, 1, kFUnit / 2, 1}, es[4] = {1, 1, 1, 1};
+  void* addr = const_cast<unsigned char*>(static_cast<const unsigned char*>(base) + lo * 256);
+  return fn(tm, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 4, addr, dims, strides, box, es, CU_TENSOR_MAP_INTERLEAVE_NONE,
+            CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
 // (column 128, token, slab) view of a cache; box = 64 columns x `rows` tokens, 128-byte swizzle
 bool make_map(CUtensorMap* tm, const void* base, int64_t cap, int LH, int rows, bool load) {
   EncodeTiledFn fn = fused_encode_fn();
@@ -400,7 +407,8 @@ bool round_fused2_supported(int dtype, int D, int chunk) {
 cudaError_t launch_round_fused2(const RoundArgs& r, int64_t units, int32_t* assign2, int64_t stride2, cudaStream_t st) {
   if (units <= 0) return cudaSuccess;
   CUtensorMap tm_k, tm_v, tm_ko, tm_vo;
-  if (!make_map(&tm_k, r.k_src, r.src_cap, r.LH, kFUnit, true) || !make_map(&tm_v, r.v_src, r.src_cap, r.LH, kFUnit, true) ||
+  if (!make_src_map(&tm_k, r.k_src, r.lo, units * (kFUnit / 2), r.src_cap, r.LH) ||
+      !make_src_map(&tm_v, r.v_src, r.lo, units * (kFUnit / 2), r.src_cap, r.LH) ||
       !make_map(&tm_ko, r.k_dst, r.dst_cap, r.LH, 32, false) || !make_map(&tm_vo, r.v_dst, r.dst_cap, r.LH, 32, false))
     return cudaErrorInvalidValue;
   FusedArgs a{};
