@@ -40,6 +40,10 @@ constexpr int kFHalf = kFUnit * 128;     // 128 rows x 64 columns (128 bytes eac
 constexpr int kFStage = 2 * kFHalf;      // one tensor's tile of a unit: 32 KiB
 constexpr int kFExtra = 400;             // per warp: degrees after round 1 [64], after round 2 [32], mbarrier, pad
 constexpr uint32_t kOneBf16 = 0x3f80u;   // 1.0
+// Round 1 leaves the centroids where round 2 wants them: even positions (its A tokens) from row 0, odd positions (its B
+// tokens) from row kFOdd.  68 rather than 64: consecutive centroids then fall into different 16-byte columns of the
+// swizzle, so the eight rows of a matrix store hit eight different banks.
+constexpr int kFOdd = 68;
 
 struct FusedArgs {
   int32_t* deg_dst;
@@ -147,7 +151,7 @@ __device__ __forceinline__ int match64(uint32_t tile, int row_a, int row_b, int 
 // Eq. 5 on one chunk of one tensor, in place.  A tokens in rows row_a .. + 31, B tokens in rows row_b .. + 31; lane i
 // holds the B index A token i merges into, lane j the summed degree n' of B token j's cluster.  deg_a / deg_b: degrees
 // of the A and B tokens, element stride 2 (null: all one).  Centroid j goes to row dst0 + j (dst_split false) or, split
-// by parity for the next round, to row dst0 + j / 2 (j even) / dst0 + 64 + j / 2 (j odd).
+// by parity for the next round, to row dst0 + j / 2 (j even) / dst0 + kFOdd + j / 2 (j odd).
 __device__ __forceinline__ void merge64(uint32_t tile, int row_a, int row_b, int dst0, bool dst_split, int my_best, int my_n,
                                         const int* deg_a, const int* deg_b, int lane) {
   const int g = lane >> 2, t = lane & 3;
@@ -239,7 +243,7 @@ __device__ __forceinline__ void merge64(uint32_t tile, int row_a, int row_b, int
           o[j] = pack_bf16x2(x, y);
         }
         const int j_out = 16 * mt + 8 * hi + (lane & 7);
-        const int row = dst_split ? dst0 + ((j_out & 1) << 6) + (j_out >> 1) : dst0 + j_out;
+        const int row = dst_split ? dst0 + (j_out & 1) * kFOdd + (j_out >> 1) : dst0 + j_out;
         stsm_x4(f_addr(tile, row, 8 * h + (lane >> 3)), o[0], o[1], o[2], o[3]);
         stsm_x4(f_addr(tile, row, 8 * h + 4 + (lane >> 3)), o[4], o[5], o[6], o[7]);
       }
@@ -299,7 +303,7 @@ round_fused2_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_const
 #pragma unroll 1
       for (int it = 0; it < 3; ++it) {  // round 1 on the unit's first and second chunk, then round 2 on the 64 centroids
         // round 1 leaves centroid j of chunk q where round 2 finds it: position 32 q + j of the 64, split by parity
-        const int row_a = it == 1 ? 32 : 0, row_b = 64 + row_a, dst0 = it == 0 ? 0 : (it == 1 ? 16 : 0);
+        const int row_a = it == 1 ? 32 : 0, row_b = it == 2 ? kFOdd : 64 + row_a, dst0 = it == 1 ? 16 : 0;
         int best, n;
         if (ph == 0) {
           best = match64(tile, row_a, row_b, lane);
