@@ -21,6 +21,9 @@ first-moment conservation, N = 1 reduces approximate attention to softmax
 attention, the q = 0 closed form, the replication identity, the duplicated-key
 construction, Theorem A.1 by enumeration, Table 1's multiply-add count, the
 at-most-half bound and untouched sinks / recent tokens.
+Storage rounding (`bf16_round`, `round_to_dtype`, the `storage=` argument of the drivers): hand-written bit
+patterns, agreement with an exact rational-arithmetic rounding and with torch's conversion on a million random
+bit patterns, a multi-round brute-force replay that rounds between rounds.
 Parity unpinned: nothing in this file; the *quality* of the clusters on real
 model caches (the paper's accuracy tables) is outside what it computes.
 """
@@ -51,14 +54,15 @@ class Params:
 # --------------------------------------------------------------------------- dtype rounding
 
 def bf16_round(x):
-    """Round to the nearest bfloat16 (ties to even), returned as float64."""
-    x32 = np.asarray(x, dtype=np.float32)
-    bits = x32.view(np.uint32).astype(np.uint64)
-    lsb = (bits >> 16) & 1
-    rounded = ((bits + 0x7FFF + lsb) >> 16) << 16
-    out = rounded.astype(np.uint32).view(np.float32)
-    out = np.where(np.isnan(x32), x32, out)
-    return out.astype(np.float64)
+    """The nearest bfloat16 (8 significant bits, fp32's exponent range, subnormals kept), ties to the even
+    significand, overflow to infinity; computed from the float64 value in one rounding and returned as float64."""
+    x = np.asarray(x, dtype=np.float64)
+    _, e = np.frexp(x)                                  # |x| = m * 2^e with 0.5 <= m < 1
+    quantum = np.ldexp(1.0, np.maximum(e - 8, -133))    # spacing of bfloat16 around x; 2^-133 in the subnormal range
+    with np.errstate(invalid="ignore", over="ignore"):
+        r = np.rint(x / quantum) * quantum              # np.rint rounds halves to the even integer
+        r = np.where(np.abs(r) >= 2.0 ** 128, np.copysign(np.inf, x), r)
+    return np.where(np.isfinite(x), r, x)
 
 
 def round_to_dtype(x, dtype: str):

@@ -442,3 +442,144 @@ def test_paged_attention_does_not_depend_on_where_the_pages_are():
 def textbook_attention_heads(q, K, V, scale, G):
     return np.stack([softmax(K[j // G] @ q[j] * scale) @ V[j // G] for j in range(q.shape[0])])
 
+
+
+# ----------------------------------------------------------------------------- storage rounding (the cache dtype)
+
+def exact_bf16(x: float) -> float:
+    """Nearest bfloat16 in exact rational arithmetic: candidates are the two multiples of the format's spacing
+    around x; the nearer wins, a tie goes to the even multiple; past the largest finite value it is infinity."""
+    from fractions import Fraction
+    if x != x or x in (math.inf, -math.inf) or x == 0.0:
+        return x
+    fx = Fraction(x)
+    e = math.frexp(x)[1]                      # |x| in [2^(e-1), 2^e)
+    q = Fraction(2) ** max(e - 8, -133)       # 8 significant bits; subnormal spacing 2^-133
+    lo = math.floor(fx / q)
+    rem = fx / q - lo
+    n = lo if rem < Fraction(1, 2) else lo + 1 if rem > Fraction(1, 2) else lo + (lo & 1)
+    r = n * q
+    if abs(r) >= Fraction(2) ** 128:
+        return math.copysign(math.inf, x)
+    return math.copysign(float(r), x)
+
+
+def f32_from_bits(b: int) -> float:
+    return float(np.array([b], dtype=np.uint32).view(np.float32)[0])
+
+
+def bf16_bits(x: float) -> int:
+    """Upper 16 bits of the float32 pattern of a value that is exactly a bfloat16."""
+    b = int(np.array([x], dtype=np.float32).view(np.uint32)[0])
+    assert b & 0xFFFF == 0, "not a bfloat16 value"
+    return b >> 16
+
+
+@pytest.mark.parametrize("bits,expect", [
+    (0x3F808000, 0x3F80),   # 1 + 2^-8: halfway, the even neighbour is 1
+    (0x3F818000, 0x3F82),   # 1 + 3 * 2^-8: halfway, the even neighbour is 1 + 2^-6
+    (0x3F808001, 0x3F81),   # just above a tie
+    (0x3F807FFF, 0x3F80),   # just below a tie
+    (0xBF808000, 0xBF80),   # ties are symmetric in sign
+    (0xBF818000, 0xBF82),
+    (0x00000000, 0x0000), (0x80000000, 0x8000),   # signed zeros
+    (0x7F800000, 0x7F80), (0xFF800000, 0xFF80),   # infinities
+    (0x7F7F0000, 0x7F7F),   # the largest finite bfloat16
+    (0x7F7F7FFF, 0x7F7F),   # below the tie with infinity
+    (0x7F7F8000, 0x7F80),   # the tie itself goes to the even side: infinity
+    (0x00000001, 0x0000),   # smallest fp32 subnormal: far below half of 2^-133
+    (0x00008000, 0x0000),   # 2^-134 = half the subnormal spacing: tie to even (zero)
+    (0x00008001, 0x0001),   # just above it
+    (0x00018000, 0x0002),   # 1.5 * 2^-133: tie, even is 2 * 2^-133
+    (0x007F8000, 0x0080),   # the largest subnormals round up into the smallest normal
+])
+def test_bf16_round_hand_written_bit_patterns(bits, expect):
+    got = float(O.bf16_round(f32_from_bits(bits)))
+    assert bf16_bits(got) == expect
+    assert bf16_bits(exact_bf16(f32_from_bits(bits))) == expect      # the rational restatement agrees with the hand values
+
+
+def test_bf16_round_keeps_nan_and_rounds_float64_once():
+    assert np.isnan(O.bf16_round(np.nan)) and np.isnan(O.round_to_dtype(np.array([np.nan]), "bf16"))[0]
+    # 1 + 2^-8 + 2^-40 lies above the tie; rounding through float32 first would land on the tie and go down
+    assert float(O.bf16_round(1 + 2.0 ** -8 + 2.0 ** -40)) == 1 + 2.0 ** -7
+    assert float(O.bf16_round(1 + 2.0 ** -8 - 2.0 ** -40)) == 1.0
+    assert float(O.bf16_round(-(1 + 3 * 2.0 ** -8 + 2.0 ** -45))) == -(1 + 2.0 ** -6)
+
+
+def test_bf16_round_agrees_with_rational_arithmetic_and_with_torch():
+    import torch
+    rng = np.random.default_rng(7)
+    bits = rng.integers(0, 2 ** 32, size=1_000_000, dtype=np.uint64).astype(np.uint32)
+    x32 = bits.view(np.float32)
+    keep = ~np.isnan(x32)
+    x32 = x32[keep]
+    ours = O.bf16_round(x32.astype(np.float64)).astype(np.float32).view(np.uint32)
+    theirs = torch.from_numpy(x32.copy()).to(torch.bfloat16).to(torch.float32).numpy().view(np.uint32)
+    np.testing.assert_array_equal(ours, theirs)
+    # float64 inputs (what the oracle actually rounds), against exact rational arithmetic
+    x64 = np.concatenate([rng.standard_normal(20000) * np.exp(rng.uniform(-30, 30, 20000)),
+                          (1 + rng.integers(0, 256, 2000) / 128.0 + 2.0 ** -8) * 2.0 ** rng.integers(-20, 20, 2000)])  # exact ties
+    got = O.bf16_round(x64)
+    want = np.array([exact_bf16(float(v)) for v in x64])
+    np.testing.assert_array_equal(got, want)
+
+
+def test_round_to_dtype_f32_is_round_to_nearest_even():
+    import struct
+    assert float(O.round_to_dtype(np.array([1 + 2.0 ** -24]), "f32")[0]) == 1.0                 # tie, even is 1
+    assert float(O.round_to_dtype(np.array([1 + 3 * 2.0 ** -24]), "f32")[0]) == 1 + 2.0 ** -22  # tie, even is 1 + 2^-22
+    assert float(O.round_to_dtype(np.array([1 + 2.0 ** -24 + 2.0 ** -50]), "f32")[0]) == 1 + 2.0 ** -23
+    rng = np.random.default_rng(8)
+    x = rng.standard_normal(5000) * np.exp(rng.uniform(-20, 20, 5000))
+    want = np.array([struct.unpack("f", struct.pack("f", float(v)))[0] for v in x])
+    np.testing.assert_array_equal(O.round_to_dtype(x, "f32"), want)
+    with pytest.raises(ValueError):
+        O.round_to_dtype(x, "fp8")
+
+
+@pytest.mark.parametrize("select", [O.SELECT_GLOBAL, O.SELECT_CHUNK])
+def test_multi_round_driver_rounds_to_storage_between_rounds(select):
+    """Algorithm 1 reassigns K, V after every call of CentroidKV; with a bf16 cache each reassignment is a rounding.
+    Replay three rounds by brute force, rounding the rows with exact rational arithmetic in between."""
+    rng = np.random.default_rng(31)
+    s, c, d = 24, 8, 5
+    K, V = rand_cache(rng, 1, 1, s, d, ar=0.7)
+    K, V = O.round_to_dtype(K, "bf16"), O.round_to_dtype(V, "bf16")
+    p = O.Params(chunk=c, n_sink=1, n_recent=2, n_rounds_max=3, r_init=1.0, r_decay=0.25, r_min=0.5, budget=0, select=select)
+    Ko, Vo, do, _, logs = O.compress_prefill(K, V, None, p, storage="bf16")
+    assert len(logs) == 3
+    Kb, Vb, db = K[0, 0].tolist(), V[0, 0].tolist(), [1] * s
+    for j in range(3):
+        r = max(p.r_init - j * p.r_decay, p.r_min)
+        if select == O.SELECT_GLOBAL:
+            n_edges = len(logs[j].edges[0].a_pos)
+            M = int(math.floor(r * n_edges + 1e-9))
+            Kn, Vn, dn, _ = brute_round(Kb, Vb, db, 1, 2, c, M)
+        else:
+            Kn, Vn, dn = brute_round_per_chunk(Kb, Vb, db, 1, 2, c, r)
+        Kb = [[exact_bf16(float(x)) for x in row] for row in Kn]
+        Vb = [[exact_bf16(float(x)) for x in row] for row in Vn]
+        db = list(dn)
+    np.testing.assert_array_equal(do[0, 0], np.array(db))
+    np.testing.assert_array_equal(Ko[0, 0], np.array(Kb))
+    np.testing.assert_array_equal(Vo[0, 0], np.array(Vb))
+    # and every stored row is a bfloat16 value
+    np.testing.assert_array_equal(Ko, O.bf16_round(Ko))
+
+
+def brute_round_per_chunk(K, V, deg, n_sink, n_recent, c, r):
+    """Per-chunk ranking by brute force: every chunk is a stand-alone call of brute_round with its own count."""
+    s = len(K)
+    lo, hi = n_sink, s - n_recent
+    Ko, Vo, do = [list(x) for x in K[:lo]], [list(x) for x in V[:lo]], list(deg[:lo])
+    start = lo
+    while start < hi:
+        end = min(start + c, hi)
+        n_a = (end - start + 1) // 2 if end - start >= 2 else 0
+        M = int(math.floor(r * n_a + 1e-9))
+        Kc, Vc, dc, _ = brute_round(K[start:end], V[start:end], deg[start:end], 0, 0, c, M)
+        Ko += Kc.tolist(); Vo += Vc.tolist(); do += dc.tolist()
+        start = end
+    Ko += [list(x) for x in K[hi:]]; Vo += [list(x) for x in V[hi:]]; do += list(deg[hi:])
+    return np.array(Ko), np.array(Vo), np.array(do)
