@@ -5,7 +5,8 @@
  *
  * Conventions
  *  - Every pointer is a DEVICE pointer owned by the caller unless its comment says "host".
- *    The library allocates and frees nothing and keeps no global state.
+ *    The library allocates and frees nothing and keeps no global state that a call could observe (the one
+ *    exception is ckv_decode_attn_static, whose scratch array is shared by every call: see its comment).
  *  - All work is enqueued on `cuda_stream` (a cudaStream_t passed as void*; NULL = the
  *    default stream) and the calls return without synchronising.
  *  - The return value is a ckv_status.  Argument errors are found on the host before any
@@ -14,7 +15,7 @@
  *    token capacity, head_dim) of which the first `len` tokens of every (layer, head)
  *    are valid; deg and logdeg: [L, H, cap].  K and V must be 16-byte aligned.
  *  - Thread safety: calls on distinct streams with distinct workspaces and outputs do
- *    not interfere.
+ *    not interfere (again except ckv_decode_attn_static).
  *  - This version supports D = 128 and even chunk sizes 2..256 (or 0 = no chunking); anything else
  *    returns CKV_ERR_UNSUPPORTED.
  */
@@ -44,6 +45,10 @@ typedef enum {
   CKV_ERR_NO_PROGRESS = 5, /* the ratio schedule merges nothing although the budget is not met */
   CKV_ERR_UNSUPPORTED = 6, /* head_dim, chunk size or group size outside this version's range */
   CKV_ERR_CUDA = 7         /* a CUDA runtime call failed (launch configuration, invalid stream ...) */
+  /* There is no "timeout" status.  The calls return before their kernels run, so a bounded wait inside a kernel that
+   * gives up cannot be reported here: the compress kernels (the only ones that wait on asynchronous copies, tensor-core
+   * completions or each other) record it in a status word at the start of their workspace, which ckv_workspace_status
+   * reads.  The decode kernels contain no such wait and have no status word. */
 } ckv_status;
 
 /* One sequence's KV cache over all layers and KV heads, with the cluster degrees N of Sec. 3
@@ -93,6 +98,10 @@ size_t ckv_workspace_bytes(const ckv_cache* shape, const ckv_params* params);
  * original order with each centroid at its B token's place, then the recent tokens.
  * dst must not overlap src or the workspace; dst->cap must be at least what ckv_compress_plan
  * reports.  On return dst->len (host field) is the new length, dst->pending is 0.
+ * CKV_OK does not imply dst->len <= params->budget: the loop also ends after n_rounds_max rounds (with Eq. 4's
+ * defaults 0.8 / 0.2 floored at 0.2, a 25 % budget takes six).  Compare dst->len, or *rounds_done with what
+ * ckv_compress_plan reports for a large n_rounds_max.  CKV_ERR_NO_PROGRESS is returned only when a round would
+ * merge nothing.
  * assign: optional [L, H, src->len] int32, receives for each source token the dst slot that
  * holds it (its cluster).  rounds_done: optional host pointer. */
 int ckv_compress_prefill(const ckv_cache* src, ckv_cache* dst, const ckv_params* params, int32_t* assign,

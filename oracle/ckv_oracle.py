@@ -120,6 +120,7 @@ class Edges:
     chunk_id: np.ndarray         # chunk the edge belongs to
     argmax_gap: np.ndarray       # relative fp64 gap between best and second-best candidate (inf if one candidate)
     macs: int = 0                # multiply-adds spent on the similarity matrices (Table 1)
+    sim64: np.ndarray = None     # the same similarity before it was rounded to float32 (for the record: near ties)
 
 
 def match_head(K, n_sink, n_recent, c) -> Edges:
@@ -129,7 +130,7 @@ def match_head(K, n_sink, n_recent, c) -> Edges:
     rounds), not weighted by degree."""
     s, d = K.shape
     _, _, chunks = chunk_bounds(s, n_sink, n_recent, c)
-    a_pos, b_pos, sim, cid, gap = [], [], [], [], []
+    a_pos, b_pos, sim, cid, gap, sim64 = [], [], [], [], [], []
     macs = 0
     for ci, (beg, end) in enumerate(chunks):
         A, B = alternating_partition(end - beg)
@@ -142,6 +143,7 @@ def match_head(K, n_sink, n_recent, c) -> Edges:
         a_pos.extend(beg + A)
         b_pos.extend(beg + B[best])
         sim.extend(S32[np.arange(len(A)), best])
+        sim64.extend(S[np.arange(len(A)), best])
         cid.extend([ci] * len(A))
         if len(B) > 1:
             top = np.sort(S, axis=1)[:, ::-1]
@@ -150,7 +152,7 @@ def match_head(K, n_sink, n_recent, c) -> Edges:
             gap.extend([np.inf] * len(A))
     return Edges(np.array(a_pos, dtype=np.int64), np.array(b_pos, dtype=np.int64),
                  np.array(sim, dtype=np.float32), np.array(cid, dtype=np.int64),
-                 np.array(gap, dtype=np.float64), macs)
+                 np.array(gap, dtype=np.float64), macs, np.array(sim64, dtype=np.float64))
 
 
 # --------------------------------------------------------------------------- Sec. 5.3: which edges are merged

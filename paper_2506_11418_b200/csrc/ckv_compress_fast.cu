@@ -18,6 +18,7 @@
 
 #include "ckv_common.cuh"
 #include "ckv_internal.h"
+#include "ckv_ptx.cuh"
 
 namespace ckv {
 
@@ -29,52 +30,8 @@ constexpr int kRowBytes = kD * 2; // one bf16 row
 constexpr int kTileBytes = kC * kRowBytes;
 constexpr int kStageBytes = 2 * kTileBytes;  // K tile then V tile
 constexpr int kExtraBytes = 400;             // per warp: degrees [64] int, best [32] int, mbarrier (8 B), pad
-constexpr uint32_t kSpinLimit = 1u << 22;
 
-__device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
-
-__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
-  asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count));
-}
-
-__device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes) {
-  asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
-}
-
-__device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
-  uint32_t ok;
-  asm volatile(
-      "{\n\t.reg .pred p;\n\t"
-      "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
-      "selp.u32 %0, 1, 0, p;\n\t}"
-      : "=r"(ok)
-      : "r"(bar), "r"(parity)
-      : "memory");
-  return ok != 0;
-}
-
-// Bounded wait: false if the phase did not complete within the spin limit.
-__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity) {
-  for (uint32_t i = 0; i < kSpinLimit; ++i) {
-    if (mbar_try_wait(bar, parity)) return true;
-    if (i > 64) __nanosleep(64);
-  }
-  return false;
-}
-
-__device__ __forceinline__ void bulk_load(uint32_t dst, const void* src, uint32_t bytes, uint32_t bar) {
-  asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];" ::"r"(dst),
-               "l"(src), "r"(bytes), "r"(bar)
-               : "memory");
-}
-
-__device__ __forceinline__ void mma_bf16(float (&d)[4], uint32_t a0, uint32_t a1, uint32_t a2, uint32_t a3, uint32_t b0,
-                                         uint32_t b1) {
-  asm volatile(
-      "mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
-      : "+f"(d[0]), "+f"(d[1]), "+f"(d[2]), "+f"(d[3])
-      : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1));
-}
+using namespace ptx;
 
 __device__ __forceinline__ void unpack4(uint2 u, float (&f)[4]) {
   f[0] = __uint_as_float(u.x << 16);
@@ -139,7 +96,7 @@ __global__ void __launch_bounds__(NW * 32, 1) round_fast_kernel(const FastArgs a
   auto issue = [&](int64_t it) {
     const uint32_t lh = (uint32_t)it / n_full, ch = (uint32_t)it - lh * n_full;
     const int64_t row0 = (int64_t)lh * a.src_cap + a.lo + (int64_t)ch * kC;
-    mbar_expect_tx(bar, KIND == kFastMatch ? kTileBytes : kStageBytes);
+    mbar_arrive_expect_tx(bar, KIND == kFastMatch ? kTileBytes : kStageBytes);
     bulk_load(k_s, a.k_src + row0 * kD, kTileBytes, bar);
     if (KIND != kFastMatch) bulk_load(v_s, a.v_src + row0 * kD, kTileBytes, bar);  // the matching alone never reads V
   };
@@ -411,18 +368,6 @@ __global__ void __launch_bounds__(NW * 32, 1) round_fast_kernel(const FastArgs a
       issue(item + stride);
     }
   }
-}
-
-int sm_count() {
-  static int cached = 0;
-  if (cached == 0) {
-    int dev = 0, n = 0;
-    if (cudaGetDevice(&dev) == cudaSuccess && cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev) == cudaSuccess && n > 0)
-      cached = n;
-    else
-      return 148;
-  }
-  return cached;
 }
 
 template <int NW, bool HAS_DEG, int KIND>

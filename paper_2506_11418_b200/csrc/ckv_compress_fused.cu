@@ -430,10 +430,7 @@ cudaError_t launch_round_fused2(const RoundArgs& r, int64_t units, int32_t* assi
   const size_t smem = (size_t)kFWarps * (kFStage + kFExtra);
   cudaError_t e = cudaFuncSetAttribute(round_fused2_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
   if (e != cudaSuccess) return e;
-  int dev = 0, sms = 0;
-  if (cudaGetDevice(&dev) != cudaSuccess || cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || sms <= 0)
-    return cudaErrorInvalidValue;
-  const int64_t ctas = std::min<int64_t>(sms, (a.n_items + kFWarps - 1) / kFWarps);
+  const int64_t ctas = std::min<int64_t>(sm_count(), (a.n_items + kFWarps - 1) / kFWarps);
   round_fused2_kernel<<<(unsigned)ctas, kFWarps * 32, smem, st>>>(tm_k, tm_v, tm_ko, tm_vo, a);
   return cudaGetLastError();
 }

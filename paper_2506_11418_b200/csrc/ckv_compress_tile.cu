@@ -481,18 +481,6 @@ __global__ void __launch_bounds__(TileCfg<C>::T, TileCfg<C>::kCtasPerSm) round_t
   }
 }
 
-int tile_sm_count() {
-  static int cached = 0;
-  if (cached == 0) {
-    int dev = 0, n = 0;
-    if (cudaGetDevice(&dev) == cudaSuccess && cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev) == cudaSuccess && n > 0)
-      cached = n;
-    else
-      return 148;
-  }
-  return cached;
-}
-
 template <int C>
 cudaError_t launch_tile_c(const RoundArgs& a, cudaStream_t st) {
   using Cfg = TileCfg<C>;
@@ -501,7 +489,7 @@ cudaError_t launch_tile_c(const RoundArgs& a, cudaStream_t st) {
   if (n_items <= 0) return cudaSuccess;
   cudaError_t e = cudaFuncSetAttribute(round_tile_kernel<C>, cudaFuncAttributeMaxDynamicSharedMemorySize, Cfg::kBytes);
   if (e != cudaSuccess) return e;
-  const int64_t ctas = std::min<int64_t>((int64_t)tile_sm_count() * Cfg::kCtasPerSm, n_items);
+  const int64_t ctas = std::min<int64_t>((int64_t)sm_count() * Cfg::kCtasPerSm, n_items);
   round_tile_kernel<C><<<(unsigned)ctas, Cfg::T, Cfg::kBytes, st>>>(a);
   return cudaGetLastError();
 }

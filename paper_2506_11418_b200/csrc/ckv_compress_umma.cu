@@ -759,18 +759,6 @@ bool make_dst_map(CUtensorMap* tm, void* base, int64_t cap, int LH) {
             CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_NONE, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
-int umma_sm_count() {
-  static int cached = 0;
-  if (cached == 0) {
-    int dev = 0, n = 0;
-    if (cudaGetDevice(&dev) == cudaSuccess && cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev) == cudaSuccess && n > 0)
-      cached = n;
-    else
-      return 148;
-  }
-  return cached;
-}
-
 }  // namespace
 
 bool round_umma_supported(const RoundArgs& a, int dtype, int D) {
@@ -796,13 +784,13 @@ cudaError_t launch_round_umma(const RoundArgs& a, int64_t n_full, cudaStream_t s
     cudaError_t em = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)msmem);
     if (em != cudaSuccess) return em;
     const int64_t items = (a.chunk == kUC ? n_full : (n_full + 1) / 2) * a.LH;
-    kern<<<(unsigned)std::min<int64_t>(umma_sm_count(), items), kMThreads, msmem, st>>>(tm_k, a, (int)n_full);
+    kern<<<(unsigned)std::min<int64_t>(sm_count(), items), kMThreads, msmem, st>>>(tm_k, a, (int)n_full);
     return cudaGetLastError();
   }
   const size_t smem = kUBytes + kUAlign;
   cudaError_t e = cudaFuncSetAttribute(round_umma_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
   if (e != cudaSuccess) return e;
-  const int64_t ctas = std::min<int64_t>(umma_sm_count(), n_full * a.LH);
+  const int64_t ctas = std::min<int64_t>(sm_count(), n_full * a.LH);
   round_umma_kernel<<<(unsigned)ctas, kUThreads, smem, st>>>(tm_k, tm_v, tm_ko, tm_vo, a, (int)n_full);
   return cudaGetLastError();
 }

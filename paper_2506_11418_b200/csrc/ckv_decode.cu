@@ -9,6 +9,7 @@
 #include "../../include/ckv.h"
 #include "ckv_common.cuh"
 #include "ckv_internal.h"
+#include "ckv_ptx.cuh"
 
 namespace ckv {
 
@@ -319,21 +320,8 @@ __device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commi
 template <int N>
 __device__ __forceinline__ void cp_async_wait() { asm volatile("cp.async.wait_group %0;" ::"n"(N) : "memory"); }
 
-__device__ __forceinline__ void ldsm_x4(uint32_t addr, uint32_t (&r)[4]) {
-  asm volatile("ldmatrix.sync.aligned.m8n8.x4.shared.b16 {%0,%1,%2,%3}, [%4];"
-               : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]) : "r"(addr));
-}
-__device__ __forceinline__ void ldsm_x4_trans(uint32_t addr, uint32_t (&r)[4]) {
-  asm volatile("ldmatrix.sync.aligned.m8n8.x4.trans.shared.b16 {%0,%1,%2,%3}, [%4];"
-               : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]) : "r"(addr));
-}
-__device__ __forceinline__ void mma_bf16_16816(float (&d)[4], uint32_t a0, uint32_t a1, uint32_t a2, uint32_t a3,
-                                               uint32_t b0, uint32_t b1) {
-  asm volatile(
-      "mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
-      : "+f"(d[0]), "+f"(d[1]), "+f"(d[2]), "+f"(d[3])
-      : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1));
-}
+using ptx::ldsm_x4;
+using ptx::ldsm_x4_trans;
 
 __device__ __forceinline__ void cluster_sync_all() {
   asm volatile("barrier.cluster.arrive.release.aligned;\n\tbarrier.cluster.wait.acquire.aligned;" ::: "memory");
@@ -466,8 +454,8 @@ __global__ void __launch_bounds__(NW * 32, 1) decode_fast_kernel(const DecodeArg
         const int chunk = 4 * kq + (lane >> 3);
         uint32_t r[4];
         ldsm_x4(ks_ + (uint32_t)tok * 256u + (uint32_t)((chunk ^ (tok & 7)) << 4), r);
-        mma_bf16_16816(sacc[j], qa[2 * kq][0], 0u, qa[2 * kq][1], 0u, r[0], r[1]);
-        mma_bf16_16816(sacc[j], qa[2 * kq + 1][0], 0u, qa[2 * kq + 1][1], 0u, r[2], r[3]);
+        ptx::mma_bf16(sacc[j], qa[2 * kq][0], 0u, qa[2 * kq][1], 0u, r[0], r[1]);
+        ptx::mma_bf16(sacc[j], qa[2 * kq + 1][0], 0u, qa[2 * kq + 1][1], 0u, r[2], r[3]);
       }
     }
     // ---- bias, mask, online softmax (thread holds head g, tokens 8j + 2t, 8j + 2t + 1)
@@ -514,7 +502,7 @@ __global__ void __launch_bounds__(NW * 32, 1) decode_fast_kernel(const DecodeArg
         const int chunk = 2 * i + (mi & 1);
         uint32_t r[4];
         ldsm_x4_trans(vs_ + (uint32_t)tok * 256u + (uint32_t)((chunk ^ (tok & 7)) << 4), r);
-        mma_bf16_16816(oacc[i], r[0], r[1], r[2], r[3], pb[2 * s], pb[2 * s + 1]);
+        ptx::mma_bf16(oacc[i], r[0], r[1], r[2], r[3], pb[2 * s], pb[2 * s + 1]);
       }
     }
   }
@@ -695,7 +683,7 @@ cudaError_t launch_decode_fast(const DecodeArgs& a, cudaStream_t st) {
 // kernel one span per warp (four per CTA).
 void decode_plan(int32_t Bz, int32_t H, int dtype, int64_t max_len, int64_t max_partial_floats, int32_t G, int32_t D,
                  int32_t* n_splits, int64_t* span) {
-  const int64_t pairs = (int64_t)Bz * H;
+  const int64_t pairs = (int64_t)Bz * H, sms = sm_count();
   int64_t ns, gran;
   if (dtype == 1) {
     // One CTA per SM (the rings fill its shared memory), four splits per CTA.  Choose the CTAs per (sequence, head)
@@ -706,7 +694,7 @@ void decode_plan(int32_t Bz, int32_t H, int dtype, int64_t max_len, int64_t max_
     const int64_t max_cpp = std::min<int64_t>(64, std::max<int64_t>(1, tiles / (4 * kFWarps)));
     int64_t best = 1, best_cost = INT64_MAX;
     for (int64_t cpp = 1; cpp <= max_cpp; ++cpp) {
-      const int64_t waves = (pairs * cpp + 147) / 148;
+      const int64_t waves = (pairs * cpp + sms - 1) / sms;
       const int64_t per_warp = (tiles + cpp * kFWarps - 1) / (cpp * kFWarps);
       const int64_t cost = waves * (per_warp + 2);
       if (cost < best_cost) {
@@ -718,7 +706,7 @@ void decode_plan(int32_t Bz, int32_t H, int dtype, int64_t max_len, int64_t max_
   } else {
     gran = 128;
     const int64_t cap = std::max<int64_t>(1, (max_len + 127) / 128);
-    ns = std::min(cap, (4 * 148 + pairs - 1) / pairs);
+    ns = std::min(cap, (4 * sms + pairs - 1) / pairs);
   }
   ns = std::max<int64_t>(ns, 1);
   const int64_t per_split = pairs * G * (D + 4);
@@ -756,7 +744,9 @@ constexpr size_t kStaticScratchFloats = (size_t)1 << 20;  // 4 MiB
 static __device__ __align__(256) float g_decode_scratch[kStaticScratchFloats];
 
 constexpr int kMaxDevices = 64;
-float* g_scratch_ptr[kMaxDevices];  // device address of g_decode_scratch per device, resolved on first use
+// device address of g_decode_scratch per device, resolved on first use (atomic: two host threads may make their
+// first call on a device at the same time; both would store the same address)
+std::atomic<float*> g_scratch_ptr[kMaxDevices];
 
 }  // namespace
 
@@ -776,18 +766,20 @@ extern "C" int ckv_decode_attn_static(const ckv_layer_view* views_dev, int32_t B
 
   int dev = -1;
   if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices) return CKV_ERR_CUDA;
-  if (!g_scratch_ptr[dev]) {
+  float* scratch = g_scratch_ptr[dev].load(std::memory_order_relaxed);
+  if (!scratch) {
     // In host code `g_decode_scratch` names a host-side shadow of the symbol, not device memory: ask the
     // runtime for the address the array has on the current device and hand that to the kernels.
     void* p = nullptr;
     if (cudaGetSymbolAddress(&p, g_decode_scratch) != cudaSuccess || !p) return CKV_ERR_CUDA;
-    g_scratch_ptr[dev] = static_cast<float*>(p);
+    scratch = static_cast<float*>(p);
+    g_scratch_ptr[dev].store(scratch, std::memory_order_relaxed);
   }
   ckv::DecodeArgs a{};
   a.views = views_dev;
   a.q = q;
   a.out = out;
-  a.partial = g_scratch_ptr[dev];
+  a.partial = scratch;
   a.Bz = Bz;
   a.H = H;
   a.G = G;

@@ -5,6 +5,8 @@
 #include <stddef.h>
 #include <stdint.h>
 
+#include <atomic>
+
 namespace ckv {
 
 enum RoundMode : int32_t {
@@ -85,6 +87,19 @@ struct DecodeArgs {
   const float* logdeg_pages;  // [n_pages, H, page_tokens] or null
   int32_t page_shift;         // log2(page_tokens), page_tokens >= 32
 };
+
+// Streaming multiprocessors of the current device, asked once per device (the grids are sized from it).
+inline int sm_count() {
+  constexpr int kMaxDev = 64;
+  static std::atomic<int> cached[kMaxDev];
+  int dev = 0, n = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess) return 148;
+  const bool slot = dev >= 0 && dev < kMaxDev;
+  if (slot && (n = cached[dev].load(std::memory_order_relaxed)) > 0) return n;
+  if (cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || n <= 0) return 148;
+  if (slot) cached[dev].store(n, std::memory_order_relaxed);
+  return n;
+}
 
 // Launch with programmatic stream serialization: the kernel may become resident while the kernel ahead of it
 // in the stream drains; it must call griddep_wait() before it touches anything that kernel produced.

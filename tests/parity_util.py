@@ -14,6 +14,12 @@ Tolerances
              storage rounding plus one ulp exceed 2e-2, so there only the one-ulp rule applies.  The
              fraction within 2e-2 over all elements is returned for the record.
   degrees    exact.  log-degrees 1e-6 relative.
+  attention  (Eq. 3) stated bar: 2e-2 absolute for bf16, 2e-4 for fp32.  Beside it, for bf16, a bound that follows
+             from the kernel's arithmetic, per output element: the output is rounded to bf16 (half an ulp:
+             2^-9 |o|) and the softmax weights enter the weighted sum of V as bf16 (2^-9 relative each, numerator
+             and normaliser: 2^-8 * sum_t w_t |v_t|), plus 2e-5 for the fp32 scores and exponentials.  A test
+             with cluster degrees also shows that it can see a wrong bias: the oracle with and without Eq. 3's
+             log n_t term must differ by at least five times that bound somewhere in the batch.
 """
 from __future__ import annotations
 
@@ -111,13 +117,13 @@ def _excuse_and_rebuild(K, V, deg, assign_gpu, e: O.Edges, sel_o, p: O.Params, s
         for ci in np.unique(e.chunk_id):
             m = e.chunk_id == ci
             assert merged[m].sum() == sel_o[m].sum(), "per-chunk merge count differs"
-    sim64 = e.sim.astype(np.float64)
+    sim64 = e.sim64            # the oracle's float64 similarities (its decisions use them rounded to float32)
     for i in np.nonzero(merged != sel_o)[0]:
-        # selection flip: the edge must be within the near-tie band of the threshold
+        # selection flip: the edge must be within the near-tie band of the threshold (the lowest similarity the oracle merged)
         thr = np.min(sim64[sel_o]) if sel_o.any() else np.inf
         scope = (e.chunk_id == e.chunk_id[i]) if p.select == O.SELECT_CHUNK else np.ones(len(sel_o), dtype=bool)
         thr = np.min(sim64[sel_o & scope]) if (sel_o & scope).any() else thr
-        assert abs(sim64[i] - thr) <= NEAR_TIE * max(abs(thr), 1e-30) * 4, f"edge {i}: selection differs without a near tie"
+        assert abs(sim64[i] - thr) <= NEAR_TIE * max(abs(thr), 1e-30), f"edge {i}: selection differs without a near tie"
         stats["near_tie_select"] += 1
     for i in np.nonzero(merged & sel_o & (target != e.b_pos))[0]:
         a, b_g = int(e.a_pos[i]), int(target[i])
@@ -143,6 +149,20 @@ def _excuse_and_rebuild(K, V, deg, assign_gpu, e: O.Edges, sel_o, p: O.Params, s
     return Kref, Vref, dsum.astype(np.int64)
 
 
+# Excused index differences are a subset of the oracle's own near ties, and those are rare on the AR(1) workloads:
+# 3.2e-4 of the edges of the 32k workload have a top-two gap below 1e-5 relative (3.8e-5 below 1e-6, the size of the
+# kernels' fp32 error).  More excused cases than this bound means the kernel is off in more than rounding.
+NEAR_TIE_MAX_FRACTION = 5e-4
+
+
+def report_near_ties(stats: dict, what: str):
+    """One line for the record (the cases the index criterion excuses are logged), and a bound on how many there are."""
+    edges, na, ns = stats.get("edges", 0), stats.get("near_tie_argmax", 0), stats.get("near_tie_select", 0)
+    print(f"[near ties] {what}: {edges} edges, {na} argmax and {ns} selection decisions differ from the oracle inside the 1e-5 band")
+    assert na + ns <= 3 + NEAR_TIE_MAX_FRACTION * edges, f"{what}: {na + ns} excused index differences among {edges} edges"
+    return na + ns
+
+
 def gpu_cache_to_np(cache, assign=None):
     n = cache.len
     out = dict(K=to_np64(cache.k[:, :, :n]), V=to_np64(cache.v[:, :, :n]), deg=cache.deg[:, :, :n].cpu().numpy().astype(np.int64),
@@ -150,3 +170,44 @@ def gpu_cache_to_np(cache, assign=None):
     if assign is not None:
         out["assign"] = assign.cpu().numpy().astype(np.int64)
     return out
+
+
+ATTN_BAR = {"f32": 2e-4, "bf16": 2e-2}
+
+
+def check_attention(got, q, K, V, deg, scale, dtype, what, bar=None):
+    """Eq. 3 for one sequence: got [H*G, d] from the GPU against the oracle on the same stored cache (K, V [H, n, d]
+    float64, deg [H, n] or None).  Returns the achieved error, the arithmetic bound and the bias sensitivity."""
+    ref = O.app_attn(q, K, V, deg, scale)
+    err = np.abs(got - ref)
+    bar = bar if bar is not None else ATTN_BAR[dtype]
+    assert err.max() <= bar, f"{what}: max abs error {err.max():.3e} above the stated bar {bar:g}"
+    res = dict(err=float(err.max()), bound=float("nan"), sens=float("nan"), n=int(K.shape[1]))
+    if dtype == "bf16":
+        spread = O.app_attn(q, K, np.abs(V), deg, scale)          # sum_t w_t |v_t|
+        bound = 2.0 ** -9 * np.abs(ref) + 2.0 ** -8 * spread + 2e-5
+        assert np.all(err <= bound), f"{what}: error {np.max(err / bound):.2f} x the arithmetic bound (max err {err.max():.3e})"
+        res["bound"] = float(bound.max())
+    if deg is not None and np.any(deg != 1):
+        res["sens"] = float(np.abs(ref - O.app_attn(q, K, V, None, scale)).max())
+    return res
+
+
+def summarize_attention(results, what, require_sensitive=True):
+    """One line per test for the record; with degrees in play the batch must be able to expose a wrong bias."""
+    if not results:   # a batch of empty sequences
+        return 0.0
+    err = max(r["err"] for r in results)
+    bounds = [r["bound"] for r in results if r["bound"] == r["bound"]]
+    sens = [r["sens"] for r in results if r["sens"] == r["sens"]]
+    line = f"[attention] {what}: max abs err {err:.3e}"
+    if bounds:
+        line += f", arithmetic bound {max(bounds):.3e}"
+    if sens:
+        line += f", dropping log n_t moves the output by {max(sens):.3e}"
+    print(line)
+    # (judged per sequence; a handful of tokens cannot: with one token the output is that token's value whatever the bias)
+    judged = [r for r in results if r["sens"] == r["sens"] and r["bound"] == r["bound"] and r["n"] >= 256]
+    if require_sensitive and judged:
+        assert any(r["sens"] >= 5 * r["bound"] for r in judged), f"{what}: the inputs cannot expose a wrong bias: {judged}"
+    return err

@@ -88,6 +88,18 @@ def test_plan_reports_no_progress_and_bad_arguments(b):
     assert e.value.status == 6
 
 
+def test_round_cap_can_end_the_loop_above_the_budget(b):
+    """Algorithm 1's loop also ends when n_rounds_max is used up: the status is ok and the length says what happened."""
+    s = 131072
+    kw = dict(chunk=64, n_sink=16, n_recent=64, r_init=0.8, r_decay=0.2, r_min=0.2, budget=s // 4)
+    out_full, rounds_full, _ = b.compress_plan(s, b.Params(n_rounds_max=16, **kw))
+    assert out_full == s // 4 and rounds_full == 6          # Eq. 4's defaults need six rounds for a 25 % budget
+    out_cut, rounds_cut, _ = b.compress_plan(s, b.Params(n_rounds_max=3, **kw))
+    assert rounds_cut == 3 and out_cut > s // 4
+    lens = oracle_lengths(s, O.Params(n_rounds_max=3, **{k: (np.float32(v).item() if isinstance(v, float) else v) for k, v in kw.items()}))
+    assert out_cut == lens[-1]
+
+
 def test_plan_without_chunks_matches_the_oracle_lengths(b):
     """chunk = 0 (no chunking): one chunk spans the middle region; lengths after every round as the oracle counts them."""
     for s, kw in ((1000, dict(n_sink=0, n_recent=0, r_init=1.0, r_decay=0.0, r_min=1.0, n_rounds_max=2)),

@@ -51,6 +51,7 @@ def single_round_case(L, H, s, dtype, p, seed, deg_max=1, **kw):
     degn = deg.cpu().numpy().astype(np.int64) if deg is not None else np.ones((L, H, s), dtype=np.int64)
     stats = {}
     PU.check_round(PU.to_np64(K), PU.to_np64(V), degn, PU.gpu_cache_to_np(dst, assign), po, O.ratio_for_round(po, 0), dtype, stats)
+    PU.report_near_ties(stats, f"one round, chunk {p.chunk}, {L}x{H}x{s} {dtype}")
     return stats
 
 
@@ -187,6 +188,8 @@ def multi_round_check(K, V, dtype, p):
                     PU.compare_values(g["V"][l, h], Vo[l, h], dtype, "V")
         if close:
             stats["end_to_end"] = True
+            stats["edges"] = sum(len(e.a_pos) for lg in logs for e in lg.edges)
+            PU.report_near_ties(stats, f"{rounds} rounds, chunk {p.chunk}, {L}x{H}x{s} {dtype}, end to end")
             return stats
     # round by round on the GPU's own intermediates
     stats["end_to_end"] = False
@@ -202,7 +205,14 @@ def multi_round_check(K, V, dtype, p):
                        PU.gpu_cache_to_np(nxt, asg_j), PU.oracle_params(pj), r, dtype, stats)
         cur = nxt
     assert cur.len == dst.len
-    assert torch.equal(cur.k[:, :, :cur.len], dst.k[:, :, :dst.len]) and torch.equal(cur.deg[:, :, :cur.len], dst.deg[:, :, :dst.len])
+    # the single rounds reproduce the multi-round call: degrees exactly; rows bit for bit, except that two ratio-1 rounds
+    # in one pass sum a cluster on the tensor cores, whose fp32 additions may round differently from the scalar sums of a
+    # single round: there one bf16 step per round
+    assert torch.equal(cur.deg[:, :, :cur.len], dst.deg[:, :, :dst.len])
+    for a_, b_ in ((cur.k, dst.k), (cur.v, dst.v)):
+        x, y = PU.to_np64(a_[:, :, :cur.len]), PU.to_np64(b_[:, :, :dst.len])
+        assert np.all(np.abs(x - y) <= rounds * PU.bf16_ulp(y) * 1.0001 + 1e-30) and np.mean(x == y) >= 0.99
+    PU.report_near_ties(stats, f"{rounds} rounds, chunk {p.chunk}, {L}x{H}x{s} {dtype}, round by round")
     return stats
 
 

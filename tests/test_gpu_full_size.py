@@ -153,12 +153,13 @@ def test_config4_decode_batch32():
         ws = torch.empty(b.decode_workspace_bytes(Bz, H, G, D, n), dtype=torch.uint8, device=DEV)
         b.decode_attn(b.layer_views(caches, 0, DEV), H, G, q, out, scale, n, ws)
         torch.cuda.synchronize()
+        results = []
         for i in (0, 13, 31):
             c = caches[i]
             deg = c.deg[0, :, :n].cpu().numpy().astype(np.int64) if with_deg else None
-            ref = O.app_attn(PU.to_np64(q[i]), PU.to_np64(c.k[0, :, :n]), PU.to_np64(c.v[0, :, :n]), deg, scale)
-            err = np.abs(PU.to_np64(out[i]) - ref).max()
-            assert err <= 2e-2, f"slots {slots}+{extra}, sequence {i}: max abs error {err:.3e}"
+            results.append(PU.check_attention(PU.to_np64(out[i]), PU.to_np64(q[i]), PU.to_np64(c.k[0, :, :n]), PU.to_np64(c.v[0, :, :n]),
+                                              deg, scale, "bf16", f"slots {slots}+{extra}, sequence {i}"))
+        PU.summarize_attention(results, f"batch 32, {slots}+{extra} slots")
         del caches
         torch.cuda.empty_cache()
 
@@ -202,6 +203,7 @@ def test_config5_serving_mix_reduced_layers():
     wsd = torch.empty(b.decode_workspace_bytes(Bz, H, G, D, max(x.len for x in caches) + steps), dtype=torch.uint8, device=DEV)
     po = PU.oracle_params(p)
     worst = 0.0
+    results = []
     for step in range(steps):
         kn = synth.ar1_keys(L, H, Bz, D, (0.7, 0.95), 0.5, seed=5000 + step, dtype="bf16", device=DEV)   # token b of every (layer, head)
         vn = synth.normal_values(L, H, Bz, D, seed=5000 + step, dtype="bf16", device=DEV)
@@ -223,10 +225,16 @@ def test_config5_serving_mix_reduced_layers():
                 n = caches[i].len
                 np.testing.assert_array_equal(caches[i].deg[1, oh, :n].cpu().numpy(), st[2][0])
                 qs = PU.to_np64(q[i]).reshape(H, G, D)[oh].reshape(len(oh) * G, D)
-                ref = O.app_attn(qs, st[0][0], st[1][0], st[2][0], scale)
                 got = PU.to_np64(outs[1][i]).reshape(H, G, D)[oh].reshape(len(oh) * G, D)
+                # against the oracle's own replay of the cache (storage rounding of two rounds may differ by an ulp in a
+                # few rows, so the stated bar alone applies here) ...
+                ref = O.app_attn(qs, st[0][0], st[1][0], st[2][0], scale)
                 worst = max(worst, float(np.abs(got - ref).max()))
+                # ... and, with the arithmetic bound, against the oracle's attention over the GPU's stored cache
+                results.append(PU.check_attention(got, qs, PU.to_np64(caches[i].k[1, oh, :n]), PU.to_np64(caches[i].v[1, oh, :n]),
+                                                  st[2][0], scale, "bf16", f"step {step}, sequence {i}"))
     assert worst <= 2e-2, f"decode attention over the serving mix: max abs error {worst:.3e}"
+    PU.summarize_attention(results, "serving mix")
     for i, cache in enumerate(caches):   # every sequence: degrees account for every token ever written
         n = cache.len
         total = ctx[i] + steps

@@ -50,14 +50,20 @@ def paged_decode_case(P, G, with_deg, lens, H):
     b.decode_attn_paged(views, kp, vp, lp if with_deg else None, H, G, q, out, scale, max_len, ws)
     torch.cuda.synchronize()
     kpn, vpn, dpn = PU.to_np64(kp), PU.to_np64(vp), dp.cpu().numpy().astype(np.int64)
+    results = []
     for i, n in enumerate(lens):
         got = PU.to_np64(out[i])
         if n == 0:
             assert np.all(got == 0)
             continue
-        ref = O.app_attn_paged(PU.to_np64(q[i]), kpn, vpn, dpn if with_deg else None, tables[i].cpu().numpy(), n, scale)
-        err = np.abs(got - ref).max()
-        assert err <= 2e-2, f"sequence {i} (len {n}): max abs error {err:.3e}"
+        tab = tables[i].cpu().numpy()
+        # Eq. 3 over a paged cache is, by definition, Eq. 3 over the gathered sequence
+        ref = O.app_attn_paged(PU.to_np64(q[i]), kpn, vpn, dpn if with_deg else None, tab, n, scale)
+        r = PU.check_attention(got, PU.to_np64(q[i]), O.gather_pages(kpn, tab, n), O.gather_pages(vpn, tab, n),
+                               O.gather_pages(dpn, tab, n) if with_deg else None, scale, "bf16", f"sequence {i} (len {n})")
+        assert abs(np.abs(got - ref).max() - r["err"]) < 1e-12
+        results.append(r)
+    PU.summarize_attention(results, f"paged, page {P}, lens {lens}")
 
 
 @pytest.mark.parametrize("P,G,with_deg", [(64, 4, True), (32, 1, True), (128, 8, False), (64, 4, False)])
@@ -115,6 +121,11 @@ def test_pages_compress_write_back_attend():
     ref_own = O.app_attn_paged(PU.to_np64(q[0]), PU.to_np64(kp), PU.to_np64(vp), dp.cpu().numpy().astype(np.int64),
                                table[:keep].cpu().numpy(), out_len, scale)
     assert np.abs(PU.to_np64(out[0]) - ref_own).max() <= 2e-2
+    tabn = table[:keep].cpu().numpy()
+    PU.summarize_attention([PU.check_attention(PU.to_np64(out[0]), PU.to_np64(q[0]), O.gather_pages(PU.to_np64(kp), tabn, out_len),
+                                               O.gather_pages(PU.to_np64(vp), tabn, out_len),
+                                               O.gather_pages(dp.cpu().numpy().astype(np.int64), tabn, out_len), scale, "bf16",
+                                               "pages after write-back")], "pages after write-back")
     ref = O.app_attn(PU.to_np64(q[0]), Ko[0], Vo[0], do[0], scale)
     assert np.abs(PU.to_np64(out[0]) - ref).max() <= 2e-2
 

@@ -1,16 +1,19 @@
 """ckv_decode_attn_static -- the decode entry point for callers that cannot allocate device memory (no
 workspace argument; its scratch is a fixed array inside the library) -- must give the same output as
-ckv_decode_attn.  This file sorts last on purpose, so that a run that stops at the first failure has
-already run every other test."""
+ckv_decode_attn, and both must agree with the oracle.  This file sorts last on purpose, so that a run that stops
+at the first failure has already run every other test."""
 import math
 
+import numpy as np
 import pytest
 import torch
 
 from paper_2506_11418_b200 import synth
+import parity_util as PU
 
 pytestmark = pytest.mark.gpu
 DEV = "cuda"
+TOL = {"bf16": 2e-2, "f32": 2e-4}
 
 
 def _batch(b, lens, H, dtype, seed):
@@ -26,24 +29,65 @@ def _batch(b, lens, H, dtype, seed):
     return caches
 
 
-@pytest.mark.parametrize("dtype,tol", [("bf16", 2e-2), ("f32", 2e-4)])
-def test_static_scratch_matches_workspace_entry_point(dtype, tol):
+def _both_entry_points(b, caches, lens, H, G, dtype, seed):
+    scale = 1.0 / math.sqrt(128)
+    q = synth.queries(len(lens), H * G, 128, seed=seed, dtype=dtype, device=DEV)
+    ref, got = torch.zeros_like(q), torch.full_like(q, 5.0)
+    max_len = max(lens)
+    ws = torch.empty(b.decode_workspace_bytes(len(lens), H, G, 128, max_len), dtype=torch.uint8, device=DEV)
+    views = b.layer_views(caches, 0, DEV)
+    b.decode_attn(views, H, G, q, ref, scale, max_len, ws)
+    b.decode_attn_static(views, H, G, q, got, scale, max_len)
+    torch.cuda.synchronize()
+    return q, ref, got, scale
+
+
+def _against_oracle(caches, q, got, scale, dtype, which, what):
+    results = []
+    for i in which:
+        c, n = caches[i], caches[i].len
+        results.append(PU.check_attention(PU.to_np64(got[i]), PU.to_np64(q[i]), PU.to_np64(c.k[0, :, :n]), PU.to_np64(c.v[0, :, :n]),
+                                          c.deg[0, :, :n].cpu().numpy().astype(np.int64), scale, dtype, f"{what}, sequence {i}"))
+    PU.summarize_attention(results, what)
+
+
+@pytest.mark.parametrize("dtype", ["bf16", "f32"])
+def test_static_scratch_matches_workspace_entry_point(dtype):
+    """Shapes whose usual number of splits fits the fixed array: both entry points then run the same launches, so
+    the outputs are equal bit for bit.  Two calls in a row with different shapes, both through the array (16
+    (sequence, head) pairs each: more than the single-launch cluster form takes): the second finds it as the first
+    left it."""
     from paper_2506_11418_b200 import binding as b
     H, G = 4, 4
-    scale = 1.0 / math.sqrt(128)
-    # two calls in a row with different shapes: the second finds the array as the first left it
-    for call, lens in enumerate([[3000, 517, 64, 2048], [129, 4100]]):
+    for call, lens in enumerate([[3000, 517, 64, 2048], [129, 4100, 700, 33]]):
         caches = _batch(b, lens, H, dtype, seed=200 + 10 * call)
-        q = synth.queries(len(lens), H * G, 128, seed=300 + call, dtype=dtype, device=DEV)
-        ref, got = torch.zeros_like(q), torch.full_like(q, 5.0)
-        max_len = max(lens)
-        ws = torch.empty(b.decode_workspace_bytes(len(lens), H, G, 128, max_len), dtype=torch.uint8, device=DEV)
-        views = b.layer_views(caches, 0, DEV)
-        b.decode_attn(views, H, G, q, ref, scale, max_len, ws)
-        b.decode_attn_static(views, H, G, q, got, scale, max_len)
-        torch.cuda.synchronize()
+        q, ref, got, scale = _both_entry_points(b, caches, lens, H, G, dtype, seed=300 + call)
         err = (got.float() - ref.float()).abs().max().item()
-        assert err <= tol, f"call {call}: static-scratch output differs from the workspace entry point by {err}"
+        assert err <= TOL[dtype], f"call {call}: static-scratch output differs from the workspace entry point by {err}"
+        assert torch.equal(got, ref), f"call {call}: same launches, yet the outputs differ"
+        _against_oracle(caches, q, got, scale, dtype, range(len(lens)), f"static scratch, call {call}")
+
+
+@pytest.mark.parametrize("dtype", ["bf16", "f32"])
+@pytest.mark.parametrize("Bz,top,splits", [(40, 9000, 3), (64, 1024, 1)])
+def test_static_scratch_with_fewer_splits_than_usual(dtype, Bz, top, splits):
+    """Batches whose usual split count does not fit 1 Mi floats: 40 x 8 x 8 query heads x 132 floats leave room for
+    three splits (not a multiple of the four warps of a CTA), 64 x 8 x 8 for one.  The partial sums are then grouped
+    differently from the workspace entry point's, so the two agree within the attention tolerance, not bit for bit;
+    sampled sequences are checked against the oracle.  Two calls in a row."""
+    from paper_2506_11418_b200 import binding as b
+    H, G = 8, 8
+    assert (1 << 20) // (Bz * H * G * 132) == splits
+    rng = np.random.default_rng(Bz)
+    for call in range(2):
+        lens = [top] + [int(x) for x in rng.integers(1, top + 1, Bz - 1)]
+        caches = _batch(b, lens, H, dtype, seed=400 + 100 * call)
+        q, ref, got, scale = _both_entry_points(b, caches, lens, H, G, dtype, seed=500 + call)
+        err = (got.float() - ref.float()).abs().max().item()
+        assert err <= TOL[dtype], f"call {call}: static-scratch output differs from the workspace entry point by {err}"
+        _against_oracle(caches, q, got, scale, dtype, (0, Bz // 2), f"static scratch, {splits} split(s), call {call}")
+        del caches
+        torch.cuda.empty_cache()
 
 
 def test_static_scratch_rejects_what_does_not_fit():
