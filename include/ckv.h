@@ -117,6 +117,15 @@ int ckv_compress_prefill(const ckv_cache* src, ckv_cache* dst, const ckv_params*
 int ckv_compress_append(ckv_cache* cache, const void* k_new, const void* v_new, int32_t t_new,
                         const ckv_params* params, void* workspace, size_t workspace_bytes, void* cuda_stream);
 
+/* The same step for Bz sequences that decode in lock step: one new token per sequence, written by a single launch
+ * (a serving batch of 64 otherwise pays 64 one-token copy launches per step).  caches: HOST array [Bz] of caches
+ * with the same L, H, D and dtype; k_new, v_new: device [L, H, Bz, D], token b belongs to caches[b].  A sequence
+ * whose appended tail reaches `chunk` tokens has that window clustered exactly as ckv_compress_append does; the host
+ * fields len and pending of every cache are updated.  Workspace: ckv_workspace_bytes of any of the caches.  Nothing is
+ * enqueued if an argument check fails (CKV_ERR_CAPACITY if some cache is full). */
+int ckv_compress_append_batch(ckv_cache* caches, int32_t Bz, const void* k_new, const void* v_new, const ckv_params* params,
+                              void* workspace, size_t workspace_bytes, void* cuda_stream);
+
 /* Algorithm 1, decoding branch, as printed: `K = [K, k], V = [V, v], N = [N, 1]`, and `if s >= B + g` one call of
  * CentroidKV over the whole cache, with B = params->budget (> 0) and g = interval (> 0).  The round keeps the sinks
  * and recent tokens, carries the degrees along, uses the ratio of round 0 (params->r_init; n_rounds_max is not

@@ -18,7 +18,7 @@ F32, BF16 = 0, 1
 SELECT_GLOBAL, SELECT_CHUNK = 0, 1
 OK = 0
 
-EXPORTS = ["ckv_compress_plan", "ckv_workspace_bytes", "ckv_compress_prefill", "ckv_compress_append",
+EXPORTS = ["ckv_compress_plan", "ckv_workspace_bytes", "ckv_compress_prefill", "ckv_compress_append", "ckv_compress_append_batch",
            "ckv_decode_workspace_bytes", "ckv_decode_attn", "ckv_status_string", "ckv_workspace_status",
            "ckv_decode_attn_static", "ckv_compress_append_recluster", "ckv_decode_attn_paged", "ckv_pages_gather",
            "ckv_pages_scatter"]
@@ -58,6 +58,9 @@ def _load():
     lib.ckv_compress_append.restype = C.c_int
     lib.ckv_compress_append.argtypes = [C.POINTER(CkvCache), C.c_void_p, C.c_void_p, C.c_int32, C.POINTER(CkvParams),
                                         C.c_void_p, C.c_size_t, C.c_void_p]
+    lib.ckv_compress_append_batch.restype = C.c_int
+    lib.ckv_compress_append_batch.argtypes = [C.POINTER(CkvCache), C.c_int32, C.c_void_p, C.c_void_p, C.POINTER(CkvParams),
+                                              C.c_void_p, C.c_size_t, C.c_void_p]
     lib.ckv_compress_append_recluster.restype = C.c_int
     lib.ckv_compress_append_recluster.argtypes = [C.POINTER(CkvCache), C.POINTER(CkvCache), C.c_void_p, C.c_void_p, C.c_int32,
                                                   C.POINTER(CkvParams), C.c_int32, C.c_void_p, C.c_size_t, C.c_void_p,
@@ -195,6 +198,17 @@ def compress_append(cache: Cache, k_new: torch.Tensor, v_new: torch.Tensor, para
     _check(lib.ckv_compress_append(C.byref(cc), k_new.data_ptr(), v_new.data_ptr(), k_new.shape[2], C.byref(params.c()),
                                    workspace.data_ptr(), workspace.numel() * workspace.element_size(), _stream_ptr()))
     cache.len, cache.pending = cc.len, cc.pending
+
+
+def compress_append_batch(caches, k_new: torch.Tensor, v_new: torch.Tensor, params: Params, workspace: torch.Tensor):
+    """ckv_compress_append_batch on the current stream: one new token for each cache of the list (k_new, v_new:
+    [L, H, len(caches), D]); every cache's len / pending are updated."""
+    assert k_new.is_contiguous() and v_new.is_contiguous() and k_new.shape == v_new.shape and k_new.shape[2] == len(caches)
+    arr = (CkvCache * len(caches))(*[c.c() for c in caches])
+    _check(lib.ckv_compress_append_batch(arr, len(caches), k_new.data_ptr(), v_new.data_ptr(), C.byref(params.c()),
+                                         workspace.data_ptr(), workspace.numel() * workspace.element_size(), _stream_ptr()))
+    for c, cc in zip(caches, arr):
+        c.len, c.pending = cc.len, cc.pending
 
 
 def compress_append_recluster(cache: Cache, spare: Cache, k_new: torch.Tensor, v_new: torch.Tensor, params: Params,

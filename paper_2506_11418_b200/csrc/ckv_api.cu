@@ -325,6 +325,26 @@ int64_t dst_cap_needed(const std::vector<RoundPlan>& plan, int64_t len) {
   return need;
 }
 
+// A completed window of `c` appended tokens at the tail of the cache is clustered on its own: copied aside, then the
+// planned rounds run back into its place.  cache->len is updated.
+int cluster_window(ckv_cache* cache, const std::vector<RoundPlan>& plan, int64_t win_out, int64_t LH, int D, int es, int c,
+                   Workspace& w, unsigned char* ws, const Buf& stage, cudaStream_t stream) {
+  const int64_t w0 = cache->len - c;
+  CopyArgs out{};
+  out.k_src = cache->k; out.v_src = cache->v; out.deg_src = cache->deg;
+  out.k_dst = stage.k; out.v_dst = stage.v; out.deg_dst = stage.deg; out.logdeg_dst = stage.logdeg;
+  out.src_cap = cache->cap; out.dst_cap = c; out.src_off = w0; out.dst_off = 0; out.count = c; out.LH = (int)LH;
+  if (launch_copy(out, cache->dtype, D, stream) != cudaSuccess) return CKV_ERR_CUDA;
+  // the window's destination is a view of the cache that starts at w0
+  const Buf dstw{static_cast<unsigned char*>(cache->k) + (size_t)w0 * D * es,
+                 static_cast<unsigned char*>(cache->v) + (size_t)w0 * D * es, cache->deg + w0,
+                 cache->logdeg ? cache->logdeg + w0 : nullptr, cache->cap};
+  const int st = run_plan(plan, stage, dstw, c, (int)LH, D, cache->dtype, c, nullptr, w, ws, stream);
+  if (st != CKV_OK) return st;
+  cache->len = w0 + win_out;
+  return CKV_OK;
+}
+
 ckv_params window_params(const ckv_params& p) {
   ckv_params wp = p;
   wp.n_sink = 0;
@@ -473,22 +493,67 @@ int ckv_compress_append(ckv_cache* cache, const void* k_new, const void* v_new, 
     cache->pending += take;
     done += take;
     if (cache->pending == c && !plan.empty()) {
-      // cluster the completed window: copy it aside, then run the rounds back into its place
-      const int64_t w0 = cache->len - c;
-      CopyArgs out{};
-      out.k_src = cache->k; out.v_src = cache->v; out.deg_src = cache->deg;
-      out.k_dst = stage.k; out.v_dst = stage.v; out.deg_dst = stage.deg; out.logdeg_dst = stage.logdeg;
-      out.src_cap = cache->cap; out.dst_cap = c; out.src_off = w0; out.dst_off = 0; out.count = c; out.LH = (int)LH;
-      if (launch_copy(out, cache->dtype, D, stream) != cudaSuccess) return CKV_ERR_CUDA;
-      // the window's destination is a view of the cache that starts at w0
-      const Buf dstw{static_cast<unsigned char*>(cache->k) + (size_t)w0 * D * es,
-                     static_cast<unsigned char*>(cache->v) + (size_t)w0 * D * es, cache->deg + w0,
-                     cache->logdeg ? cache->logdeg + w0 : nullptr, cache->cap};
-      st = run_plan(plan, stage, dstw, c, (int)LH, D, cache->dtype, c, nullptr, w, ws, stream);
-      if (st != CKV_OK) return st;
-      cache->len = w0 + win_out;
+      if ((st = cluster_window(cache, plan, win_out, LH, D, es, c, w, ws, stage, stream)) != CKV_OK) return st;
     }
     if (cache->pending == c) cache->pending = 0;
+  }
+  return CKV_OK;
+}
+
+int ckv_compress_append_batch(ckv_cache* caches, int32_t Bz, const void* k_new, const void* v_new, const ckv_params* params,
+                              void* workspace, size_t workspace_bytes, void* cuda_stream) {
+  int st;
+  if ((st = check_params(params)) != CKV_OK) return st;
+  if (!caches || Bz <= 0 || !k_new || !v_new) return CKV_ERR_INVALID_ARG;
+  if (params->chunk == 0) return CKV_ERR_INVALID_ARG;
+  if (!aligned16(k_new) || !aligned16(v_new)) return CKV_ERR_ALIGNMENT;
+  const ckv_cache& c0 = caches[0];
+  for (int32_t b = 0; b < Bz; ++b) {
+    const ckv_cache& cb = caches[b];
+    if ((st = check_cache_shape(&cb)) != CKV_OK) return st;
+    if (cb.L != c0.L || cb.H != c0.H || cb.D != c0.D || cb.dtype != c0.dtype) return CKV_ERR_INVALID_ARG;
+    if (!cb.k || !cb.v || !cb.deg) return CKV_ERR_INVALID_ARG;
+    if (!aligned16(cb.k) || !aligned16(cb.v)) return CKV_ERR_ALIGNMENT;
+    if (cb.pending >= params->chunk) return CKV_ERR_INVALID_ARG;
+    if (cb.len + 1 > cb.cap) return CKV_ERR_CAPACITY;
+  }
+  const int64_t LH = (int64_t)c0.L * c0.H;
+  const int D = c0.D, es = esize_of(c0.dtype), c = params->chunk;
+  const ckv_params wp = window_params(*params);
+  std::vector<RoundPlan> plan;
+  if ((st = plan_rounds(c, wp, plan)) != CKV_OK) return st;
+  const int64_t win_out = plan.empty() ? c : plan.back().s_out;
+  Workspace w = layout_workspace(LH, D, es, c, plan, false);
+  const size_t base = w.total;
+  const size_t win_kv = align_up((size_t)LH * c * D * es), win_dg = align_up((size_t)LH * c * 4);
+  if (!workspace || workspace_bytes < base + 2 * win_kv + 2 * win_dg || !aligned16(workspace)) return CKV_ERR_WORKSPACE;
+  unsigned char* ws = static_cast<unsigned char*>(workspace);
+  const Buf stage{ws + base, ws + base + win_kv, reinterpret_cast<int32_t*>(ws + base + 2 * win_kv),
+                  reinterpret_cast<float*>(ws + base + 2 * win_kv + win_dg), c};
+  cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
+  if (cudaMemsetAsync(workspace, 0, 256, stream) != cudaSuccess) return CKV_ERR_CUDA;
+
+  // K = [K, k], V = [V, v], N = [N, 1] for every sequence: one launch per kAppendBatchMax sequences
+  for (int32_t first = 0; first < Bz; first += kAppendBatchMax) {
+    AppendBatchArgs a{};
+    a.k_new = k_new; a.v_new = v_new;
+    a.n = std::min<int32_t>(kAppendBatchMax, Bz - first);
+    a.first = first; a.n_total = Bz; a.LH = (int32_t)LH;
+    for (int32_t i = 0; i < a.n; ++i) {
+      const ckv_cache& cb = caches[first + i];
+      a.k[i] = cb.k; a.v[i] = cb.v; a.deg[i] = cb.deg; a.logdeg[i] = cb.logdeg;
+      a.cap[i] = cb.cap; a.len[i] = cb.len;
+    }
+    if (launch_append_batch(a, c0.dtype, D, stream) != cudaSuccess) return CKV_ERR_CUDA;
+  }
+  for (int32_t b = 0; b < Bz; ++b) {
+    ckv_cache* cb = &caches[b];
+    cb->len += 1;
+    cb->pending += 1;
+    if (cb->pending == c) {
+      if (!plan.empty() && (st = cluster_window(cb, plan, win_out, LH, D, es, c, w, ws, stage, stream)) != CKV_OK) return st;
+      cb->pending = 0;
+    }
   }
   return CKV_OK;
 }

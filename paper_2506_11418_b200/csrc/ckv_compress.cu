@@ -265,6 +265,27 @@ __global__ void __launch_bounds__(256) copy_rows_kernel(const CopyArgs a) {
   }
 }
 
+// Algorithm 1, decoding branch, K = [K, k], V = [V, v], N = [N, 1] for a batch of sequences in one launch: block
+// (x, lh) copies the rows of slab lh, one 16-byte piece per thread.
+template <typename T, int D>
+__global__ void __launch_bounds__(256) append_batch_kernel(const __grid_constant__ AppendBatchArgs a) {
+  constexpr int kVecPerRow = D * (int)sizeof(T) / 16;
+  const int lh = blockIdx.y;
+  const int nvec = a.n * kVecPerRow;
+  for (int i = blockIdx.x * blockDim.x + threadIdx.x; i < nvec; i += gridDim.x * blockDim.x) {
+    const int b = i / kVecPerRow, piece = i - b * kVecPerRow;
+    const int64_t src = ((int64_t)lh * a.n_total + a.first + b) * kVecPerRow + piece;
+    const int64_t dst = ((int64_t)lh * a.cap[b] + a.len[b]) * kVecPerRow + piece;
+    reinterpret_cast<uint4*>(a.k[b])[dst] = reinterpret_cast<const uint4*>(a.k_new)[src];
+    reinterpret_cast<uint4*>(a.v[b])[dst] = reinterpret_cast<const uint4*>(a.v_new)[src];
+    if (piece == 0) {
+      const int64_t di = (int64_t)lh * a.cap[b] + a.len[b];
+      a.deg[b][di] = 1;
+      if (a.logdeg[b]) a.logdeg[b][di] = 0.f;
+    }
+  }
+}
+
 // ---- Sec. 5.3, ranking across all chunks of one (layer, head) ---------------------------------
 // Exact top-M of the edges by (similarity descending, position ascending): a 4 x 8-bit radix
 // select finds the M-th largest similarity, then one pass in position order resolves ties at the
@@ -460,6 +481,18 @@ cudaError_t launch_copy(const CopyArgs& a, int dtype, int D, cudaStream_t st) {
     copy_rows_kernel<float, 128><<<grid, 256, 0, st>>>(a);
   else
     copy_rows_kernel<__nv_bfloat16, 128><<<grid, 256, 0, st>>>(a);
+  return cudaGetLastError();
+}
+
+cudaError_t launch_append_batch(const AppendBatchArgs& a, int dtype, int D, cudaStream_t st) {
+  if (D != 128) return cudaErrorInvalidValue;
+  if (a.n <= 0) return cudaSuccess;
+  const int nvec = a.n * (D * (dtype == 0 ? 4 : 2) / 16);
+  const dim3 grid((unsigned)((nvec + 255) / 256), (unsigned)a.LH);
+  if (dtype == 0)
+    append_batch_kernel<float, 128><<<grid, 256, 0, st>>>(a);
+  else
+    append_batch_kernel<__nv_bfloat16, 128><<<grid, 256, 0, st>>>(a);
   return cudaGetLastError();
 }
 

@@ -60,6 +60,24 @@ struct CopyArgs {
   int32_t LH;
 };
 
+// One new token (degree 1) for each of up to kAppendBatchMax sequences: token b of k_new / v_new [LH, n_total, D] goes
+// to slot len[b] of sequence b.
+constexpr int kAppendBatchMax = 64;
+struct AppendBatchArgs {
+  const void* k_new;
+  const void* v_new;
+  void* k[kAppendBatchMax];
+  void* v[kAppendBatchMax];
+  int32_t* deg[kAppendBatchMax];
+  float* logdeg[kAppendBatchMax];  // entries may be null
+  int64_t cap[kAppendBatchMax];
+  int64_t len[kAppendBatchMax];
+  int32_t n;        // sequences in this launch
+  int32_t first;    // index of the first of them in k_new / v_new
+  int32_t n_total;  // sequences in k_new / v_new
+  int32_t LH;
+};
+
 struct SelectArgs {
   const float* edge_sim;
   uint8_t* sel;
@@ -122,6 +140,7 @@ inline cudaError_t launch_dependent(void (*kernel)(KArgs...), dim3 grid, dim3 bl
 cudaError_t launch_round(const RoundArgs& a, int dtype, int D, cudaStream_t st);
 cudaError_t launch_copy(const CopyArgs& a, int dtype, int D, cudaStream_t st);
 cudaError_t launch_select(const SelectArgs& a, cudaStream_t st);
+cudaError_t launch_append_batch(const AppendBatchArgs& a, int dtype, int D, cudaStream_t st);
 cudaError_t launch_compose_assign(int32_t* total, const int32_t* step, int64_t n_src, int64_t step_stride, int32_t LH,
                                   cudaStream_t st);
 cudaError_t launch_decode(const DecodeArgs& a, int dtype, int D, cudaStream_t st);

@@ -303,6 +303,66 @@ def test_append_with_chunk_trigger(dtype):
                     PU.compare_values(g["V"][l, h], Vo[l, h], dtype, "V")
 
 
+@pytest.mark.parametrize("dtype,Bz", [("bf16", 5), ("f32", 3), ("bf16", 70)])
+def test_append_batch_in_lock_step(dtype, Bz):
+    """One new token per sequence and step, all sequences written by one launch (two past 64 sequences); the sequences
+    start with different lengths and different numbers of pending tokens, so their windows complete at different steps.
+    Every sequence is replayed by the oracle, and a second set of caches driven one sequence at a time through
+    ckv_compress_append must end up identical bit for bit."""
+    b = B()
+    L, H, c, steps = 2, 2, 64, 70
+    p = b.Params(chunk=c, n_sink=0, n_recent=0, n_rounds_max=2, r_init=1.0, r_decay=0.0, r_min=1.0, select=b.SELECT_GLOBAL)
+    po = PU.oracle_params(p)
+    rng = np.random.default_rng(Bz)
+    lens = [int(x) for x in rng.integers(1, 200, Bz)]
+    pend0 = [int(min(n, x)) for n, x in zip(lens, rng.integers(0, c, Bz))]
+    replay = range(Bz) if Bz <= 8 else (0, 63, 64, Bz - 1)      # sequences the oracle follows
+    batch, single, oracle = [], [], {}
+    for i, n in enumerate(lens):
+        K, V, _ = make_inputs(L, H, n, dtype, seed=500 + i)
+        for group in (batch, single):
+            cache = b.Cache.empty(L, H, n + steps + 3, 128, K.dtype, DEV)
+            cache.k[:, :, :n], cache.v[:, :, :n] = K, V
+            cache.deg[:, :, :n] = 1
+            cache.len, cache.pending = n, pend0[i]
+            group.append(cache)
+        if i in replay:
+            oracle[i] = [PU.to_np64(K), PU.to_np64(V), np.ones((L, H, n), dtype=np.int64), pend0[i]]
+    ws = torch.empty(max(b.workspace_bytes(x, p) for x in batch), dtype=torch.uint8, device=DEV)
+    for step in range(steps):
+        kn, vn, _ = make_inputs(L, H, Bz, dtype, seed=900 + step)
+        b.compress_append_batch(batch, kn, vn, p, ws)
+        for i, cache in enumerate(single):
+            b.compress_append(cache, kn[:, :, i:i + 1].contiguous(), vn[:, :, i:i + 1].contiguous(), p, ws)
+        for i, st in oracle.items():
+            st[0], st[1], st[2], st[3] = O.compress_append(st[0], st[1], st[2], st[3], PU.to_np64(kn[:, :, i:i + 1]),
+                                                           PU.to_np64(vn[:, :, i:i + 1]), po, storage=dtype)
+            assert batch[i].len == st[0].shape[2] and batch[i].pending == st[3]
+    assert b.workspace_status(ws) == 0
+    for x, y in zip(batch, single):
+        n = x.len
+        assert n == y.len and x.pending == y.pending
+        assert torch.equal(x.k[:, :, :n], y.k[:, :, :n]) and torch.equal(x.v[:, :, :n], y.v[:, :, :n])
+        assert torch.equal(x.deg[:, :, :n], y.deg[:, :, :n]) and torch.equal(x.logdeg[:, :, :n], y.logdeg[:, :, :n])
+    for i, (Ko, Vo, do, _) in oracle.items():
+        g = PU.gpu_cache_to_np(batch[i])
+        np.testing.assert_array_equal(g["deg"], do)
+        np.testing.assert_allclose(g["logdeg"], np.log(do.astype(np.float64)), rtol=1e-6, atol=1e-7)
+        for l in range(L):
+            for h in range(H):
+                if dtype == "bf16":
+                    assert np.all(np.abs(g["K"][l, h] - Ko[l, h]) <= 2 * PU.bf16_ulp(Ko[l, h]) * 1.0001)
+                    assert np.all(np.abs(g["V"][l, h] - Vo[l, h]) <= 2 * PU.bf16_ulp(Vo[l, h]) * 1.0001 + 1e-30)
+                else:
+                    PU.compare_values(g["K"][l, h], Ko[l, h], dtype, "K")
+                    PU.compare_values(g["V"][l, h], Vo[l, h], dtype, "V")
+    # a full cache is refused before anything is enqueued
+    batch[0].len = batch[0].cap
+    with pytest.raises(b.CkvError) as e:
+        b.compress_append_batch(batch, kn, vn, p, ws)
+    assert e.value.status == 3
+
+
 def test_status_codes_on_device_buffers():
     b = B()
     K, V, _ = make_inputs(1, 1, 256, "bf16", seed=1)
