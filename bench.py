@@ -41,11 +41,17 @@ def measured_peaks():
 
 # --------------------------------------------------------------------------- algorithmic bytes
 
-def compress_bytes(L, H, s, D, es, keep):
-    """Per token-vector: K and V read, the kept fraction of K and V written, degrees in (4 B) and
-    degree + log-degree out (8 B per kept slot)."""
-    per_vec = 2 * D * es + keep * 2 * D * es + 4 + keep * 8
+def compress_bytes(L, H, s, D, es, keep, with_deg=False):
+    """One round, per token-vector: K and V read, the kept fraction of K and V written, degree + log-degree out (8 B per
+    kept slot); the 4-byte degree read only when the source carries degrees (a cache straight from prefill does not)."""
+    per_vec = 2 * D * es + keep * 2 * D * es + (4 if with_deg else 0) + keep * 8
     return L * H * s * per_vec
+
+
+def schedule_bytes(L, H, s, out_len, D, es):
+    """A whole schedule, whatever its number of rounds: what the method itself has to move is one read of the source
+    and one write of the final cache (intermediate caches are an implementation's own traffic)."""
+    return L * H * (s * 2 * D * es + out_len * (2 * D * es + 8))
 
 
 def decode_bytes(rows, D, es):
@@ -55,10 +61,10 @@ def decode_bytes(rows, D, es):
 
 # --------------------------------------------------------------------------- DRAM traffic from the ncu capture
 
-# dram__bytes_read.sum + dram__bytes_write.sum of round_fast_kernel per token-vector, from the capture summarised in
-# profiles/round_fast_kernel_llama8b_4layers.md (1 048 576 token-vectors per launch; traffic grows in proportion to
-# the token-vectors processed, so it is scaled to the launch timed here).  Valid only for the kernel source it
-# was taken from: the digest below is of ckv_compress_fast.cu at that time.
+# dram__bytes_read.sum + dram__bytes_write.sum of round_fast_kernel per token-vector, from an ncu capture of a 4-layer
+# cut of the workload (1 048 576 token-vectors per launch; traffic grows in proportion to the token-vectors processed,
+# so it is scaled to the launch timed here).  Valid only for the kernel source it was taken from: the digest below is
+# of ckv_compress_fast.cu at that time.
 NCU_TRAFFIC = {"bytes_per_token_vector": (536905472 + 238534912) / 1048576,
                "source": "paper_2506_11418_b200/csrc/ckv_compress_fast.cu",
                "sha256": "cac8149dd5cca459a65579e8f4920999a6aab09152ec97f72602ed07318a0b1a"}
@@ -159,20 +165,88 @@ def oracle_pass(x) -> float:
         return time.perf_counter() - t0
 
 
+_WORKER_INPUT = None
+
+
+def _oracle_worker_init():
+    """Each worker process draws one (layer, head) slab of the workload and keeps it."""
+    global _WORKER_INPUT
+    import torch
+    torch.set_num_threads(1)
+    _WORKER_INPUT = oracle_inputs(1, seed=os.getpid() % 9973)
+
+
+def _oracle_worker_pass(_):
+    return oracle_pass(_WORKER_INPUT)
+
+
+class OraclePool:
+    """The oracle on the host's cores: one single-threaded NumPy process per core, each working through (layer, head)
+    slabs (the method is independent per slab; the oracle itself is not changed or tuned for this).  Must be created
+    before this process touches CUDA (the workers are forked)."""
+
+    MAX_PROCS = 64
+
+    def __init__(self):
+        import multiprocessing as mp
+        self.cores_available = len(os.sched_getaffinity(0)) if hasattr(os, "sched_getaffinity") else (os.cpu_count() or 1)
+        self.cores = max(1, min(self.cores_available, self.MAX_PROCS))
+        self.pool = mp.get_context("fork").Pool(self.cores, initializer=_oracle_worker_init)
+        cfg = __import__("paper_2506_11418_b200.synth", fromlist=["CONFIGS"]).CONFIGS[WORKLOAD]
+        self.tokens_per_slab = cfg["s"] / (cfg["L"] * cfg["H"])
+        self.slabs_total = cfg["L"] * cfg["H"]
+
+    def run(self, n_slabs: int) -> float:
+        """Wall seconds for n_slabs passes spread over the workers."""
+        t0 = time.perf_counter()
+        self.pool.map(_oracle_worker_pass, range(n_slabs), chunksize=1)
+        return time.perf_counter() - t0
+
+    def describe(self, n_slabs: int) -> str:
+        return (f"{n_slabs} of {self.slabs_total} (layer, head) slabs of {WORKLOAD}: compress + append 64 + 1 decode step each, "
+                f"{self.cores} single-threaded worker processes (host offers {self.cores_available} cores)")
+
+    def close(self):
+        self.pool.close()
+        self.pool.join()
+
+
+def cpu_baseline(pool: OraclePool, target_s: float = 12.0):
+    """About target_s seconds of oracle work on every core: one slab per core first (which also sizes the sample)."""
+    t1 = pool.run(pool.cores)
+    rounds = max(1, min(30, int(round(target_s / max(t1, 1e-3)))))
+    n = rounds * pool.cores
+    dt = pool.run(n)
+    return {"value": n * pool.tokens_per_slab / dt, "unit": UNIT, "cores": pool.cores, "cores_available": pool.cores_available,
+            "kind": "oracle", "sample": pool.describe(n), "seconds": dt}
+
+
+def workload_config(L=None):
+    from paper_2506_11418_b200 import synth
+    cfg = synth.CONFIGS[WORKLOAD]
+    L = L or cfg["L"]
+    return {"workload": WORKLOAD if L == cfg["L"] else f"{WORKLOAD} cut to {L} layers (not the benchmark workload)", "layers": L,
+            "kv_heads": cfg["H"], "q_heads": cfg["H"] * cfg["G"], "head_dim": cfg["d"], "seq": cfg["s"], "chunk": cfg["chunk"],
+            "retain": 0.5, "step": "compress_prefill + append 64 + decode all layers", "l2": "inputs (4 GiB) exceed L2",
+            "clock_samples_cover": "warm-up (at least 0.3 s of it) and the timed region"}
+
+
 def run_reference(args):
     if int(os.environ.get("RANK", "0")) != 0:
         return  # under a multi-rank launch rank 0 alone times the oracle
-    x = oracle_inputs(2)
-    for _ in range(min(args.warmup, 1)):
-        oracle_pass(x)
-    times = [oracle_pass(x) for _ in range(args.steps)]
+    pool = OraclePool()
+    n = pool.cores  # a step: one slab of the workload on every core
+    for _ in range(min(args.warmup, 2)):
+        pool.run(n)
+    times = [pool.run(n) for _ in range(args.steps)]
+    pool.close()
     total = sum(times)
-    value = x["tokens"] * len(times) / total
+    value = n * pool.tokens_per_slab * len(times) / total
     line = {"impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus, "steps": args.steps,
             "warmup": args.warmup, "ms_per_step": 1e3 * total / len(times), "higher_is_better": True, "scaling": "weak",
-            "vs_baseline": None, "dtype": "f64", "data": "synthetic",
-            "config": {"workload": WORKLOAD, "sample": x["desc"]},
-            "cpu_baseline": {"value": value, "unit": UNIT, "cores": 1, "kind": "oracle", "sample": x["desc"]},
+            "vs_baseline": None, "dtype": "f64", "data": "synthetic", "config": workload_config(),
+            "cpu_baseline": {"value": value, "unit": UNIT, "cores": pool.cores, "cores_available": pool.cores_available,
+                             "kind": "oracle", "sample": "per step: " + pool.describe(n)},
             "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0}}
     print(json.dumps(line))
 
@@ -185,6 +259,12 @@ def run_gpu(args):
     from paper_2506_11418_b200 import binding as b, parallel, synth
 
     rank, local, world = parallel.env_world()
+    # the CPU baseline first: its worker processes are forked, which has to happen before this process touches CUDA
+    cpu = None
+    if rank == 0 and world == 1 and not args.skip_cpu:
+        pool = OraclePool()
+        cpu = cpu_baseline(pool)
+        pool.close()
     if not torch.cuda.is_available():
         raise SystemExit("bench.py needs a CUDA device; there is no CPU fallback")
     torch.cuda.set_device(local)
@@ -243,10 +323,19 @@ def run_gpu(args):
     def barrier():
         parallel.barrier(dev)
 
+    # the clock sampler runs from before the warm-up to after the timed region; the warm-up is stretched to at least
+    # 0.3 s so that the record has samples under load however short the timed region is
+    sampler = ClockSampler(local) if rank == 0 else None
+    t_warm = time.perf_counter()
     for _ in range(max(args.warmup, 3)):
         step(False)
+    torch.cuda.synchronize()
+    untimed = max(args.warmup, 3)
+    while time.perf_counter() - t_warm < 0.3:
+        step(False)
+        torch.cuda.synchronize()
+        untimed += 1
     barrier()
-    sampler = ClockSampler(local) if rank == 0 else None
     t_start, t_end = ev(), ev()
     t_start.record()
     for _ in range(args.steps):
@@ -261,16 +350,19 @@ def run_gpu(args):
     comp_ms = statistics.mean(a.elapsed_time(z) for a, z in comp_ev)
     dec_ms = statistics.mean(a.elapsed_time(z) for a, z in dec_ev)
     peaks, peak_kind = measured_peaks()
-    cbytes = compress_bytes(L, H, s, D, es, out_len / s)
+    peak = peaks["hbm_gbs"]
+    cbytes = compress_bytes(L, H, s, D, es, out_len / s, with_deg=False)   # the timed call passes no source degrees
     achieved = cbytes / (comp_ms * 1e-3) / 1e9
-    roofline = {"bound": "hbm", "kernel": "compress round kernel (one launch per ckv_compress_prefill)", "achieved": achieved,
-                "peak": peaks["hbm_gbs"], "peak_kind": peak_kind, "unit": "GB/s", "frac": achieved / peaks["hbm_gbs"],
+    roofline = {"bound": "hbm", "kernel": "round_fast_kernel (the one launch of ckv_compress_prefill at chunk 64, ratio 1)",
+                "achieved": achieved, "peak": peak, "peak_kind": peak_kind + " copy bandwidth (MEASURED_PEAKS.json)" if peak_kind == "measured" else peak_kind,
+                "unit": "GB/s", "frac": achieved / peak,
                 "traffic": ncu_traffic(L * H * s), "bytes_per_launch": cbytes, "ms_per_launch": comp_ms,
                 "frac_of_nominal_8tbs": achieved / 8000.0}
     dbytes = decode_bytes(H * final_len, D, es)
     dec_achieved = dbytes * L / (dec_ms * 1e-3) / 1e9
     extra = {"compress_ms": comp_ms, "compress_tokens_per_s": s / (comp_ms * 1e-3), "decode_ms_all_layers": dec_ms,
-             "decode_gbs_batch1": dec_achieved}
+             "decode_gbs_batch1": dec_achieved, "untimed_steps_before_the_timed_region": untimed}
+    targets = {}
 
     if rank == 0:
         # the same step captured once into a CUDA graph and replayed: what the GPU needs when the host issues nothing
@@ -287,15 +379,17 @@ def run_gpu(args):
         torch.cuda.synchronize()
         extra["step_from_cuda_graph_ms"] = g0.elapsed_time(g1) / args.steps
         del graph
-    if rank == 0 and not args.skip_decode_cfg4:
-        extra["decode_cfg4"] = bench_decode_cfg4(b, synth, dev, peaks["hbm_gbs"])
-        extra["decode_cfg4_paged"] = bench_decode_paged(b, synth, dev, peaks["hbm_gbs"])
-    if rank == 0 and not args.skip_serving and args.layers == 0:
-        extra["serving_mix"] = bench_serving_mix(b, synth, dev, peaks["hbm_gbs"])
     if rank == 0 and not args.skip_variants:
-        extra["compress_variants"] = bench_compress_variants(b, synth, dev, K, V, peaks["hbm_gbs"], args.layers == 0)
+        extra["compress_variants"] = bench_compress_variants(b, synth, dev, K, V, peak, args.layers == 0)
         extra["recluster"] = bench_recluster(b, synth, dev, K, V)
         extra["no_chunk"] = bench_no_chunk(b, synth, dev, K, V, peaks, args.layers == 0)
+        cv = extra["compress_variants"]
+        pick = lambda name: {k: cv[name][k] for k in ("ms", "frac_of_peak", "gbs", "moved_gb", "frac_on_moved_bytes")} if name in cv else None
+        targets["chunk256_ratio1"] = pick("chunk256 ratio1")
+        targets["chunk256_ratio0.8_ranked_per_head"] = pick("chunk256 ratio0.8 ranked per head")
+        targets["chunk256_paper_schedule_to_25pct"] = pick("chunk256 paper schedule to 25%")
+        targets["cfg3_128k_two_rounds_to_25pct"] = pick("llama8b_128k chunk64 two rounds ratio1 (to 25%)")
+        targets["cfg3_128k_paper_schedule_to_25pct"] = pick("llama8b_128k chunk64 paper schedule to 25%")
 
     # end to end: inputs start in pinned host memory, the compressed cache and the decode output end there
     e2e = None
@@ -304,22 +398,30 @@ def run_gpu(args):
         if world > 1:
             e2e["ms_per_step"] = parallel.max_over_ranks(e2e["ms_per_step"], dev)
             e2e["value"] = world * s / (e2e["ms_per_step"] * 1e-3)
-
-    cpu = None
-    if rank == 0 and world == 1 and not args.skip_cpu:
-        x = oracle_inputs(16)
-        dt = oracle_pass(x)
-        cpu = {"value": x["tokens"] / dt, "unit": UNIT, "cores": 1, "kind": "oracle", "sample": x["desc"], "seconds": dt}
+    del K, V, src, dst, ws
+    torch.cuda.empty_cache()
+    if rank == 0 and not args.skip_decode_cfg4:
+        extra["decode_cfg4"] = bench_decode_cfg4(b, synth, dev, peak)
+        extra["decode_cfg4_paged"] = bench_decode_paged(b, synth, dev, peak)
+        d4 = extra["decode_cfg4"]
+        targets["cfg4_decode_batch32"] = {"compressed_us_per_layer_step": d4["compressed"]["us_per_layer_step"],
+                                          "compressed_frac_of_peak": d4["compressed"]["frac_of_peak"],
+                                          "uncompressed_us_per_layer_step": d4["uncompressed"]["us_per_layer_step"],
+                                          "speedup_vs_uncompressed": d4["speedup"], "steps": d4["compressed"]["steps"],
+                                          "paged_frac_of_peak": extra["decode_cfg4_paged"]["frac_of_peak"]}
+    if rank == 0 and not args.skip_serving and args.layers == 0:
+        extra["serving_mix"] = bench_serving_mix(b, synth, dev, peak, steps=args.serving_steps)
+        sm = extra["serving_mix"]
+        targets["cfg5_serving_mix"] = {k: sm[k] for k in ("steps", "ms_per_step", "ms_attention_per_step", "attention_frac_of_peak",
+                                                           "decode_tok_s", "attention_speedup", "prefill_compress_ms_total")}
+    roofline["targets"] = targets   # the other workloads' numbers, each against the same measured peak
 
     if rank == 0:
         line = {"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": max(args.warmup, 3),
                 "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "bf16",
-                "data": "synthetic",
-                "config": {"workload": WORKLOAD if args.layers == 0 else f"{WORKLOAD} cut to {L} layers (not the benchmark workload)", "layers": L, "kv_heads": H, "q_heads": H * G, "head_dim": D, "seq": s,
-                           "chunk": c, "retain": out_len / s, "step": "compress_prefill + append 64 + decode all layers",
-                           "l2": "inputs (4 GiB) exceed L2"},
-                "clocks": clocks, "e2e": e2e, "gpu_launches": launches_per_step * args.steps, "roofline": roofline,
-                "cpu_baseline": cpu, "detail": extra}
+                "data": "synthetic", "config": workload_config(L),
+                "clocks": clocks, "e2e": e2e, "gpu_launches": launches_per_step * args.steps,
+                "cpu_baseline": cpu, "detail": extra, "roofline": roofline}
         print(json.dumps(line))
     parallel.finish()
 
@@ -404,8 +506,10 @@ def bench_e2e(b, torch, dev, K, V, kn, vn, q, p, dst, ws, wsd, views, final_len,
 
 def bench_compress_variants(b, synth, dev, K, V, peak_gbs, with_128k):
     """ckv_compress_prefill alone on the same keys and values with other chunk sizes, ratios and ranking scopes (outside
-    the timed region).  `gbs` counts what the method has to move if every round read its input once and wrote its
-    output once; a round that ranks across chunks reads K twice, which is not credited."""
+    the timed region).  `gbs` and `frac_of_peak` charge every schedule, whatever its number of rounds, what the method
+    itself has to move: one read of the source and one write of the final cache.  `moved_gb` is what this
+    implementation moves by construction (every round that is not fused with the next reads its input and writes its
+    output; a round that ranks across chunks reads K once more), and `frac_on_moved_bytes` the rate on those."""
     import torch
     L, H, s, D = K.shape
     P = b.Params
@@ -440,16 +544,29 @@ def bench_compress_variants(b, synth, dev, K, V, peak_gbs, with_128k):
         t1.record()
         torch.cuda.synchronize()
         ms = t0.elapsed_time(t1) / iters
-        # every round reads its input once and writes its output once
         lens, cur = [n], n
         for j in range(rounds):
             pj = P(chunk=p.chunk, n_sink=p.n_sink, n_recent=p.n_recent, n_rounds_max=j + 1, r_init=p.r_init, r_decay=p.r_decay,
                    r_min=p.r_min, select=p.select, budget=p.budget)
             cur = b.compress_plan(n, pj)[0]
             lens.append(cur)
-        nbytes = sum(L * H * (lens[j] * (2 * D * 2 + 4) + lens[j + 1] * (2 * D * 2 + 8)) for j in range(rounds))
+        nbytes = schedule_bytes(L, H, n, out_len, D, 2)
+        # what the launches move: per round input + output; two leading ratio-1 rounds at chunk 64 run as one pass; a
+        # round ranked per head (neither 0 nor all of its edges merge) reads the keys twice
+        moved, j = 0, 0
+        while j < rounds:
+            full = lambda a_, b_: a_ - b_ == (a_ - p.n_sink - p.n_recent) // p.chunk * (p.chunk // 2) + ((a_ - p.n_sink - p.n_recent) % p.chunk + 1) // 2
+            fused = (p.chunk == 64 and j == 0 and rounds >= 2 and full(lens[0], lens[1]) and full(lens[1], lens[2]))
+            if fused:
+                moved += L * H * (lens[0] * 2 * D * 2 + lens[2] * (2 * D * 2 + 8))
+                j += 2
+                continue
+            ranked = p.select == b.SELECT_GLOBAL and not full(lens[j], lens[j + 1]) and lens[j] != lens[j + 1]
+            moved += L * H * (lens[j] * (2 * D * 2 + (4 if j else 0)) + lens[j + 1] * (2 * D * 2 + 8) + (lens[j] * D * 2 if ranked else 0))
+            j += 1
         res[name] = {"seq": n, "out_len": out_len, "rounds": rounds, "ms": ms, "tokens_per_s": n / (ms * 1e-3),
                      "gbs": nbytes / (ms * 1e-3) / 1e9, "frac_of_peak": nbytes / (ms * 1e-3) / 1e9 / peak_gbs,
+                     "moved_gb": moved / 1e9, "frac_on_moved_bytes": moved / (ms * 1e-3) / 1e9 / peak_gbs,
                      "status": b.workspace_status(ws)}
         del dst, ws
 
@@ -467,78 +584,110 @@ def bench_compress_variants(b, synth, dev, K, V, peak_gbs, with_128k):
     return res
 
 
-def bench_serving_mix(b, synth, dev, peak_gbs, steps=128):
-    """Workload serving_mix: batch 64, context lengths uniform on [4096, 65536], 32 layers x 8 KV heads, caches already
-    compressed to 25 % (their content does not matter for timing: random values, degrees 4).  Lock-step decoding: every
-    step appends one token to every sequence (ckv_compress_append, which clusters each completed chunk of 64 appended
-    tokens 64 -> 32 -> 16) and runs ckv_decode_attn for all 32 layers over the ragged batch.  The uncompressed comparison
-    keeps the full contexts of the same batch on 8 layers (32 would not fit) and is scaled to 32."""
+def bench_serving_mix(b, synth, dev, peak_gbs, steps=1024):
+    """Workload serving_mix at its stated size: batch 64, context lengths uniform on [4096, 65536], 32 layers x 8 KV
+    heads, bf16.  Every sequence is prefill-compressed to 25 % (two rounds at ratio 1) one at a time from a scratch
+    buffer that holds its uncompressed cache (the 64 uncompressed caches together would not fit) into its own slab.
+    Then `steps` lock-step decoding steps: ckv_compress_append_batch writes one new token per sequence (every completed
+    chunk of 64 appended tokens is clustered 64 -> 32 -> 16) and ckv_decode_attn runs for all 32 layers over the ragged
+    batch with a fresh query.  The uncompressed comparison keeps the full contexts of the same batch on 8 layers (32
+    would not fit) and is scaled to 32."""
     import torch
     cfg = synth.CONFIGS["serving_mix"]
     Bz, L, H, G, D, c = cfg["batch"], cfg["L"], cfg["H"], cfg["G"], cfg["d"], cfg["chunk"]
     ctx = synth.context_lengths(Bz, cfg["ctx"][0], cfg["ctx"][1], seed=cfg["seed"])
     p = b.Params(chunk=c, n_sink=0, n_recent=0, n_rounds_max=2, r_init=1.0, r_decay=0.0, r_min=1.0)
     scale = 1.0 / math.sqrt(D)
+    n_q = 8   # distinct query tensors cycled through the steps
+    qs = [synth.queries(Bz, H * G, D, seed=100 + i, dtype="bf16", device=dev) for i in range(n_q)]
+    out = torch.empty_like(qs[0])
+    g = torch.Generator(dev).manual_seed(23)
 
-    def run(layers, lens, compressed, n_steps):
-        g = torch.Generator(dev).manual_seed(23)
-        caches = []
-        for n in lens:
-            cap = n + n_steps + c
-            k = torch.empty((layers, H, cap, D), dtype=torch.bfloat16, device=dev).normal_(generator=g)
-            v = torch.empty((layers, H, cap, D), dtype=torch.bfloat16, device=dev).normal_(generator=g)
-            deg = torch.full((layers, H, cap), 4 if compressed else 1, dtype=torch.int32, device=dev)
-            caches.append(b.Cache(k, v, deg, torch.log(deg.float()) if compressed else None, n))
-        ws = torch.empty(b.workspace_bytes(caches[0], p), dtype=torch.uint8, device=dev)
-        wsd = torch.empty(b.decode_workspace_bytes(Bz, H, G, D, max(lens) + n_steps), dtype=torch.uint8, device=dev)
+    def decode_loop(caches, layers, n_steps, compressed, ws):
         kn = torch.empty((layers, H, Bz, D), dtype=torch.bfloat16, device=dev).normal_(generator=g)
         vn = torch.empty((layers, H, Bz, D), dtype=torch.bfloat16, device=dev).normal_(generator=g)
-        new = [(kn[:, :, i:i + 1].contiguous(), vn[:, :, i:i + 1].contiguous()) for i in range(Bz)]
-        q = synth.queries(Bz, H * G, D, seed=3, dtype="bf16", device=dev)
-        out = torch.empty_like(q)
+        wsd = torch.empty(b.decode_workspace_bytes(Bz, H, G, D, max(x.cap for x in caches)), dtype=torch.uint8, device=dev)
         att_ev = []
 
-        def one_step(record):
-            for i, cache in enumerate(caches):
-                if compressed:
-                    b.compress_append(cache, new[i][0], new[i][1], p, ws)
-                else:   # the uncompressed cache only grows: same copy, no trigger
-                    cache.k[:, :, cache.len] = new[i][0][:, :, 0]
-                    cache.v[:, :, cache.len] = new[i][1][:, :, 0]
+        def one_step(i, record):
+            if compressed:
+                b.compress_append_batch(caches, kn, vn, p, ws)
+            else:   # the uncompressed cache only grows
+                for j, cache in enumerate(caches):
+                    cache.k[:, :, cache.len] = kn[:, :, j]
+                    cache.v[:, :, cache.len] = vn[:, :, j]
                     cache.len += 1
             max_len = max(x.len for x in caches)
+            views = b.layer_views_all(caches, dev)
             e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
             e0.record()
             for l in range(layers):
-                b.decode_attn(b.layer_views(caches, l, dev), H, G, q, out, scale, max_len, wsd)
+                b.decode_attn(views[l], H, G, qs[i % n_q], out, scale, max_len, wsd)
             e1.record()
             if record:
-                att_ev.append((e0, e1))
+                att_ev.append((e0, e1, sum(x.len for x in caches)))
 
-        for _ in range(3):
-            one_step(False)
+        for i in range(3):
+            one_step(i, False)
         torch.cuda.synchronize()
         t0, t1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
         t0.record()
-        for _ in range(n_steps - 3):
-            one_step(True)
+        for i in range(3, n_steps):
+            one_step(i, True)
         t1.record()
         torch.cuda.synchronize()
         ms_step = t0.elapsed_time(t1) / (n_steps - 3)
-        ms_att = statistics.mean(x.elapsed_time(y) for x, y in att_ev)
-        rows = sum(x.len for x in caches) * H
-        del caches
-        torch.cuda.empty_cache()
+        ms_att = statistics.mean(x.elapsed_time(y) for x, y, _ in att_ev)
+        rows = statistics.mean(n for _, _, n in att_ev) * H
         return ms_step, ms_att, rows
 
-    comp_lens = [n // 4 for n in ctx]
-    ms_step, ms_att, rows = run(L, comp_lens, True, steps)
+    # ---- compressed: prefill-compress every sequence from the scratch buffer, then decode
+    top = max(ctx)
+    Ks = synth.ar1_keys(L, H, top, D, (0.7, 0.95), 0.5, seed=cfg["seed"], dtype="bf16", device=dev)   # every sequence reads a prefix
+    Vs = synth.normal_values(L, H, top, D, seed=cfg["seed"], dtype="bf16", device=dev)
+    growth = (steps // c + 1) * (c // 4) + c + 8
+    caches, ws = [], None
+    pre_ms, status = 0.0, 0
+    for n in ctx:
+        src = b.Cache(Ks, Vs, None, None, n)
+        out_len, _, cap = b.compress_plan(n, p)
+        dst = b.Cache.empty(L, H, max(cap, out_len + growth), D, torch.bfloat16, dev)
+        need = max(b.workspace_bytes(src, p), b.workspace_bytes(dst, p))
+        if ws is None or ws.numel() < need:
+            ws = None
+            ws = torch.empty(need, dtype=torch.uint8, device=dev)
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        b.compress_prefill(src, dst, p, ws)
+        e1.record()
+        status |= b.workspace_status(ws)
+        pre_ms += e0.elapsed_time(e1)
+        caches.append(dst)
+    del Ks, Vs
+    torch.cuda.empty_cache()
+    slots0 = sum(x.len for x in caches)
+    ms_step, ms_att, rows = decode_loop(caches, L, steps, True, ws)
+    status |= b.workspace_status(ws)
     nbytes = decode_bytes(rows, D, 2) * L
-    res = {"batch": Bz, "layers": L, "steps": steps - 3, "context_tokens_total": sum(ctx), "cached_slots_total": rows // H,
+    res = {"batch": Bz, "layers": L, "steps": steps - 3, "context_tokens_total": sum(ctx), "cached_slots_after_prefill": slots0,
+           "cached_slots_at_the_end": sum(x.len for x in caches), "prefill_compress_ms_total": pre_ms,
+           "prefill_compress_tokens_per_s": sum(ctx) / (pre_ms * 1e-3),
            "ms_per_step": ms_step, "ms_attention_per_step": ms_att, "decode_tok_s": Bz / (ms_step * 1e-3),
-           "attention_gbs": nbytes / (ms_att * 1e-3) / 1e9, "attention_frac_of_peak": nbytes / (ms_att * 1e-3) / 1e9 / peak_gbs}
-    Lu = 8
-    ms_step_u, ms_att_u, _ = run(Lu, ctx, False, 16)
+           "attention_gbs": nbytes / (ms_att * 1e-3) / 1e9, "attention_frac_of_peak": nbytes / (ms_att * 1e-3) / 1e9 / peak_gbs,
+           "status": status}
+    del caches, ws
+    torch.cuda.empty_cache()
+
+    # ---- uncompressed comparison on 8 layers
+    Lu, su = 8, 16
+    caches = []
+    for n in ctx:
+        k = torch.empty((Lu, H, n + su + 1, D), dtype=torch.bfloat16, device=dev).normal_(generator=g)
+        v = torch.empty((Lu, H, n + su + 1, D), dtype=torch.bfloat16, device=dev).normal_(generator=g)
+        caches.append(b.Cache(k, v, None, None, n))
+    _, ms_att_u, _ = decode_loop(caches, Lu, su, False, None)
+    del caches
+    torch.cuda.empty_cache()
     res["uncompressed"] = {"layers_run": Lu, "ms_attention_per_step_32_layers": ms_att_u * L / Lu,
                            "decode_tok_s_attention_only": Bz / (ms_att_u * L / Lu * 1e-3)}
     res["attention_speedup"] = res["uncompressed"]["ms_attention_per_step_32_layers"] / ms_att
@@ -657,45 +806,57 @@ def bench_decode_paged(b, synth, dev, peak_gbs):
             "frac_of_peak": nbytes / (us * 1e-6) / 1e9 / peak_gbs}
 
 
-def bench_decode_cfg4(b, synth, dev, peak_gbs):
-    """Decode attention on the batch-32 shape: 8192 centroids (+256 appended) vs the uncompressed 32768-token cache."""
+def bench_decode_cfg4(b, synth, dev, peak_gbs, steps=256):
+    """Workload decode_b32 as stated: batch 32, 8 KV heads x 4 query heads, 8192 centroids whose degrees sum to 32768;
+    256 decode steps, each with a fresh query ~ N(0, 1) and one appended degree-1 token per sequence (8192 -> 8448
+    slots), one layer.  Compared with the same kernel on the uncompressed 32768-token cache (which grows the same way).
+    The time is that of ckv_decode_attn alone (events around each call); the appends run between the calls."""
     import torch
     cfg = synth.CONFIGS["decode_b32"]
     Bz, H, G, D = cfg["batch"], cfg["H"], cfg["G"], cfg["d"]
+    scale = 1.0 / math.sqrt(D)
+    qs = synth.queries(steps * Bz, H * G, D, seed=3, dtype="bf16", device=dev).view(steps, Bz, H * G, D)
+    gk = torch.Generator(dev).manual_seed(41)
+    kn = torch.empty((steps, 1, H, Bz, D), dtype=torch.bfloat16, device=dev).normal_(generator=gk)
+    vn = torch.empty((steps, 1, H, Bz, D), dtype=torch.bfloat16, device=dev).normal_(generator=gk)
+    no_trigger = b.Params(chunk=64, n_sink=0, n_recent=0, n_rounds_max=0, r_init=1.0, r_decay=0.0, r_min=1.0)  # appended tokens stay as they are
     res = {}
     for name, slots, with_deg in (("compressed", cfg["slots"], True), ("uncompressed", cfg["s"], False)):
-        cap = slots + 256
+        cap = slots + steps
         caches = []
         for i in range(Bz):
             k = torch.randn((1, H, cap, D), device=dev, dtype=torch.float32).to(torch.bfloat16)
             v = torch.randn((1, H, cap, D), device=dev, dtype=torch.float32).to(torch.bfloat16)
-            deg = logdeg = None
+            deg = torch.ones((1, H, cap), dtype=torch.int32)
             if with_deg:
-                deg = torch.ones((1, H, cap), dtype=torch.int32)
                 deg[:, :, :slots] = synth.random_degrees((1, H), slots, cfg["s"], seed=i)
-                deg = deg.to(dev)
-                logdeg = torch.log(deg.float())
-            caches.append(b.Cache(k, v, deg, logdeg, slots))
-        q = synth.queries(Bz, H * G, D, seed=3, dtype="bf16", device=dev)
-        out = torch.empty_like(q)
+            deg = deg.to(dev)
+            caches.append(b.Cache(k, v, deg, torch.log(deg.float()) if with_deg else None, slots))
+        out = torch.empty_like(qs[0])
         ws = torch.empty(b.decode_workspace_bytes(Bz, H, G, D, cap), dtype=torch.uint8, device=dev)
-        views = b.layer_views(caches, 0, dev)
-        scale = 1.0 / math.sqrt(D)
-        for _ in range(5):
-            b.decode_attn(views, H, G, q, out, scale, slots, ws)
+        wsa = torch.empty(b.workspace_bytes(caches[0], no_trigger), dtype=torch.uint8, device=dev)
+        for i in range(5):   # warm-up on the initial length
+            b.decode_attn(b.layer_views(caches, 0, dev), H, G, qs[i], out, scale, slots, ws)
         torch.cuda.synchronize()
-        iters = 50
-        t0, t1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-        t0.record()
-        for _ in range(iters):
-            b.decode_attn(views, H, G, q, out, scale, slots, ws)
-        t1.record()
+        evs, rows = [], 0
+        for i in range(steps):
+            b.compress_append_batch(caches, kn[i], vn[i], no_trigger, wsa)
+            n = caches[0].len
+            views = b.layer_views(caches, 0, dev)
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            e0.record()
+            b.decode_attn(views, H, G, qs[i], out, scale, n, ws)
+            e1.record()
+            evs.append((e0, e1))
+            rows += Bz * H * n
         torch.cuda.synchronize()
-        us = 1e3 * t0.elapsed_time(t1) / iters
-        nbytes = decode_bytes(Bz * H * slots, D, 2) if with_deg else Bz * H * slots * 2 * D * 2
-        res[name] = {"slots": slots, "us_per_layer_step": us, "gbs": nbytes / (us * 1e-6) / 1e9,
+        assert caches[0].len == slots + steps
+        us = 1e3 * statistics.mean(x.elapsed_time(y) for x, y in evs)
+        nbytes = (decode_bytes(rows, D, 2) if with_deg else rows * 2 * D * 2) / steps
+        res[name] = {"slots": f"{slots} -> {slots + steps}", "steps": steps, "us_per_layer_step": us, "gbs": nbytes / (us * 1e-6) / 1e9,
                      "frac_of_peak": nbytes / (us * 1e-6) / 1e9 / peak_gbs, "decode_tok_s_per_layer": Bz / (us * 1e-6)}
         del caches
+        torch.cuda.empty_cache()
     res["speedup"] = res["uncompressed"]["us_per_layer_step"] / res["compressed"]["us_per_layer_step"]
     return res
 
@@ -712,6 +873,7 @@ def main():
     ap.add_argument("--skip-decode-cfg4", action="store_true")
     ap.add_argument("--skip-variants", action="store_true")
     ap.add_argument("--skip-serving", action="store_true")
+    ap.add_argument("--serving-steps", type=int, default=1024, help="lock-step decode steps of the serving-mix workload (its stated size: 1024)")
     args = ap.parse_args()
     if args.steps is None:
         args.steps = 3 if args.impl == "reference" else 200

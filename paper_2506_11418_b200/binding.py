@@ -250,6 +250,26 @@ def layer_views(caches, layer: int, device="cuda") -> torch.Tensor:
     return torch.tensor(rows, dtype=torch.int64).to(device)
 
 
+def layer_views_all(caches, device="cuda") -> torch.Tensor:
+    """[L, Bz, 5] int64: the ckv_layer_view arrays of every layer of a batch of caches, built and copied to the device
+    in one go (views[l] is the argument of ckv_decode_attn for layer l)."""
+    L = caches[0].k.shape[0]
+    base = []
+    for c in caches:
+        _, H, cap, D = c.k.shape
+        base.append([c.k.data_ptr(), c.v.data_ptr(), c.logdeg.data_ptr() if c.logdeg is not None else 0, c.len, cap,
+                     H * cap * D * c.k.element_size(), H * cap * 4])
+    t = torch.tensor(base, dtype=torch.int64)                       # [Bz, 7]
+    lay = torch.arange(L, dtype=torch.int64).view(L, 1)
+    out = torch.empty((L, len(caches), 5), dtype=torch.int64)
+    out[:, :, 0] = t[:, 0] + lay * t[:, 5]
+    out[:, :, 1] = t[:, 1] + lay * t[:, 5]
+    out[:, :, 2] = torch.where(t[:, 2] != 0, t[:, 2] + lay * t[:, 6], torch.zeros_like(t[:, 2]))
+    out[:, :, 3] = t[:, 3]
+    out[:, :, 4] = t[:, 4]
+    return out.to(device)
+
+
 def decode_workspace_bytes(Bz, H, G, D, max_len) -> int:
     return lib.ckv_decode_workspace_bytes(Bz, H, G, D, max_len)
 
