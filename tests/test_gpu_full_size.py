@@ -250,6 +250,94 @@ def test_config5_serving_mix_reduced_layers():
     torch.cuda.empty_cache()
 
 
+def test_config5_serving_mix_at_its_stated_size():
+    """The serving mix as stated: batch 64, context lengths uniform on [4096, 65536], 32 layers x 8 KV heads, bf16.
+    Every sequence is prefill-compressed to 25 % one at a time from a scratch buffer (the uncompressed caches together
+    would not fit), then 1024 lock-step steps: one appended token per sequence (ckv_compress_append_batch; every
+    completed chunk of 64 appended tokens is clustered 64 -> 32 -> 16: sixteen triggers per sequence) and decode
+    attention over the ragged batch on all 32 layers.  The oracle replays two sampled sequences on one layer and two
+    KV heads: cache lengths and pending counts at every step; degrees, stored rows and attention outputs at sampled
+    steps, among them the steps around a trigger; degree sums over everything at the end."""
+    need_free(110)
+    b = B()
+    cfg = synth.CONFIGS["serving_mix"]
+    Bz, L, H, G, D, c = cfg["batch"], cfg["L"], cfg["H"], cfg["G"], cfg["d"], cfg["chunk"]
+    steps = 1024
+    ctx = synth.context_lengths(Bz, cfg["ctx"][0], cfg["ctx"][1], seed=cfg["seed"])
+    p = b.Params(chunk=c, n_sink=0, n_recent=0, n_rounds_max=2, r_init=1.0, r_decay=0.0, r_min=1.0)
+    po = PU.oracle_params(p)
+    scale = 1.0 / math.sqrt(D)
+    ol, oh = 17, [2, 5]                        # the layer and KV heads the oracle follows
+    sampled = {3: None, 41: None}              # and the sequences
+    growth = (steps // c + 1) * (c // 4) + c + 8
+    caches, ws = [], None
+    for i, n0 in enumerate(ctx):
+        K = synth.ar1_keys(L, H, n0, D, (0.7, 0.95), 0.5, seed=100 + i, dtype="bf16", device=DEV)
+        V = synth.normal_values(L, H, n0, D, seed=100 + i, dtype="bf16", device=DEV)
+        src = b.Cache(K, V, None, None, n0)
+        out_len, rounds, cap = b.compress_plan(n0, p)
+        dst = b.Cache.empty(L, H, max(cap, out_len + growth), D, K.dtype, DEV)
+        need = max(b.workspace_bytes(src, p), b.workspace_bytes(dst, p))
+        if ws is None or ws.numel() < need:
+            ws = None
+            torch.cuda.empty_cache()
+            ws = torch.empty(need, dtype=torch.uint8, device=DEV)
+        b.compress_prefill(src, dst, p, ws)
+        assert b.workspace_status(ws) == 0 and rounds == 2 and dst.len == out_len
+        assert torch.equal(dst.deg[:, :, :out_len].sum(dim=2, dtype=torch.int64), torch.full((L, H), n0, dtype=torch.int64, device=DEV))
+        caches.append(dst)
+        if i in sampled:
+            Ko, Vo, do, _, _ = O.compress_prefill(PU.to_np64(K[ol:ol + 1, oh]), PU.to_np64(V[ol:ol + 1, oh]), None, po, storage="bf16")
+            sampled[i] = [Ko, Vo, do, 0]
+        del K, V, src
+    torch.cuda.empty_cache()
+    wsd = torch.empty(b.decode_workspace_bytes(Bz, H, G, D, max(x.cap for x in caches)), dtype=torch.uint8, device=DEV)
+    results, worst, triggers = [], 0.0, 0
+    out = torch.empty((Bz, H * G, D), dtype=torch.bfloat16, device=DEV)   # the other layers' outputs
+    out_l = torch.empty_like(out)                                          # the followed layer's
+    for step in range(steps):
+        kn = synth.ar1_keys(L, H, Bz, D, (0.7, 0.95), 0.5, seed=5000 + step, dtype="bf16", device=DEV)   # token b of every (layer, head)
+        vn = synth.normal_values(L, H, Bz, D, seed=5000 + step, dtype="bf16", device=DEV)
+        q = synth.queries(Bz, H * G, D, seed=7000 + step, dtype="bf16", device=DEV)
+        before = caches[0].len
+        b.compress_append_batch(caches, kn, vn, p, ws)
+        triggers += caches[0].len < before
+        max_len = max(x.len for x in caches)
+        views = b.layer_views_all(caches, DEV)
+        check = step % 97 == 0 or step % 64 in (62, 63, 0) and step % 256 < 70 or step == steps - 1
+        for l in range(L):
+            b.decode_attn(views[l], H, G, q, out_l if l == ol else out, scale, max_len, wsd)
+        for i, st in sampled.items():
+            st[0], st[1], st[2], st[3] = O.compress_append(st[0], st[1], st[2], st[3], PU.to_np64(kn[ol:ol + 1, oh, i:i + 1]),
+                                                           PU.to_np64(vn[ol:ol + 1, oh, i:i + 1]), po, storage="bf16")
+            assert caches[i].len == st[0].shape[2] and caches[i].pending == st[3]
+            if check:
+                torch.cuda.synchronize()
+                n = caches[i].len
+                np.testing.assert_array_equal(caches[i].deg[ol, oh, :n].cpu().numpy(), st[2][0])
+                qs = PU.to_np64(q[i]).reshape(H, G, D)[oh].reshape(len(oh) * G, D)
+                got = PU.to_np64(out_l[i]).reshape(H, G, D)[oh].reshape(len(oh) * G, D)
+                worst = max(worst, float(np.abs(got - O.app_attn(qs, st[0][0], st[1][0], st[2][0], scale)).max()))
+                results.append(PU.check_attention(got, qs, PU.to_np64(caches[i].k[ol, oh, :n]), PU.to_np64(caches[i].v[ol, oh, :n]),
+                                                  st[2][0], scale, "bf16", f"step {step}, sequence {i}"))
+    assert b.workspace_status(ws) == 0
+    assert triggers == steps // c                       # sixteen windows per sequence
+    assert worst <= 2e-2, f"decode attention over the serving mix: max abs error {worst:.3e}"
+    PU.summarize_attention(results, f"serving mix at full size, {len(results)} sampled outputs")
+    for i, cache in enumerate(caches):   # every sequence: degrees account for every token ever written
+        n = cache.len
+        assert torch.equal(cache.deg[:, :, :n].sum(dim=2, dtype=torch.int64),
+                           torch.full((L, H), ctx[i] + steps, dtype=torch.int64, device=DEV))
+        torch.testing.assert_close(cache.logdeg[:, :, :n], torch.log(cache.deg[:, :, :n].float()), rtol=1e-6, atol=1e-7)
+    for i, st in sampled.items():        # the cache itself: two ulp for the two rounds of storage rounding
+        n = caches[i].len
+        for t, ref in ((caches[i].k, st[0]), (caches[i].v, st[1])):
+            got = PU.to_np64(t[ol, oh, :n])
+            assert np.all(np.abs(got - ref[0]) <= 2 * PU.bf16_ulp(ref[0]) * 1.0001 + 1e-30)
+    del caches
+    torch.cuda.empty_cache()
+
+
 def test_no_chunking_16k_four_layers():
     """chunk = 0 (plain Bipartite Soft Matching) in the launch the benchmark's no-chunk section times: the first 16384
     tokens of 4 layers x 8 KV heads, every edge merged.  Invariants over everything, two slabs against the oracle."""
