@@ -195,6 +195,42 @@ int ckv_pages_scatter(const int32_t* block_table, int64_t len, const void* k, co
                       int32_t page_tokens, int32_t H, int32_t D, int32_t dtype, void* k_pages, void* v_pages, int32_t* deg_pages,
                       float* logdeg_pages, void* cuda_stream);
 
+/* ---- Clustering a paged cache directly (the paper's Appendix on its vLLM integration: read pages -> compress -> write
+ * back -> free blocks).  A sequence's cache lives in pages of per-layer pools that all layers index with one block
+ * table.  A round cannot run in place (thread blocks would overwrite rows that others still read), so the rounds
+ * alternate between the sequence's own pages and scratch pages of the same pools: round 0 reads through block_table and
+ * writes through scratch_table, round 1 the other way round (from position 0 of the sequence's own pages), and so on.
+ * With an odd number of rounds the result therefore sits in the first pages of scratch_table, otherwise in the first
+ * pages of block_table; ckv_pages_plan tells which, and how many pages the sequence keeps: the caller swaps the
+ * tables if need be and returns every other page to its free list.  The contents of all pages of both tables are
+ * overwritten.  This version: bf16, D = 128, chunk 64, page_tokens a power of two >= 64, up to 64 layers per call
+ * (CKV_ERR_UNSUPPORTED otherwise: ckv_pages_gather -> ckv_compress_prefill -> ckv_pages_scatter serves the rest). */
+typedef struct ckv_page_pool { /* one layer's pool */
+  void* k_pages;       /* [n_pages, H, page_tokens, D] */
+  void* v_pages;       /* [n_pages, H, page_tokens, D] */
+  int32_t* deg_pages;  /* [n_pages, H, page_tokens], required */
+  float* logdeg_pages; /* [n_pages, H, page_tokens] or NULL */
+} ckv_page_pool;
+
+/* Host-only: Algorithm 1's loop for a paged sequence of `len` tokens: final length, rounds, the scratch pages the call
+ * needs, whether the result ends up in the scratch pages (1) or in the sequence's own (0), and the number of pages the
+ * sequence keeps afterwards: ceil(out_len / page_tokens).  Any output pointer may be NULL. */
+int ckv_pages_plan(int64_t len, const ckv_params* params, int32_t page_tokens, int64_t* out_len, int64_t* rounds,
+                   int64_t* scratch_pages, int32_t* result_in_scratch, int64_t* pages_kept);
+
+/* Host-only: workspace bytes of ckv_compress_paged (per-edge arrays of rounds ranked per head, staging of each round's
+ * shorter last chunk); 0 for invalid arguments. */
+size_t ckv_paged_workspace_bytes(int32_t L, int32_t H, int32_t D, int32_t dtype, int64_t len, const ckv_params* params);
+
+/* Algorithm 1, pre-filling branch, on a paged sequence (Sec. 5.2, Sec. 5.3, Eq. 4, Eq. 5 as ckv_compress_prefill).
+ * pools: HOST array [L]; block_table, scratch_table: device; has_deg: 0 = the source pages carry no degrees (all
+ * ones).  *out_len, *result_in_scratch (host, optional) as ckv_pages_plan reports them.  CKV_ERR_CAPACITY if
+ * scratch_pages is less than the plan needs. */
+int ckv_compress_paged(const ckv_page_pool* pools, int32_t L, int32_t H, int32_t D, int32_t dtype, int32_t page_tokens,
+                       const int32_t* block_table, int64_t len, int32_t has_deg, const int32_t* scratch_table,
+                       int64_t scratch_pages, const ckv_params* params, void* workspace, size_t workspace_bytes,
+                       void* cuda_stream, int64_t* out_len, int32_t* result_in_scratch);
+
 /* ckv_decode_attn for callers that cannot hand over a workspace because they cannot allocate device
  * memory at the point of the call: code running inside a serving engine's steady-state loop whose memory
  * pool is frozen after start-up, a plug-in that is given only its input and output tensors, or a host

@@ -21,7 +21,11 @@ OK = 0
 EXPORTS = ["ckv_compress_plan", "ckv_workspace_bytes", "ckv_compress_prefill", "ckv_compress_append", "ckv_compress_append_batch",
            "ckv_decode_workspace_bytes", "ckv_decode_attn", "ckv_status_string", "ckv_workspace_status",
            "ckv_decode_attn_static", "ckv_compress_append_recluster", "ckv_decode_attn_paged", "ckv_pages_gather",
-           "ckv_pages_scatter"]
+           "ckv_pages_scatter", "ckv_pages_plan", "ckv_paged_workspace_bytes", "ckv_compress_paged"]
+
+
+class CkvPagePool(C.Structure):
+    _fields_ = [("k_pages", C.c_void_p), ("v_pages", C.c_void_p), ("deg_pages", C.c_void_p), ("logdeg_pages", C.c_void_p)]
 
 
 class CkvCache(C.Structure):
@@ -75,6 +79,15 @@ def _load():
     lib.ckv_pages_scatter.restype = C.c_int
     lib.ckv_pages_scatter.argtypes = [C.c_void_p, C.c_int64, C.c_void_p, C.c_void_p, C.c_void_p, C.c_int64, C.c_int32, C.c_int32,
                                       C.c_int32, C.c_int32, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p]
+    lib.ckv_pages_plan.restype = C.c_int
+    lib.ckv_pages_plan.argtypes = [C.c_int64, C.POINTER(CkvParams), C.c_int32, C.POINTER(C.c_int64), C.POINTER(C.c_int64),
+                                   C.POINTER(C.c_int64), C.POINTER(C.c_int32), C.POINTER(C.c_int64)]
+    lib.ckv_paged_workspace_bytes.restype = C.c_size_t
+    lib.ckv_paged_workspace_bytes.argtypes = [C.c_int32, C.c_int32, C.c_int32, C.c_int32, C.c_int64, C.POINTER(CkvParams)]
+    lib.ckv_compress_paged.restype = C.c_int
+    lib.ckv_compress_paged.argtypes = [C.POINTER(CkvPagePool), C.c_int32, C.c_int32, C.c_int32, C.c_int32, C.c_int32, C.c_void_p,
+                                       C.c_int64, C.c_int32, C.c_void_p, C.c_int64, C.POINTER(CkvParams), C.c_void_p, C.c_size_t,
+                                       C.c_void_p, C.POINTER(C.c_int64), C.POINTER(C.c_int32)]
     lib.ckv_workspace_status.restype = C.c_int
     lib.ckv_workspace_status.argtypes = [C.c_void_p, C.c_void_p, C.POINTER(C.c_int32)]
     lib.ckv_decode_workspace_bytes.restype = C.c_size_t
@@ -248,6 +261,35 @@ def layer_views(caches, layer: int, device="cuda") -> torch.Tensor:
         rows.append([c.k.data_ptr() + off * D * es, c.v.data_ptr() + off * D * es,
                      (c.logdeg.data_ptr() + off * 4) if c.logdeg is not None else 0, c.len, cap])
     return torch.tensor(rows, dtype=torch.int64).to(device)
+
+
+def pages_plan(length: int, params: Params, page_tokens: int):
+    """ckv_pages_plan: (final length, rounds, scratch pages needed, result in scratch?, pages kept).  Host only."""
+    out_len, rounds, scratch, kept, in_scratch = C.c_int64(), C.c_int64(), C.c_int64(), C.c_int64(), C.c_int32()
+    _check(lib.ckv_pages_plan(length, C.byref(params.c()), page_tokens, C.byref(out_len), C.byref(rounds), C.byref(scratch),
+                              C.byref(in_scratch), C.byref(kept)))
+    return out_len.value, rounds.value, scratch.value, bool(in_scratch.value), kept.value
+
+
+def paged_workspace_bytes(L: int, H: int, D: int, dtype: torch.dtype, length: int, params: Params) -> int:
+    return lib.ckv_paged_workspace_bytes(L, H, D, dtype_code(dtype), length, C.byref(params.c()))
+
+
+def compress_paged(pools, block_table: torch.Tensor, length: int, has_deg: bool, scratch_table: torch.Tensor, params: Params,
+                   workspace: torch.Tensor):
+    """ckv_compress_paged on the current stream.  pools: one (k_pages, v_pages, deg_pages, logdeg_pages or None) per layer,
+    k_pages [n_pages, H, page_tokens, D].  Returns (final length, result in the scratch table's pages?)."""
+    kp = pools[0][0]
+    n_pages, H, P, D = kp.shape
+    arr = (CkvPagePool * len(pools))(*[CkvPagePool(k.data_ptr(), v.data_ptr(), d.data_ptr(), lg.data_ptr() if lg is not None else None)
+                                       for k, v, d, lg in pools])
+    out_len, in_scratch = C.c_int64(), C.c_int32()
+    _check(lib.ckv_compress_paged(arr, len(pools), H, D, dtype_code(kp.dtype), P, block_table.data_ptr(), length, int(has_deg),
+                                  scratch_table.data_ptr() if scratch_table is not None else None,
+                                  scratch_table.numel() if scratch_table is not None else 0, C.byref(params.c()),
+                                  workspace.data_ptr(), workspace.numel() * workspace.element_size(), _stream_ptr(),
+                                  C.byref(out_len), C.byref(in_scratch)))
+    return out_len.value, bool(in_scratch.value)
 
 
 def layer_views_all(caches, device="cuda") -> torch.Tensor:

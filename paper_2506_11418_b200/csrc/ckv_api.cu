@@ -352,12 +352,215 @@ ckv_params window_params(const ckv_params& p) {
   return wp;
 }
 
+// ---- clustering a paged cache in place of a slab (bf16, chunk 64) ---------------------------------------------------
+// The full chunks go through the warp-per-chunk kernel, which fetches a chunk's rows from its page (two pieces when the
+// chunk straddles a page boundary) and writes the surviving rows into the destination pages.  The shorter last chunk of
+// a round is staged: its rows are copied to a small slab, the tile kernel clusters it slab to slab, and the result is
+// copied into the destination pages.  Sinks and recent tokens are row copies from pages to pages.
+
+struct PagedWorkspace {
+  size_t edge_sim, edge_b, sel, chunk_off;
+  int64_t edge_stride, max_chunks;
+  size_t a_k, a_v, a_deg, b_k, b_v, b_deg, b_logdeg;  // staging slabs [LH, 64, ...] of the last chunk
+  size_t total;
+};
+
+PagedWorkspace layout_paged_workspace(int64_t LH, int D, int es, int chunk, const std::vector<RoundPlan>& plan) {
+  PagedWorkspace w{};
+  for (const RoundPlan& rp : plan)
+    if (rp.mode == kModeExternal) w.max_chunks = std::max<int64_t>(w.max_chunks, rp.n_chunks);
+  size_t off = 256;
+  auto take = [&off](size_t bytes) {
+    const size_t at = off;
+    off += align_up(bytes);
+    return at;
+  };
+  w.edge_stride = w.max_chunks * (chunk / 2);
+  w.edge_sim = take((size_t)LH * w.edge_stride * 4);
+  w.edge_b = take((size_t)LH * w.edge_stride * 4);
+  w.sel = take((size_t)LH * w.edge_stride);
+  w.chunk_off = take((size_t)LH * std::max<int64_t>(w.max_chunks, 1) * 4);
+  const size_t kv = (size_t)LH * chunk * D * es, dg = (size_t)LH * chunk * 4;
+  w.a_k = take(kv); w.a_v = take(kv); w.a_deg = take(dg);
+  w.b_k = take(kv); w.b_v = take(kv); w.b_deg = take(dg); w.b_logdeg = take(dg);
+  w.total = off;
+  return w;
+}
+
+cudaError_t run_round_paged(const RoundPlan& rp, PagedArgs pg, bool src_has_deg, int LH, int D, int chunk, const PagedWorkspace& w,
+                            unsigned char* ws, cudaStream_t st) {
+  cudaError_t e;
+  const int es = 2, row_bytes = D * es;
+  pg.dst_last_page = std::max<int64_t>(rp.s_out - 1, 0) >> pg.shift;
+  RowsCopyArgs c{};
+  c.src.table = pg.src_table; c.dst.table = pg.dst_table;
+  c.LH = LH; c.row_bytes = row_bytes; c.src_has_deg = src_has_deg;
+  if (rp.mode < 0) {  // nothing merges: the round is the identity
+    c.src_off = 0; c.dst_off = 0; c.count = rp.s_in;
+    return launch_rows_copy(c, pg, st);
+  }
+  c.src_off = 0; c.dst_off = 0; c.count = rp.lo;
+  if ((e = launch_rows_copy(c, pg, st)) != cudaSuccess) return e;
+  c.src_off = rp.hi; c.dst_off = rp.hi - rp.M; c.count = rp.s_in - rp.hi;
+  if ((e = launch_rows_copy(c, pg, st)) != cudaSuccess) return e;
+
+  const int64_t n_full = (rp.hi - rp.lo) / chunk;
+  const bool has_tail = rp.n_chunks > n_full;
+  const int64_t p_tail = rp.lo + n_full * chunk, tail = rp.hi - p_tail;
+  const int64_t q_end = rp.hi - rp.M;  // where the middle region's output ends
+  RoundArgs a{};
+  a.deg_src = src_has_deg ? reinterpret_cast<const int32_t*>(ws) : nullptr;  // only says: the pages carry degrees
+  a.lo = rp.lo; a.hi = rp.hi;
+  a.chunk = chunk; a.n_chunks = rp.n_chunks;
+  a.m_full = rp.m_full; a.m_tail = rp.m_tail;
+  a.out_stride = chunk - rp.m_full;
+  a.out_lo = rp.lo;
+  a.LH = LH;
+  a.status = reinterpret_cast<int32_t*>(ws);
+  a.edge_stride = (int64_t)rp.n_chunks * (chunk / 2);
+  // the last chunk as a slab-to-slab round: base pointers shifted so that the chunk's positions in the sequence (source
+  // p_tail ..., output ... q_end) index rows 0 .. 63 of the staging slabs
+  RoundArgs t = a;
+  const int64_t vbase = q_end - chunk;
+  t.k_src = ws + w.a_k - p_tail * row_bytes; t.v_src = ws + w.a_v - p_tail * row_bytes;
+  t.deg_src = src_has_deg ? reinterpret_cast<const int32_t*>(ws + w.a_deg) - p_tail : nullptr;
+  t.k_dst = ws + w.b_k - vbase * row_bytes; t.v_dst = ws + w.b_v - vbase * row_bytes;
+  t.deg_dst = reinterpret_cast<int32_t*>(ws + w.b_deg) - vbase;
+  t.logdeg_dst = reinterpret_cast<float*>(ws + w.b_logdeg) - vbase;
+  t.src_cap = chunk; t.dst_cap = chunk;
+  t.chunk_first = (int32_t)n_full; t.n_launch = 1;
+  if (has_tail) {
+    RowsCopyArgs in{};
+    in.src.table = pg.src_table;
+    in.dst.k = ws + w.a_k; in.dst.v = ws + w.a_v; in.dst.deg = reinterpret_cast<int32_t*>(ws + w.a_deg); in.dst.cap = chunk;
+    in.src_off = p_tail; in.dst_off = 0; in.count = tail;
+    in.LH = LH; in.row_bytes = row_bytes; in.src_has_deg = src_has_deg;
+    if ((e = launch_rows_copy(in, pg, st)) != cudaSuccess) return e;
+  }
+  auto launch_pass = [&](int mode) -> cudaError_t {
+    RoundArgs x = a;
+    x.mode = mode;
+    cudaError_t err = launch_round_fast_paged(x, pg, n_full, st);
+    if (err != cudaSuccess || !has_tail) return err;
+    RoundArgs y = t;
+    y.mode = mode;
+    y.edge_sim = x.edge_sim; y.edge_b = x.edge_b; y.sel = x.sel; y.chunk_out_off = x.chunk_out_off;
+    return launch_round_tile(y, st);
+  };
+  if (rp.mode == kModeExternal) {
+    a.edge_sim = reinterpret_cast<float*>(ws + w.edge_sim);
+    a.edge_b = reinterpret_cast<int32_t*>(ws + w.edge_b);
+    a.sel = ws + w.sel;
+    a.chunk_out_off = reinterpret_cast<int32_t*>(ws + w.chunk_off);
+    if ((e = launch_pass(kModeMatchOnly)) != cudaSuccess) return e;
+    SelectArgs sa{};
+    sa.edge_sim = a.edge_sim; sa.sel = a.sel; sa.chunk_out_off = a.chunk_out_off;
+    sa.edge_stride = a.edge_stride; sa.M = rp.M; sa.lo = rp.lo; sa.chunk = chunk; sa.n_chunks = rp.n_chunks; sa.LH = LH;
+    if ((e = launch_select(sa, st)) != cudaSuccess) return e;
+  }
+  if ((e = launch_pass(rp.mode)) != cudaSuccess) return e;
+  if (has_tail) {
+    RowsCopyArgs out{};
+    out.src.k = ws + w.b_k; out.src.v = ws + w.b_v; out.src.deg = reinterpret_cast<int32_t*>(ws + w.b_deg); out.src.cap = chunk;
+    out.dst.table = pg.dst_table;
+    out.LH = LH; out.row_bytes = row_bytes; out.src_has_deg = true;
+    out.dst_end = q_end;
+    if (rp.mode == kModeExternal) {  // where the last chunk's survivors start is only known on the device
+      out.begin = a.chunk_out_off; out.begin_stride = rp.n_chunks; out.begin_index = n_full;
+      out.src_off = 0; out.dst_off = vbase;
+    } else {
+      const int64_t q_tail = rp.lo + n_full * a.out_stride;
+      out.src_off = q_tail - vbase; out.dst_off = q_tail; out.count = q_end - q_tail;
+    }
+    if ((e = launch_rows_copy(out, pg, st)) != cudaSuccess) return e;
+  }
+  return cudaSuccess;
+}
+
+int paged_args_ok(const ckv_page_pool* pools, int32_t L, int32_t H, int32_t D, int32_t dtype, int32_t page_tokens,
+                  const ckv_params* params) {
+  int st;
+  if ((st = check_params(params)) != CKV_OK) return st;
+  if (!pools || L <= 0 || H <= 0) return CKV_ERR_INVALID_ARG;
+  if (dtype != CKV_F32 && dtype != CKV_BF16) return CKV_ERR_INVALID_ARG;
+  if (page_shift(page_tokens) < 0 || page_tokens < 64 || D != 128 || dtype != CKV_BF16 || params->chunk != 64 || L > kMaxPoolLayers ||
+      (int64_t)L * H > 65535)
+    return CKV_ERR_UNSUPPORTED;
+  return CKV_OK;
+}
+
 }  // namespace
 }  // namespace ckv
 
 using namespace ckv;
 
 extern "C" {
+
+int ckv_pages_plan(int64_t len, const ckv_params* params, int32_t page_tokens, int64_t* out_len, int64_t* rounds,
+                   int64_t* scratch_pages, int32_t* result_in_scratch, int64_t* pages_kept) {
+  int st = check_params(params);
+  if (st != CKV_OK) return st;
+  if (len < 0 || page_tokens <= 0) return CKV_ERR_INVALID_ARG;
+  std::vector<RoundPlan> plan;
+  if ((st = plan_rounds(len, *params, plan)) != CKV_OK) return st;
+  int64_t need = 0;
+  for (size_t j = 0; j < plan.size(); j += 2) need = std::max(need, (plan[j].s_out + page_tokens - 1) / page_tokens);  // rounds 0, 2, ... land in the scratch pages
+  const int64_t final_len = plan.empty() ? len : plan.back().s_out;
+  if (out_len) *out_len = final_len;
+  if (rounds) *rounds = (int64_t)plan.size();
+  if (scratch_pages) *scratch_pages = need;
+  if (result_in_scratch) *result_in_scratch = (int32_t)(plan.size() & 1);
+  if (pages_kept) *pages_kept = (final_len + page_tokens - 1) / page_tokens;
+  return CKV_OK;
+}
+
+size_t ckv_paged_workspace_bytes(int32_t L, int32_t H, int32_t D, int32_t dtype, int64_t len, const ckv_params* params) {
+  if (check_params(params) != CKV_OK || L <= 0 || H <= 0 || len < 0 || params->chunk != 64) return 0;
+  std::vector<RoundPlan> plan;
+  if (plan_rounds(len, *params, plan) != CKV_OK) return 256;
+  return layout_paged_workspace((int64_t)L * H, D, esize_of(dtype), params->chunk, plan).total;
+}
+
+int ckv_compress_paged(const ckv_page_pool* pools, int32_t L, int32_t H, int32_t D, int32_t dtype, int32_t page_tokens,
+                       const int32_t* block_table, int64_t len, int32_t has_deg, const int32_t* scratch_table,
+                       int64_t scratch_pages, const ckv_params* params, void* workspace, size_t workspace_bytes,
+                       void* cuda_stream, int64_t* out_len, int32_t* result_in_scratch) {
+  int st;
+  if ((st = paged_args_ok(pools, L, H, D, dtype, page_tokens, params)) != CKV_OK) return st;
+  if (!block_table || len < 0) return CKV_ERR_INVALID_ARG;
+  PagedArgs pg{};
+  for (int32_t l = 0; l < L; ++l) {
+    if (!pools[l].k_pages || !pools[l].v_pages || !pools[l].deg_pages) return CKV_ERR_INVALID_ARG;
+    if (!aligned16(pools[l].k_pages) || !aligned16(pools[l].v_pages)) return CKV_ERR_ALIGNMENT;
+    pg.k[l] = static_cast<unsigned char*>(pools[l].k_pages);
+    pg.v[l] = static_cast<unsigned char*>(pools[l].v_pages);
+    pg.deg[l] = pools[l].deg_pages;
+    pg.logdeg[l] = pools[l].logdeg_pages;
+  }
+  pg.H = H;
+  pg.shift = page_shift(page_tokens);
+  std::vector<RoundPlan> plan;
+  if ((st = plan_rounds(len, *params, plan)) != CKV_OK) return st;
+  int64_t need = 0;
+  for (size_t j = 0; j < plan.size(); j += 2) need = std::max(need, (plan[j].s_out + page_tokens - 1) / page_tokens);
+  if (need > 0 && (!scratch_table || scratch_pages < need)) return CKV_ERR_CAPACITY;
+  const int64_t LH = (int64_t)L * H;
+  const PagedWorkspace w = layout_paged_workspace(LH, D, esize_of(dtype), params->chunk, plan);
+  if (!workspace || workspace_bytes < w.total || !aligned16(workspace)) return CKV_ERR_WORKSPACE;
+  cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
+  if (cudaMemsetAsync(workspace, 0, 256, stream) != cudaSuccess) return CKV_ERR_CUDA;
+  unsigned char* ws = static_cast<unsigned char*>(workspace);
+  bool src_has_deg = has_deg != 0;
+  for (size_t j = 0; j < plan.size(); ++j) {
+    pg.src_table = (j & 1) ? scratch_table : block_table;
+    pg.dst_table = (j & 1) ? block_table : scratch_table;
+    if (run_round_paged(plan[j], pg, src_has_deg, (int)LH, D, params->chunk, w, ws, stream) != cudaSuccess) return CKV_ERR_CUDA;
+    src_has_deg = true;  // every round writes degrees
+  }
+  if (out_len) *out_len = plan.empty() ? len : plan.back().s_out;
+  if (result_in_scratch) *result_in_scratch = (int32_t)(plan.size() & 1);
+  return CKV_OK;
+}
 
 const char* ckv_status_string(int status) {
   switch (status) {

@@ -15,6 +15,7 @@
 // Waits on the mbarrier are bounded: a warp that gives up records it in the status word and leaves.
 #include <algorithm>
 #include <cstdint>
+#include <type_traits>
 
 #include "ckv_common.cuh"
 #include "ckv_internal.h"
@@ -70,8 +71,23 @@ struct FastArgs {
 
 enum FastKind : int { kFastAll = 0, kFastSelect = 1, kFastMatch = 2 };
 
-template <int NW, bool HAS_DEG, int KIND>
-__global__ void __launch_bounds__(NW * 32, 1) round_fast_kernel(const FastArgs a) {
+// row of token `pos` of KV head h in a pool's [n_pages, H, page_tokens] grid
+__device__ __forceinline__ int64_t page_row(const int32_t* table, int H, int shift, int h, int64_t pos) {
+  return (((int64_t)table[pos >> shift] * H + h) << shift) + (pos & (((int64_t)1 << shift) - 1));
+}
+
+__device__ __forceinline__ unsigned char* pg_k(const PagedArgs& pg, int l) { return pg.k[l]; }
+__device__ __forceinline__ unsigned char* pg_v(const PagedArgs& pg, int l) { return pg.v[l]; }
+__device__ __forceinline__ int32_t* pg_deg(const PagedArgs& pg, int l) { return pg.deg[l]; }
+__device__ __forceinline__ float* pg_logdeg(const PagedArgs& pg, int l) { return pg.logdeg[l]; }
+__device__ __forceinline__ unsigned char* pg_k(const NoPages&, int) { return nullptr; }
+__device__ __forceinline__ unsigned char* pg_v(const NoPages&, int) { return nullptr; }
+__device__ __forceinline__ int32_t* pg_deg(const NoPages&, int) { return nullptr; }
+__device__ __forceinline__ float* pg_logdeg(const NoPages&, int) { return nullptr; }
+
+template <int NW, bool HAS_DEG, int KIND, bool PAGED>
+__global__ void __launch_bounds__(NW * 32, 1)
+round_fast_kernel(const FastArgs a, const __grid_constant__ typename std::conditional<PAGED, PagedArgs, NoPages>::type pg) {
   extern __shared__ __align__(128) unsigned char smem[];
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
   const int g = lane >> 2, t = lane & 3;
@@ -95,10 +111,25 @@ __global__ void __launch_bounds__(NW * 32, 1) round_fast_kernel(const FastArgs a
   int64_t item = (int64_t)blockIdx.x * NW + warp;
   auto issue = [&](int64_t it) {
     const uint32_t lh = (uint32_t)it / n_full, ch = (uint32_t)it - lh * n_full;
-    const int64_t row0 = (int64_t)lh * a.src_cap + a.lo + (int64_t)ch * kC;
     mbar_arrive_expect_tx(bar, KIND == kFastMatch ? kTileBytes : kStageBytes);
-    bulk_load(k_s, a.k_src + row0 * kD, kTileBytes, bar);
-    if (KIND != kFastMatch) bulk_load(v_s, a.v_src + row0 * kD, kTileBytes, bar);  // the matching alone never reads V
+    if constexpr (PAGED) {
+      // a chunk is one run of rows inside a page, or two runs when it straddles a page boundary
+      const int l = (int)(lh / (uint32_t)pg.H), h = (int)(lh - (uint32_t)l * pg.H);
+      const int64_t pos0 = a.lo + (int64_t)ch * kC, page_tokens = (int64_t)1 << pg.shift;
+      const int n1 = (int)min((int64_t)kC, page_tokens - (pos0 & (page_tokens - 1)));
+      const int64_t r1 = page_row(pg.src_table, pg.H, pg.shift, h, pos0);
+      bulk_load(k_s, pg.k[l] + r1 * kRowBytes, (uint32_t)n1 * kRowBytes, bar);
+      if (KIND != kFastMatch) bulk_load(v_s, pg.v[l] + r1 * kRowBytes, (uint32_t)n1 * kRowBytes, bar);
+      if (n1 < kC) {
+        const int64_t r2 = page_row(pg.src_table, pg.H, pg.shift, h, pos0 + n1);
+        bulk_load(k_s + n1 * kRowBytes, pg.k[l] + r2 * kRowBytes, (uint32_t)(kC - n1) * kRowBytes, bar);
+        if (KIND != kFastMatch) bulk_load(v_s + n1 * kRowBytes, pg.v[l] + r2 * kRowBytes, (uint32_t)(kC - n1) * kRowBytes, bar);
+      }
+    } else {
+      const int64_t row0 = (int64_t)lh * a.src_cap + a.lo + (int64_t)ch * kC;
+      bulk_load(k_s, a.k_src + row0 * kD, kTileBytes, bar);
+      if (KIND != kFastMatch) bulk_load(v_s, a.v_src + row0 * kD, kTileBytes, bar);  // the matching alone never reads V
+    }
   };
   if (item < a.n_items && lane == 0) issue(item);
 
@@ -109,16 +140,46 @@ __global__ void __launch_bounds__(NW * 32, 1) round_fast_kernel(const FastArgs a
     const int64_t eslot = (int64_t)lh * a.edge_stride + (int64_t)ch * (kC / 2);
     int64_t out_row0 = (int64_t)lh * a.dst_cap;
     int ext_b = 1, ext_sel = 0;
+    int64_t out_pos0;  // position in the sequence of the chunk's first output row
     if (external) {
-      out_row0 += a.chunk_out_off[(int64_t)lh * a.n_chunks + ch];
+      out_pos0 = a.chunk_out_off[(int64_t)lh * a.n_chunks + ch];
       ext_b = a.edge_b[eslot + lane];
       ext_sel = a.sel[eslot + lane];
     } else {
-      out_row0 += a.out_lo + (int64_t)ch * a.out_stride;
+      out_pos0 = a.out_lo + (int64_t)ch * a.out_stride;
     }
+    out_row0 += out_pos0;
+    // paged: the layer and head of this slab, and the (at most two) destination pages the chunk's output rows reach
+    int pl = 0, ph = 0;
+    int64_t dst_pg0 = 0, dst_id0 = 0, dst_id1 = 0;
+    if constexpr (PAGED) {
+      pl = (int)(lh / (uint32_t)pg.H);
+      ph = (int)(lh - (uint32_t)pl * pg.H);
+      if (KIND != kFastMatch) {
+        dst_pg0 = out_pos0 >> pg.shift;
+        dst_id0 = pg.dst_table[min(dst_pg0, pg.dst_last_page)];
+        dst_id1 = pg.dst_table[min((out_pos0 + kC - 1) >> pg.shift, pg.dst_last_page)];
+      }
+    }
+    // row of output row `op` of this chunk: in the destination slab array, or in the destination pool's page grid
+    auto dst_row = [&](int op) -> int64_t {
+      if constexpr (PAGED) {
+        const int64_t pos = out_pos0 + op;
+        const int64_t id = (pos >> pg.shift) == dst_pg0 ? dst_id0 : dst_id1;
+        return ((id * pg.H + ph) << pg.shift) + (pos & (((int64_t)1 << pg.shift) - 1));
+      } else {
+        return out_row0 + op;
+      }
+    };
     if (HAS_DEG && KIND != kFastMatch) {
-      degs[lane] = a.deg_src[src_row0 + lane];
-      degs[lane + 32] = a.deg_src[src_row0 + lane + 32];
+      if constexpr (PAGED) {
+        const int64_t pos0 = a.lo + (int64_t)ch * kC;
+        degs[lane] = pg.deg[pl][page_row(pg.src_table, pg.H, pg.shift, ph, pos0 + lane)];
+        degs[lane + 32] = pg.deg[pl][page_row(pg.src_table, pg.H, pg.shift, ph, pos0 + lane + 32)];
+      } else {
+        degs[lane] = a.deg_src[src_row0 + lane];
+        degs[lane + 32] = a.deg_src[src_row0 + lane + 32];
+      }
     }
     if (!mbar_wait(bar, parity)) {
       if (lane == 0) atomicExch(a.status, 1);
@@ -280,8 +341,8 @@ __global__ void __launch_bounds__(NW * 32, 1) round_fast_kernel(const FastArgs a
 
       // ---- Eq. 5: one output row per B token, members gathered from the staged tiles; unmerged A tokens pass through
       int deg_lo = 0, deg_hi = 0;  // degrees of output rows `lane` and `lane + 32`
-      __nv_bfloat16* kdst = a.k_dst + out_row0 * kD + lane * 4;
-      __nv_bfloat16* vdst = a.v_dst + out_row0 * kD + lane * 4;
+      __nv_bfloat16* const kbase = (PAGED ? reinterpret_cast<__nv_bfloat16*>(pg_k(pg, pl)) : a.k_dst) + lane * 4;
+      __nv_bfloat16* const vbase = (PAGED ? reinterpret_cast<__nv_bfloat16*>(pg_v(pg, pl)) : a.v_dst) + lane * 4;
 #pragma unroll 2
       for (int j = 0; j < 32; ++j) {
         if (KIND == kFastSelect && !((selm >> j) & 1u)) {
@@ -290,8 +351,9 @@ __global__ void __launch_bounds__(NW * 32, 1) round_fast_kernel(const FastArgs a
           uint2 ck, cv;
           asm volatile("ld.shared.v2.u32 {%0,%1}, [%2];" : "=r"(ck.x), "=r"(ck.y) : "r"(k_s + arow));
           asm volatile("ld.shared.v2.u32 {%0,%1}, [%2];" : "=r"(cv.x), "=r"(cv.y) : "r"(v_s + arow));
-          *reinterpret_cast<uint2*>(kdst + (int64_t)op * kD) = ck;
-          *reinterpret_cast<uint2*>(vdst + (int64_t)op * kD) = cv;
+          const int64_t orow = dst_row(op);
+          *reinterpret_cast<uint2*>(kbase + orow * kD) = ck;
+          *reinterpret_cast<uint2*>(vbase + orow * kD) = cv;
           const int n_a = HAS_DEG ? degs[2 * j] : 1;
           if (lane == (op & 31)) (op < 32 ? deg_lo : deg_hi) = n_a;
         }
@@ -339,22 +401,27 @@ __global__ void __launch_bounds__(NW * 32, 1) round_fast_kernel(const FastArgs a
           uv.x = pack_bf16x2(fv[0] * inv, fv[1] * inv);
           uv.y = pack_bf16x2(fv[2] * inv, fv[3] * inv);
         }
-        *reinterpret_cast<uint2*>(kdst + (int64_t)op * kD) = uk;  // a B token nobody chose is copied bit for bit
-        *reinterpret_cast<uint2*>(vdst + (int64_t)op * kD) = uv;
+        const int64_t orow = dst_row(op);
+        *reinterpret_cast<uint2*>(kbase + orow * kD) = uk;  // a B token nobody chose is copied bit for bit
+        *reinterpret_cast<uint2*>(vbase + orow * kD) = uv;
         if (lane == (op & 31)) (op < 32 ? deg_lo : deg_hi) = n_new;
       }
       const int n_out = kC - __popc(selm);
+      int32_t* const deg_out = PAGED ? pg_deg(pg, pl) : a.deg_dst;
+      float* const logdeg_out = PAGED ? pg_logdeg(pg, pl) : a.logdeg_dst;
       if (lane < n_out) {
-        a.deg_dst[out_row0 + lane] = deg_lo;
-        if (a.logdeg_dst) a.logdeg_dst[out_row0 + lane] = logf((float)deg_lo);
+        const int64_t orow = dst_row(lane);
+        deg_out[orow] = deg_lo;
+        if (logdeg_out) logdeg_out[orow] = logf((float)deg_lo);
       }
       if (KIND == kFastSelect && lane + 32 < n_out) {
-        a.deg_dst[out_row0 + 32 + lane] = deg_hi;
-        if (a.logdeg_dst) a.logdeg_dst[out_row0 + 32 + lane] = logf((float)deg_hi);
+        const int64_t orow = dst_row(lane + 32);
+        deg_out[orow] = deg_hi;
+        if (logdeg_out) logdeg_out[orow] = logf((float)deg_hi);
       }
       if (a.assign) {
         int32_t* as = a.assign + (int64_t)lh * a.assign_stride + a.lo + (int64_t)ch * kC;
-        const int32_t slot0 = (int32_t)(out_row0 - (int64_t)lh * a.dst_cap);
+        const int32_t slot0 = (int32_t)out_pos0;
         const bool merged = (selm >> lane) & 1u;
         as[2 * lane] = slot0 + (merged ? slot_b(my_best) : slot_a(lane));  // a merged A token joins its B token's slot
         as[2 * lane + 1] = slot0 + slot_b(lane);
@@ -370,30 +437,25 @@ __global__ void __launch_bounds__(NW * 32, 1) round_fast_kernel(const FastArgs a
   }
 }
 
-template <int NW, bool HAS_DEG, int KIND>
-cudaError_t launch_fast_inst(const FastArgs& a, cudaStream_t st) {
+template <int NW, bool HAS_DEG, int KIND, bool PAGED, typename PG>
+cudaError_t launch_fast_inst(const FastArgs& a, const PG& pg, cudaStream_t st) {
   const size_t smem = (size_t)NW * ((KIND == kFastMatch ? kTileBytes : kStageBytes) + kExtraBytes);
   const int64_t ctas = std::min<int64_t>(sm_count(), (a.n_items + NW - 1) / NW);
-  cudaError_t e = cudaFuncSetAttribute(round_fast_kernel<NW, HAS_DEG, KIND>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+  cudaError_t e = cudaFuncSetAttribute(round_fast_kernel<NW, HAS_DEG, KIND, PAGED>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
   if (e != cudaSuccess) return e;
-  round_fast_kernel<NW, HAS_DEG, KIND><<<(unsigned)ctas, NW * 32, smem, st>>>(a);
+  round_fast_kernel<NW, HAS_DEG, KIND, PAGED><<<(unsigned)ctas, NW * 32, smem, st>>>(a, pg);
   return cudaGetLastError();
 }
 
-template <int NW, int KIND>
-cudaError_t launch_fast_kind(const FastArgs& a, cudaStream_t st) {
+template <int NW, int KIND, bool PAGED, typename PG>
+cudaError_t launch_fast_kind(const FastArgs& a, const PG& pg, cudaStream_t st) {
   // the matching alone never reads degrees
-  return (a.deg_src && KIND != kFastMatch) ? launch_fast_inst<NW, true, KIND>(a, st) : launch_fast_inst<NW, false, KIND>(a, st);
+  return (a.deg_src && KIND != kFastMatch) ? launch_fast_inst<NW, true, KIND, PAGED>(a, pg, st)
+                                           : launch_fast_inst<NW, false, KIND, PAGED>(a, pg, st);
 }
 
-}  // namespace
-
-bool round_fast_supported(const RoundArgs& a, int dtype, int D) {
-  return dtype == 1 && D == 128 && a.chunk == kC && a.status != nullptr && (int64_t)a.LH * a.n_chunks < (1ll << 31);
-}
-
-// The full chunks of a round in any mode.  The shorter last chunk, if any, is left to the tile kernel.
-cudaError_t launch_round_fast(const RoundArgs& r, int64_t n_full, cudaStream_t st) {
+template <bool PAGED, typename PG>
+cudaError_t launch_fast_any(const RoundArgs& r, const PG& pg, int64_t n_full, cudaStream_t st) {
   // r.chunk_first > 0: only the full chunks from that one on (modes whose output offsets are a multiple of the chunk index)
   const int64_t first = r.chunk_first;
   n_full -= first;
@@ -426,10 +488,23 @@ cudaError_t launch_round_fast(const RoundArgs& r, int64_t n_full, cudaStream_t s
   a.sel = r.sel;
   a.chunk_out_off = r.chunk_out_off;
   switch (r.mode) {
-    case kModeAll: return launch_fast_kind<7, kFastAll>(a, st);
-    case kModeMatchOnly: return launch_fast_kind<13, kFastMatch>(a, st);  // half the bytes per warp: twice the warps
-    default: return launch_fast_kind<7, kFastSelect>(a, st);
+    case kModeAll: return launch_fast_kind<7, kFastAll, PAGED>(a, pg, st);
+    case kModeMatchOnly: return launch_fast_kind<13, kFastMatch, PAGED>(a, pg, st);  // half the bytes per warp: twice the warps
+    default: return launch_fast_kind<7, kFastSelect, PAGED>(a, pg, st);
   }
+}
+
+}  // namespace
+
+bool round_fast_supported(const RoundArgs& a, int dtype, int D) {
+  return dtype == 1 && D == 128 && a.chunk == kC && a.status != nullptr && (int64_t)a.LH * a.n_chunks < (1ll << 31);
+}
+
+// The full chunks of a round in any mode.  The shorter last chunk, if any, is left to the tile kernel.
+cudaError_t launch_round_fast(const RoundArgs& r, int64_t n_full, cudaStream_t st) { return launch_fast_any<false>(r, NoPages{}, n_full, st); }
+
+cudaError_t launch_round_fast_paged(const RoundArgs& r, const PagedArgs& pg, int64_t n_full, cudaStream_t st) {
+  return launch_fast_any<true>(r, pg, n_full, st);
 }
 
 }  // namespace ckv

@@ -78,6 +78,42 @@ struct AppendBatchArgs {
   int32_t LH;
 };
 
+// A cache in pages (the block layout of serving engines): per layer one pool k, v [n_pages, H, page_tokens, D], deg and
+// logdeg [n_pages, H, page_tokens]; a sequence's token t sits in page table[t >> shift] at offset t & (page_tokens - 1).
+// A round reads the sequence through src_table and writes it through dst_table (other pages of the same pools).
+constexpr int kMaxPoolLayers = 64;
+struct PagedArgs {
+  unsigned char* k[kMaxPoolLayers];
+  unsigned char* v[kMaxPoolLayers];
+  int32_t* deg[kMaxPoolLayers];
+  float* logdeg[kMaxPoolLayers];   // entries may be null
+  const int32_t* src_table;
+  const int32_t* dst_table;
+  int64_t dst_last_page;           // last entry of dst_table that the round's output reaches
+  int32_t H, shift;
+};
+struct NoPages {};
+
+// Row copies between the two homes a sequence can have: pages of the per-layer pools, or a contiguous [LH, cap] slab.
+struct RowsEnd {
+  const int32_t* table;  // non-null: the rows live in pages (pools of the PagedArgs that comes with the call)
+  unsigned char* k;      // else: slab arrays
+  unsigned char* v;
+  int32_t* deg;
+  float* logdeg;         // may be null
+  int64_t cap;
+};
+struct RowsCopyArgs {
+  RowsEnd src, dst;
+  int64_t src_off, dst_off, count;  // `count` rows from position src_off to position dst_off, for every slab
+  // optional (device): for slab lh the copy starts at dst position begin[lh * begin_stride + begin_index] instead of
+  // dst_off and ends at dst_end; the source moves along (src position = src_off + (position - dst_off))
+  const int32_t* begin;
+  int64_t begin_stride, begin_index, dst_end;
+  int32_t LH, row_bytes;
+  bool src_has_deg;  // else every copied row gets degree 1
+};
+
 struct SelectArgs {
   const float* edge_sim;
   uint8_t* sel;
@@ -140,6 +176,8 @@ inline cudaError_t launch_dependent(void (*kernel)(KArgs...), dim3 grid, dim3 bl
 cudaError_t launch_round(const RoundArgs& a, int dtype, int D, cudaStream_t st);
 cudaError_t launch_copy(const CopyArgs& a, int dtype, int D, cudaStream_t st);
 cudaError_t launch_select(const SelectArgs& a, cudaStream_t st);
+int page_shift(int32_t page_tokens);  // log2 of a valid page size (a power of two >= 32), else -1
+cudaError_t launch_rows_copy(const RowsCopyArgs& a, const PagedArgs& pools, cudaStream_t st);
 cudaError_t launch_append_batch(const AppendBatchArgs& a, int dtype, int D, cudaStream_t st);
 cudaError_t launch_compose_assign(int32_t* total, const int32_t* step, int64_t n_src, int64_t step_stride, int32_t LH,
                                   cudaStream_t st);
@@ -151,6 +189,8 @@ size_t decode_partial_floats(int32_t Bz, int32_t H, int32_t G, int32_t D, int64_
 size_t round_smem_bytes(int chunk, int D);
 bool round_fast_supported(const RoundArgs& a, int dtype, int D);
 cudaError_t launch_round_fast(const RoundArgs& a, int64_t n_full, cudaStream_t st);
+// the same round on a paged cache (a.k_src, a.k_dst ... are not used; a.deg_src != null only says that the pages carry degrees)
+cudaError_t launch_round_fast_paged(const RoundArgs& a, const PagedArgs& pg, int64_t n_full, cudaStream_t st);
 bool round_umma_supported(const RoundArgs& a, int dtype, int D);
 cudaError_t launch_round_umma(const RoundArgs& a, int64_t n_full, cudaStream_t st);
 bool bsm_supported(int dtype, int D);

@@ -63,6 +63,44 @@ __global__ void __launch_bounds__(256) page_copy_kernel(const PageCopyArgs a) {
   }
 }
 
+// grid (x, slab lh): K and V rows 16 bytes per thread and step, then degrees and log-degrees one row per thread
+__global__ void __launch_bounds__(256) rows_copy_kernel(const RowsCopyArgs a, const __grid_constant__ PagedArgs pools) {
+  const int lh = blockIdx.y;
+  const int l = lh / pools.H, h = lh - l * pools.H;
+  const int64_t mask = ((int64_t)1 << pools.shift) - 1;
+  int64_t dst_off = a.dst_off, count = a.count;
+  if (a.begin) {
+    dst_off = a.begin[(int64_t)lh * a.begin_stride + a.begin_index];
+    count = a.dst_end - dst_off;
+  }
+  const int64_t src_off = a.src_off + (dst_off - a.dst_off);
+  auto row_of = [&](const RowsEnd& e, int64_t pos) -> int64_t {
+    return e.table ? ((((int64_t)e.table[pos >> pools.shift] * pools.H + h) << pools.shift) + (pos & mask)) : ((int64_t)lh * e.cap + pos);
+  };
+  const unsigned char* ks = a.src.table ? pools.k[l] : a.src.k;
+  const unsigned char* vs = a.src.table ? pools.v[l] : a.src.v;
+  unsigned char* kd = a.dst.table ? pools.k[l] : a.dst.k;
+  unsigned char* vd = a.dst.table ? pools.v[l] : a.dst.v;
+  const int vec_per_row = a.row_bytes / 16;
+  const int64_t nvec = count * vec_per_row, stride = (int64_t)gridDim.x * blockDim.x;
+  for (int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; i < nvec; i += stride) {
+    const int64_t t = i / vec_per_row;
+    const int c = (int)(i - t * vec_per_row);
+    const int64_t sr = row_of(a.src, src_off + t), dr = row_of(a.dst, dst_off + t);
+    reinterpret_cast<uint4*>(kd + dr * a.row_bytes)[c] = reinterpret_cast<const uint4*>(ks + sr * a.row_bytes)[c];
+    reinterpret_cast<uint4*>(vd + dr * a.row_bytes)[c] = reinterpret_cast<const uint4*>(vs + sr * a.row_bytes)[c];
+  }
+  const int32_t* ds = a.src.table ? pools.deg[l] : a.src.deg;
+  int32_t* dd = a.dst.table ? pools.deg[l] : a.dst.deg;
+  float* ld = a.dst.table ? pools.logdeg[l] : a.dst.logdeg;
+  for (int64_t t = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; t < count; t += stride) {
+    const int dg = (a.src_has_deg && ds) ? ds[row_of(a.src, src_off + t)] : 1;
+    const int64_t dr = row_of(a.dst, dst_off + t);
+    if (dd) dd[dr] = dg;
+    if (ld) ld[dr] = logf((float)dg);
+  }
+}
+
 inline int page_shift_of(int32_t page_tokens) {
   if (page_tokens < 32 || (page_tokens & (page_tokens - 1))) return -1;
   int s = 0;
@@ -84,6 +122,18 @@ int page_copy(bool to_pages, const PageCopyArgs& a, cudaStream_t st) {
 inline bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
 
 }  // namespace
+
+cudaError_t launch_rows_copy(const RowsCopyArgs& a, const PagedArgs& pools, cudaStream_t st) {
+  if (a.LH <= 0 || (!a.begin && a.count <= 0)) return cudaSuccess;
+  const int64_t rows = a.begin ? 64 : a.count;  // with a device-side start the copy is a chunk's worth at most
+  const int64_t nvec = rows * (a.row_bytes / 16);
+  const dim3 grid((unsigned)std::min<int64_t>((nvec + 255) / 256, 1184), (unsigned)a.LH);
+  rows_copy_kernel<<<grid, 256, 0, st>>>(a, pools);
+  return cudaGetLastError();
+}
+
+int page_shift(int32_t page_tokens) { return page_shift_of(page_tokens); }
+
 }  // namespace ckv
 
 using namespace ckv;

@@ -137,3 +137,131 @@ def test_paged_argument_checks():
     assert b.lib.ckv_decode_attn_paged(0x1000, 0x2000, 0x3000, None, 64, 1, 1, 1, 128, b.F32, 0x4000, 0x5000, 0.1, 10, 0x6000, 1 << 20, None) == 6
     assert b.lib.ckv_pages_gather(0x1000, 10, 0x2000, 0x3000, None, 16, 1, 128, b.BF16, 0x4000, 0x5000, None, None, 10, None) == 6
     assert b.lib.ckv_pages_gather(0x1000, 10, 0x2000, 0x3000, None, 64, 1, 128, b.BF16, 0x4000, 0x5000, None, None, 5, None) == 1
+
+
+# ----------------------------------------------------------------------------- clustering directly on pages
+
+def make_pools(L, n_pages, H, P, D, seed):
+    pools = []
+    for l in range(L):
+        kp, vp, dp, lp = make_pool(n_pages, H, P, D, seed=seed + l)
+        pools.append((kp, vp, dp, lp))
+    return pools
+
+
+def gathered(pools, table, n):
+    """The sequence a block table describes, as the oracle sees it: K, V [L, H, n, D] float64, deg [L, H, n]."""
+    tab = table.cpu().numpy()
+    K = np.stack([O.gather_pages(PU.to_np64(kp), tab, n) for kp, _, _, _ in pools])
+    V = np.stack([O.gather_pages(PU.to_np64(vp), tab, n) for _, vp, _, _ in pools])
+    deg = np.stack([O.gather_pages(dp.cpu().numpy().astype(np.int64), tab, n) for _, _, dp, _ in pools])
+    lg = np.stack([O.gather_pages(lp.cpu().numpy().astype(np.float64), tab, n) for _, _, _, lp in pools])
+    return K, V, deg, lg
+
+
+def paged_compress_case(L, H, P, s, p, seed):
+    """read pages -> compress -> write back -> free blocks, without leaving the pages.  By definition the result is the
+    oracle's compress_prefill of the gathered sequence, found through the table that ckv_pages_plan names; the number of
+    pages the sequence keeps is ceil(out_len / P)."""
+    from paper_2506_11418_b200 import binding as b
+    D = 128
+    own = (s + P - 1) // P
+    out_len, rounds, n_scratch, in_scratch, kept = b.pages_plan(s, p, P)
+    assert kept == (out_len + P - 1) // P
+    pool_pages = own + n_scratch + 3
+    pools = make_pools(L, pool_pages, H, P, D, seed)
+    perm = torch.randperm(pool_pages, generator=torch.Generator().manual_seed(seed)).to(torch.int32)
+    table, scratch = perm[:own].to(DEV), perm[own:own + n_scratch].to(DEV)
+    spare = perm[own + n_scratch:]
+    K = synth.ar1_keys(L, H, s, D, (0.7, 0.95), 0.5, seed=seed, dtype="bf16", device=DEV)
+    V = synth.normal_values(L, H, s, D, seed=seed, dtype="bf16", device=DEV)
+    for l, (kp, vp, dp, lp) in enumerate(pools):
+        b.pages_scatter(table, s, K[l], V[l], None, kp, vp, dp, lp)
+    untouched = [(kp[spare.long()].clone(), vp[spare.long()].clone()) for kp, vp, _, _ in pools]
+    ws = torch.empty(b.paged_workspace_bytes(L, H, D, torch.bfloat16, s, p), dtype=torch.uint8, device=DEV)
+    got_len, got_in_scratch = b.compress_paged(pools, table, s, False, scratch if n_scratch else None, p, ws)
+    assert b.workspace_status(ws) == 0
+    assert got_len == out_len and got_in_scratch == in_scratch
+    result_table = (scratch if in_scratch else table)[:kept]
+    Kg, Vg, dg, lg = gathered(pools, result_table, out_len)
+    po = PU.oracle_params(p)
+    Ko, Vo, do, _, logs = O.compress_prefill(PU.to_np64(K), PU.to_np64(V), None, po, storage="bf16")
+    assert len(logs) == rounds and Ko.shape[2] == out_len
+    np.testing.assert_array_equal(dg, do)
+    np.testing.assert_allclose(lg, np.log(do.astype(np.float64)), rtol=1e-6, atol=1e-7)
+    for got, ref in ((Kg, Ko), (Vg, Vo)):
+        assert np.all(np.abs(got - ref) <= max(rounds, 1) * PU.bf16_ulp(ref) * 1.0001 + 1e-30)
+        assert np.mean(got == ref) >= 0.99
+    for (kp, vp, _, _), (k0, v0) in zip(pools, untouched):          # pages of neither table are left alone
+        assert torch.equal(kp[spare.long()], k0) and torch.equal(vp[spare.long()], v0)
+    return pools, result_table, out_len, K, V
+
+
+@pytest.mark.parametrize("P,s,sink,recent,rounds,r,decay,select,budget", [
+    (64, 4096, 0, 0, 1, 1.0, 0.0, 0, 0),          # page-aligned chunks, one round: the result is in the scratch pages
+    (64, 4096 + 37, 16, 64, 2, 1.0, 0.0, 0, 0),   # chunks straddle pages, a shorter last chunk, two rounds: back in its own pages
+    (128, 3000, 16, 64, 1, 0.8, 0.0, 0, 0),       # ranked per head: matching pass, ranking, merge pass; last chunk staged
+    (256, 5000, 5, 9, 3, 0.5, 0.0, 1, 0),         # ranked per chunk, three rounds
+    (64, 6000, 16, 64, 16, 0.8, 0.2, 0, 1500),    # the paper's schedule to a 25 % budget: six rounds, the last one trimmed
+    (64, 100, 0, 0, 1, 1.0, 0.0, 0, 0),           # one full chunk and a last chunk
+    (64, 50, 0, 0, 2, 1.0, 0.0, 0, 0),            # nothing but a last chunk
+    (64, 1, 0, 0, 1, 1.0, 0.0, 0, 0),             # nothing to merge
+])
+def test_compress_paged_against_the_oracle(P, s, sink, recent, rounds, r, decay, select, budget):
+    from paper_2506_11418_b200 import binding as b
+    p = b.Params(chunk=64, n_sink=sink, n_recent=recent, n_rounds_max=rounds, r_init=r, r_decay=decay, r_min=min(r, 0.2) if decay else r,
+                 select=select, budget=budget)
+    paged_compress_case(2, 3, P, s, p, seed=600 + s)
+
+
+def test_compress_paged_again_with_degrees_then_attend():
+    """A second compression of the same sequence reads the degrees the first one left in the pages; decode attention then
+    runs over the kept pages."""
+    from paper_2506_11418_b200 import binding as b
+    L, H, G, P, s, D = 2, 2, 4, 64, 3000, 128
+    p1 = b.Params(chunk=64, n_sink=16, n_recent=64, n_rounds_max=1, r_init=0.6, r_decay=0.0, r_min=0.6, select=b.SELECT_GLOBAL)
+    pools, table, n1, K, V = paged_compress_case(L, H, P, s, p1, seed=77)
+    # second call: fresh scratch pages (appended to every pool)
+    out_len, rounds, n_scratch, in_scratch, kept = b.pages_plan(n1, p1, P)
+    base = pools[0][0].shape[0]
+    pools = [(torch.cat([kp, torch.zeros((n_scratch, H, P, D), dtype=kp.dtype, device=DEV)]),
+              torch.cat([vp, torch.zeros((n_scratch, H, P, D), dtype=vp.dtype, device=DEV)]),
+              torch.cat([dp, torch.zeros((n_scratch, H, P), dtype=dp.dtype, device=DEV)]),
+              torch.cat([lp, torch.zeros((n_scratch, H, P), dtype=lp.dtype, device=DEV)])) for kp, vp, dp, lp in pools]
+    scratch = torch.arange(base, base + n_scratch, dtype=torch.int32, device=DEV)
+    K1, V1, d1, _ = gathered(pools, table, n1)
+    ws = torch.empty(b.paged_workspace_bytes(L, H, D, torch.bfloat16, n1, p1), dtype=torch.uint8, device=DEV)
+    got_len, got_in = b.compress_paged(pools, table, n1, True, scratch, p1, ws)
+    assert b.workspace_status(ws) == 0 and got_len == out_len and got_in == in_scratch
+    res = (scratch if in_scratch else table)[:kept]
+    Kg, Vg, dg, _ = gathered(pools, res, out_len)
+    Ko, Vo, do, _, _ = O.compress_prefill(K1, V1, d1, PU.oracle_params(p1), storage="bf16")
+    np.testing.assert_array_equal(dg, do)
+    assert int(dg.sum(axis=2).min()) == s == int(dg.sum(axis=2).max())     # every original token is still accounted for
+    for got, ref in ((Kg, Ko), (Vg, Vo)):
+        assert np.all(np.abs(got - ref) <= PU.bf16_ulp(ref) * 1.0001 + 1e-30)
+    q = synth.queries(1, H * G, D, seed=13, dtype="bf16", device=DEV)
+    out = torch.empty_like(q)
+    wsd = torch.empty(b.decode_workspace_bytes(1, H, G, D, out_len), dtype=torch.uint8, device=DEV)
+    scale = 1.0 / math.sqrt(D)
+    kp, vp, dp, lp = pools[1]
+    b.decode_attn_paged(b.paged_views([res], [out_len], DEV), kp, vp, lp, H, G, q, out, scale, out_len, wsd)
+    torch.cuda.synchronize()
+    PU.summarize_attention([PU.check_attention(PU.to_np64(out[0]), PU.to_np64(q[0]), Kg[1], Vg[1], dg[1], scale, "bf16",
+                                               "pages clustered twice")], "pages clustered twice")
+
+
+def test_compress_paged_argument_checks():
+    from paper_2506_11418_b200 import binding as b
+    import ctypes as C
+    pool = (b.CkvPagePool * 1)(b.CkvPagePool(0x1000, 0x2000, 0x3000, None))
+    p = b.Params(chunk=64, n_sink=0, n_recent=0, n_rounds_max=1, r_init=1.0, r_decay=0.0, r_min=1.0)
+    call = lambda **kw: b.lib.ckv_compress_paged(pool, 1, kw.get("H", 2), 128, kw.get("dtype", b.BF16), kw.get("P", 64), 0x4000, kw.get("n", 1000), 0,
+                                                 kw.get("scratch", 0x5000), kw.get("n_scratch", 100), C.byref(kw.get("p", p).c()), kw.get("ws", 0x6000),
+                                                 kw.get("ws_bytes", 1 << 30), None, None, None)
+    assert call(P=48) == 6 and call(P=32) == 6 and call(dtype=b.F32) == 6             # page size, dtype: unsupported here
+    assert call(p=b.Params(chunk=128, n_sink=0, n_recent=0, n_rounds_max=1, r_init=1.0, r_decay=0.0, r_min=1.0)) == 6
+    assert call(n_scratch=3) == 3                                                     # too few scratch pages
+    assert call(ws_bytes=64) == 4                                                     # workspace too small
+    out_len, rounds, n_scratch, in_scratch, kept = b.pages_plan(1000, p, 64)
+    assert (out_len, rounds, n_scratch, in_scratch, kept) == (500, 1, 8, True, 8)
