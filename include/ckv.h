@@ -184,6 +184,17 @@ int ckv_decode_attn_paged(const ckv_paged_view* views_dev, const void* k_pages, 
                           int32_t page_tokens, int32_t Bz, int32_t H, int32_t G, int32_t D, int32_t dtype, const void* q,
                           void* out, float scale, int64_t max_len, void* workspace, size_t workspace_bytes, void* cuda_stream);
 
+/* One decoding step of Algorithm 1 on a paged cache in a single launch: `K = [K, k], V = [V, v], N = [N, 1]` and Eq. 3
+ * over the result.  views_dev[b].len is the length BEFORE the step; sequence b's new token k_new, v_new [Bz, H, D] is
+ * written to slot len of its pages (the page block_table[len / page_tokens] must already belong to the sequence) with
+ * degree 1 and log-degree 0, and the attention runs over len + 1 tokens, the new one read straight from k_new / v_new.
+ * The device views are not modified: the caller raises len for the next step.  max_len (host): an upper bound on every
+ * len + 1.  deg_pages is required, logdeg_pages NULL = all degrees one.  Otherwise as ckv_decode_attn_paged. */
+int ckv_decode_append_attn_paged(const ckv_paged_view* views_dev, void* k_pages, void* v_pages, int32_t* deg_pages,
+                                 float* logdeg_pages, int32_t page_tokens, int32_t Bz, int32_t H, int32_t G, int32_t D, int32_t dtype,
+                                 const void* k_new, const void* v_new, const void* q, void* out, float scale, int64_t max_len,
+                                 void* workspace, size_t workspace_bytes, void* cuda_stream);
+
 /* Copies one sequence's first `len` tokens of one layer between its pages and a contiguous slab k, v [H, cap, D],
  * deg [H, cap] (logdeg [H, cap] optional): gather = pages -> slab (to run ckv_compress_* on it), scatter = slab -> pages
  * (degrees and their logarithms are written to the pages as well; deg NULL on scatter = all ones).  deg_pages may be

@@ -21,7 +21,8 @@ OK = 0
 EXPORTS = ["ckv_compress_plan", "ckv_workspace_bytes", "ckv_compress_prefill", "ckv_compress_append", "ckv_compress_append_batch",
            "ckv_decode_workspace_bytes", "ckv_decode_attn", "ckv_status_string", "ckv_workspace_status",
            "ckv_decode_attn_static", "ckv_compress_append_recluster", "ckv_decode_attn_paged", "ckv_pages_gather",
-           "ckv_pages_scatter", "ckv_pages_plan", "ckv_paged_workspace_bytes", "ckv_compress_paged"]
+           "ckv_pages_scatter", "ckv_pages_plan", "ckv_paged_workspace_bytes", "ckv_compress_paged",
+           "ckv_decode_append_attn_paged"]
 
 
 class CkvPagePool(C.Structure):
@@ -79,6 +80,10 @@ def _load():
     lib.ckv_pages_scatter.restype = C.c_int
     lib.ckv_pages_scatter.argtypes = [C.c_void_p, C.c_int64, C.c_void_p, C.c_void_p, C.c_void_p, C.c_int64, C.c_int32, C.c_int32,
                                       C.c_int32, C.c_int32, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p]
+    lib.ckv_decode_append_attn_paged.restype = C.c_int
+    lib.ckv_decode_append_attn_paged.argtypes = [C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_int32, C.c_int32, C.c_int32,
+                                                 C.c_int32, C.c_int32, C.c_int32, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_float,
+                                                 C.c_int64, C.c_void_p, C.c_size_t, C.c_void_p]
     lib.ckv_pages_plan.restype = C.c_int
     lib.ckv_pages_plan.argtypes = [C.c_int64, C.POINTER(CkvParams), C.c_int32, C.POINTER(C.c_int64), C.POINTER(C.c_int64),
                                    C.POINTER(C.c_int64), C.POINTER(C.c_int32), C.POINTER(C.c_int64)]
@@ -353,6 +358,19 @@ def decode_attn_paged(views: torch.Tensor, k_pages, v_pages, logdeg_pages, H: in
     _check(lib.ckv_decode_attn_paged(views.data_ptr(), k_pages.data_ptr(), v_pages.data_ptr(), _ptr(logdeg_pages), k_pages.shape[2],
                                      Bz, H, G, D, dtype_code(q.dtype), q.data_ptr(), out.data_ptr(), scale, max_len,
                                      workspace.data_ptr(), workspace.numel() * workspace.element_size(), _stream_ptr()))
+
+
+def decode_append_attn_paged(views: torch.Tensor, k_pages, v_pages, deg_pages, logdeg_pages, H: int, G: int, k_new, v_new, q, out,
+                             scale: float, max_len: int, workspace: torch.Tensor):
+    """ckv_decode_append_attn_paged on the current stream: k_new, v_new [Bz, H, D] are written to slot views[b].len of
+    every sequence's pages and attended to in the same launch; max_len bounds every len + 1."""
+    Bz, HG, D = q.shape
+    assert HG == H * G and q.is_contiguous() and out.is_contiguous() and k_new.is_contiguous() and v_new.is_contiguous()
+    assert k_new.shape == (Bz, H, D) and v_new.shape == (Bz, H, D)
+    _check(lib.ckv_decode_append_attn_paged(views.data_ptr(), k_pages.data_ptr(), v_pages.data_ptr(), deg_pages.data_ptr(),
+                                            _ptr(logdeg_pages), k_pages.shape[2], Bz, H, G, D, dtype_code(q.dtype), k_new.data_ptr(),
+                                            v_new.data_ptr(), q.data_ptr(), out.data_ptr(), scale, max_len, workspace.data_ptr(),
+                                            workspace.numel() * workspace.element_size(), _stream_ptr()))
 
 
 def pages_gather(block_table, length, k_pages, v_pages, deg_pages, k, v, deg, logdeg=None):

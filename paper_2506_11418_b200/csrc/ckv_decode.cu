@@ -356,11 +356,14 @@ __global__ void __launch_bounds__(NW * 32, 1) decode_fast_kernel(const DecodeArg
   if (PAGED) {
     const ckv_paged_view pv = reinterpret_cast<const ckv_paged_view*>(a.views)[b];
     table = pv.block_table;
-    view.len = pv.len;
+    view.len = pv.len + (a.k_new ? 1 : 0);  // fused append: the new token is position pv.len
   } else {
     view = reinterpret_cast<const ckv_layer_view*>(a.views)[b];
   }
   const int64_t len = view.len;
+  const int64_t new_pos = (PAGED && a.k_new) ? len - 1 : -1;
+  const __nv_bfloat16* knew = PAGED ? reinterpret_cast<const __nv_bfloat16*>(a.k_new) + ((int64_t)b * a.H + h) * 128 : nullptr;
+  const __nv_bfloat16* vnew = PAGED ? reinterpret_cast<const __nv_bfloat16*>(a.v_new) + ((int64_t)b * a.H + h) * 128 : nullptr;
   // the sequence's own tiles are dealt evenly to the splits (a ragged batch stays balanced)
   const int64_t seq_tiles = (len + TT - 1) / TT;
   const int64_t t_begin = TT * (seq_tiles * split / a.n_splits);
@@ -412,14 +415,27 @@ __global__ void __launch_bounds__(NW * 32, 1) decode_fast_kernel(const DecodeArg
       const bool ok = t0 + r < t_end;
       const int64_t row = ok ? row0 + r : row0;  // clamped address, zero-filled when out of range
       const uint32_t off = (uint32_t)r * 256u + (uint32_t)((c ^ (r & 7)) << 4);
-      cp_async16(st + off, kbase + row * D + c * 8, ok ? 16u : 0u);
-      cp_async16(st + kTileBytes + off, vbase + row * D + c * 8, ok ? 16u : 0u);
+      const bool fresh = PAGED && t0 + r == new_pos;  // the appended token is read from where the caller put it
+      cp_async16(st + off, (fresh ? knew : kbase + row * D) + c * 8, ok ? 16u : 0u);
+      cp_async16(st + kTileBytes + off, (fresh ? vnew : vbase + row * D) + c * 8, ok ? 16u : 0u);
     }
     if (ldbase) {  // one log-degree per lane; 4-byte copies have no alignment demands on the slab
-      const bool ok = lane < TT && t0 + lane < t_end;
+      // (the appended token has degree 1: its log-degree is the zero fill)
+      const bool ok = lane < TT && t0 + lane < t_end && t0 + lane != new_pos;
       if (TT == 32 || lane < TT) cp_async4(st + 2 * kTileBytes + lane * 4, ldbase + (ok ? row0 + lane : row0), ok ? 4u : 0u);
     }
   };
+
+  if (PAGED && new_pos >= t_begin && new_pos < t_end) {
+    // K = [K, k], V = [V, v], N = [N, 1]: the warp whose span holds the new position writes it to its page slot
+    const int64_t row = (((int64_t)table[new_pos >> a.page_shift] * a.H + h) << a.page_shift) + (new_pos & (((int64_t)1 << a.page_shift) - 1));
+    const uint4 x = reinterpret_cast<const uint4*>(lane < 16 ? knew : vnew)[lane & 15];
+    reinterpret_cast<uint4*>(reinterpret_cast<__nv_bfloat16*>(lane < 16 ? a.k_pages_w : a.v_pages_w) + row * D)[lane & 15] = x;
+    if (lane == 0) {
+      a.deg_pages_w[row] = 1;
+      if (a.logdeg_pages_w) a.logdeg_pages_w[row] = 0.f;
+    }
+  }
 
   float oacc[8][4];
 #pragma unroll

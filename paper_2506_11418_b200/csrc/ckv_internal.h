@@ -140,6 +140,14 @@ struct DecodeArgs {
   const void* v_pages;
   const float* logdeg_pages;  // [n_pages, H, page_tokens] or null
   int32_t page_shift;         // log2(page_tokens), page_tokens >= 32
+  // paged, fused append (all null otherwise): sequence b's new token k_new / v_new [Bz, H, D] is attended to as
+  // position len and written to that slot of its page with degree 1
+  const void* k_new;
+  const void* v_new;
+  void* k_pages_w;
+  void* v_pages_w;
+  int32_t* deg_pages_w;
+  float* logdeg_pages_w;      // may be null
 };
 
 // Streaming multiprocessors of the current device, asked once per device (the grids are sized from it).

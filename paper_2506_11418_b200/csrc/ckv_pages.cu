@@ -197,4 +197,30 @@ int ckv_decode_attn_paged(const ckv_paged_view* views_dev, const void* k_pages, 
   return launch_decode_paged(a, static_cast<cudaStream_t>(cuda_stream)) == cudaSuccess ? CKV_OK : CKV_ERR_CUDA;
 }
 
+int ckv_decode_append_attn_paged(const ckv_paged_view* views_dev, void* k_pages, void* v_pages, int32_t* deg_pages,
+                                 float* logdeg_pages, int32_t page_tokens, int32_t Bz, int32_t H, int32_t G, int32_t D, int32_t dtype,
+                                 const void* k_new, const void* v_new, const void* q, void* out, float scale, int64_t max_len,
+                                 void* workspace, size_t workspace_bytes, void* cuda_stream) {
+  if (!views_dev || !k_pages || !v_pages || !deg_pages || !k_new || !v_new || !q || !out || Bz <= 0 || H <= 0 || G <= 0 || max_len < 1)
+    return CKV_ERR_INVALID_ARG;
+  if (dtype != CKV_F32 && dtype != CKV_BF16) return CKV_ERR_INVALID_ARG;
+  const int shift = page_shift_of(page_tokens);
+  if (dtype != CKV_BF16 || shift < 0 || D != 128 || G > 8 || H > 65535 || Bz > 65535) return CKV_ERR_UNSUPPORTED;
+  if (!aligned16(q) || !aligned16(out) || !aligned16(k_pages) || !aligned16(v_pages) || !aligned16(k_new) || !aligned16(v_new))
+    return CKV_ERR_ALIGNMENT;
+  const size_t need = ckv_decode_workspace_bytes(Bz, H, G, D, max_len);
+  if (!workspace || workspace_bytes < need || !aligned16(workspace)) return CKV_ERR_WORKSPACE;
+  DecodeArgs a{};
+  a.views = views_dev; a.q = q; a.out = out;
+  a.partial = static_cast<float*>(workspace);
+  a.Bz = Bz; a.H = H; a.G = G;
+  decode_plan(Bz, H, dtype, max_len, 0, G, D, &a.n_splits, &a.span);
+  a.max_len = max_len;
+  a.scale = scale;
+  a.k_pages = k_pages; a.v_pages = v_pages; a.logdeg_pages = logdeg_pages; a.page_shift = shift;
+  a.k_new = k_new; a.v_new = v_new;
+  a.k_pages_w = k_pages; a.v_pages_w = v_pages; a.deg_pages_w = deg_pages; a.logdeg_pages_w = logdeg_pages;
+  return launch_decode_paged(a, static_cast<cudaStream_t>(cuda_stream)) == cudaSuccess ? CKV_OK : CKV_ERR_CUDA;
+}
+
 }  // extern "C"

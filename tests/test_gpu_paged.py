@@ -265,3 +265,65 @@ def test_compress_paged_argument_checks():
     assert call(ws_bytes=64) == 4                                                     # workspace too small
     out_len, rounds, n_scratch, in_scratch, kept = b.pages_plan(1000, p, 64)
     assert (out_len, rounds, n_scratch, in_scratch, kept) == (500, 1, 8, True, 8)
+
+
+# ----------------------------------------------------------------------------- append + attention in one launch
+
+@pytest.mark.parametrize("P,G,H,lens", [(64, 4, 2, [0, 1, 63, 64, 65, 1000, 4100, 2500, 127]), (128, 8, 1, [20000]),
+                                        (32, 1, 8, [9000, 31, 32]), (256, 4, 8, [16415])])
+def test_decode_append_attn_paged(P, G, H, lens):
+    """One decoding step of Algorithm 1 in one launch: the new token of every sequence lands in slot len of its pages
+    with degree 1, and Eq. 3 runs over len + 1 tokens.  By definition: append, then the oracle's attention over the
+    gathered sequence.  Several steps in a row (the lengths cross page and tile boundaries); the pages must end up
+    exactly as a separate append would leave them, and pages of other sequences untouched."""
+    from paper_2506_11418_b200 import binding as b
+    D, steps = 128, 3
+    n_blocks = [(n + steps + P - 1) // P for n in lens]
+    pool = sum(n_blocks) + 5
+    kp, vp, dp, lp = make_pool(pool, H, P, D, seed=21)
+    perm = torch.randperm(pool, generator=torch.Generator().manual_seed(4)).to(torch.int32)
+    tables, off = [], 0
+    ref = []   # per sequence: K, V [H, n, D] float64, deg [H, n]
+    for i, n in enumerate(lens):
+        tab = perm[off:off + n_blocks[i]].to(DEV)
+        off += n_blocks[i]
+        tables.append(tab)
+        if n > 0:
+            K = synth.ar1_keys(1, H, n, D, (0.7, 0.95), 0.5, seed=80 + i, dtype="bf16", device=DEV)[0]
+            V = synth.normal_values(1, H, n, D, seed=80 + i, dtype="bf16", device=DEV)[0]
+            deg = synth.random_degrees((H,), n, 3 * n, seed=80 + i).to(DEV)
+            b.pages_scatter(tab, n, K, V, deg, kp, vp, dp, lp)
+            ref.append([PU.to_np64(K), PU.to_np64(V), deg.cpu().numpy().astype(np.int64)])
+        else:
+            ref.append([np.zeros((H, 0, D)), np.zeros((H, 0, D)), np.zeros((H, 0), dtype=np.int64)])
+    idle = perm[off:].long()
+    idle_before = (kp[idle].clone(), vp[idle].clone(), dp[idle].clone())
+    scale = 1.0 / math.sqrt(D)
+    cur = list(lens)
+    for step in range(steps):
+        kn = synth.ar1_keys(1, len(lens) * H, 1, D, (0.7, 0.95), 0.5, seed=900 + step, dtype="bf16", device=DEV).view(len(lens), H, D).contiguous()
+        vn = synth.normal_values(1, len(lens) * H, 1, D, seed=900 + step, dtype="bf16", device=DEV).view(len(lens), H, D).contiguous()
+        q = synth.queries(len(lens), H * G, D, seed=950 + step, dtype="bf16", device=DEV)
+        out = torch.full_like(q, 5.0)
+        max_len = max(cur) + 1
+        ws = torch.empty(b.decode_workspace_bytes(len(lens), H, G, D, max_len), dtype=torch.uint8, device=DEV)
+        b.decode_append_attn_paged(b.paged_views(tables, cur, DEV), kp, vp, dp, lp, H, G, kn, vn, q, out, scale, max_len, ws)
+        torch.cuda.synchronize()
+        results = []
+        for i in range(len(lens)):
+            ref[i][0] = np.concatenate([ref[i][0], PU.to_np64(kn[i])[:, None, :]], axis=1)
+            ref[i][1] = np.concatenate([ref[i][1], PU.to_np64(vn[i])[:, None, :]], axis=1)
+            ref[i][2] = np.concatenate([ref[i][2], np.ones((H, 1), dtype=np.int64)], axis=1)
+            cur[i] += 1
+            results.append(PU.check_attention(PU.to_np64(out[i]), PU.to_np64(q[i]), ref[i][0], ref[i][1], ref[i][2], scale, "bf16",
+                                              f"step {step}, sequence {i} (len {cur[i]})"))
+        PU.summarize_attention(results, f"append + attention, page {P}, step {step}")
+    # the pages hold what a separate append would have written
+    kpn, vpn, dpn, lpn = PU.to_np64(kp), PU.to_np64(vp), dp.cpu().numpy().astype(np.int64), lp.cpu().numpy().astype(np.float64)
+    for i, n in enumerate(cur):
+        tab = tables[i].cpu().numpy()
+        np.testing.assert_array_equal(O.gather_pages(kpn, tab, n), ref[i][0])
+        np.testing.assert_array_equal(O.gather_pages(vpn, tab, n), ref[i][1])
+        np.testing.assert_array_equal(O.gather_pages(dpn, tab, n), ref[i][2])
+        np.testing.assert_allclose(O.gather_pages(lpn, tab, n), np.log(ref[i][2].astype(np.float64)), rtol=1e-6, atol=1e-7)
+    assert torch.equal(kp[idle], idle_before[0]) and torch.equal(vp[idle], idle_before[1]) and torch.equal(dp[idle], idle_before[2])
