@@ -383,6 +383,8 @@ def run_gpu(args):
         extra["compress_variants"] = bench_compress_variants(b, synth, dev, K, V, peak, args.layers == 0)
         extra["recluster"] = bench_recluster(b, synth, dev, K, V)
         extra["no_chunk"] = bench_no_chunk(b, synth, dev, K, V, peaks, args.layers == 0)
+        extra["paged_compress"] = bench_paged_compress(b, synth, dev, K, V, peak)
+        targets["paged_compress_ratio1"] = {k: extra["paged_compress"]["chunk64 ratio1"][k] for k in ("ms", "frac_of_peak", "pages_freed")}
         cv = extra["compress_variants"]
         pick = lambda name: {k: cv[name][k] for k in ("ms", "frac_of_peak", "gbs", "moved_gb", "frac_on_moved_bytes")} if name in cv else None
         targets["chunk256_ratio1"] = pick("chunk256 ratio1")
@@ -802,8 +804,71 @@ def bench_decode_paged(b, synth, dev, peak_gbs):
     torch.cuda.synchronize()
     us = 1e3 * t0.elapsed_time(t1) / iters
     nbytes = decode_bytes(Bz * H * slots, D, 2)
-    return {"slots": slots, "page_tokens": P, "us_per_layer_step": us, "gbs": nbytes / (us * 1e-6) / 1e9,
-            "frac_of_peak": nbytes / (us * 1e-6) / 1e9 / peak_gbs}
+    res = {"slots": slots, "page_tokens": P, "us_per_layer_step": us, "gbs": nbytes / (us * 1e-6) / 1e9,
+           "frac_of_peak": nbytes / (us * 1e-6) / 1e9 / peak_gbs}
+    # the same step with the new token appended inside the launch (slot `slots - 1` is rewritten every time)
+    dp = torch.ones((pool, H, P), dtype=torch.int32, device=dev)
+    views1 = b.paged_views(tables, [slots - 1] * Bz, dev)
+    kn = torch.randn((Bz, H, D), device=dev, generator=g).to(torch.bfloat16)
+    vn = torch.randn((Bz, H, D), device=dev, generator=g).to(torch.bfloat16)
+    for _ in range(5):
+        b.decode_append_attn_paged(views1, kp, vp, dp, lp, H, G, kn, vn, q, out, scale, slots, ws)
+    torch.cuda.synchronize()
+    t0.record()
+    for _ in range(iters):
+        b.decode_append_attn_paged(views1, kp, vp, dp, lp, H, G, kn, vn, q, out, scale, slots, ws)
+    t1.record()
+    torch.cuda.synchronize()
+    us2 = 1e3 * t0.elapsed_time(t1) / iters
+    res["append_and_attend_us_per_layer_step"] = us2
+    res["append_and_attend_frac_of_peak"] = nbytes / (us2 * 1e-6) / 1e9 / peak_gbs
+    return res
+
+
+def bench_paged_compress(b, synth, dev, K, V, peak_gbs, page_tokens=64):
+    """ckv_compress_paged on the benchmark workload held in 64-token pages scattered over per-layer pools: one round at
+    ratio 1 (the timed step's compression, without leaving the pages) and the paper's schedule to 25 %, against the
+    gather -> ckv_compress_prefill -> scatter route."""
+    import torch
+    L, H, s, D = K.shape
+    P = page_tokens
+    own = s // P
+    res = {}
+    paper = dict(n_sink=16, n_recent=64, n_rounds_max=16, r_init=0.8, r_decay=0.2, r_min=0.2)
+    for name, p in (("chunk64 ratio1", b.Params(chunk=64, n_sink=0, n_recent=0, n_rounds_max=1, r_init=1.0, r_decay=0.0, r_min=1.0)),
+                    ("chunk64 paper schedule to 25%", b.Params(chunk=64, budget=s // 4, **paper))):
+        out_len, rounds, n_scratch, in_scratch, kept = b.pages_plan(s, p, P)
+        n_pages = own + n_scratch
+        perm = torch.randperm(n_pages, generator=torch.Generator().manual_seed(5)).to(torch.int32).to(dev)
+        table, scratch = perm[:own].contiguous(), perm[own:].contiguous()
+        pools = []
+        for l in range(L):
+            kp = torch.empty((n_pages, H, P, D), dtype=torch.bfloat16, device=dev)
+            vp = torch.empty_like(kp)
+            dp = torch.ones((n_pages, H, P), dtype=torch.int32, device=dev)
+            lp = torch.zeros((n_pages, H, P), dtype=torch.float32, device=dev)
+            b.pages_scatter(table, s, K[l], V[l], None, kp, vp, dp, lp)
+            pools.append((kp, vp, dp, lp))
+        ws = torch.empty(b.paged_workspace_bytes(L, H, D, torch.bfloat16, s, p), dtype=torch.uint8, device=dev)
+        # the call overwrites its source pages, which does not change what a repeated call costs
+        for _ in range(2):
+            b.compress_paged(pools, table, s, False, scratch, p, ws)
+        torch.cuda.synchronize()
+        iters = 5
+        t0, t1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        t0.record()
+        for _ in range(iters):
+            b.compress_paged(pools, table, s, False, scratch, p, ws)
+        t1.record()
+        torch.cuda.synchronize()
+        ms = t0.elapsed_time(t1) / iters
+        nbytes = schedule_bytes(L, H, s, out_len, D, 2)
+        res[name] = {"page_tokens": P, "seq": s, "out_len": out_len, "rounds": rounds, "ms": ms, "gbs": nbytes / (ms * 1e-3) / 1e9,
+                     "frac_of_peak": nbytes / (ms * 1e-3) / 1e9 / peak_gbs, "pages_kept": kept, "pages_freed": own - kept,
+                     "status": b.workspace_status(ws)}
+        del pools, ws
+        torch.cuda.empty_cache()
+    return res
 
 
 def bench_decode_cfg4(b, synth, dev, peak_gbs, steps=256):
