@@ -926,6 +926,40 @@ def bench_decode_cfg4(b, synth, dev, peak_gbs, steps=256):
     return res
 
 
+def run_profile_case(name):
+    """A small stand-alone case for a profiler capture (a few launches of one kernel on a 4-layer cut of a workload,
+    inputs larger than L2, a few GB on the device at most).  Prints nothing that is a benchmark number."""
+    import torch
+
+    from paper_2506_11418_b200 import binding as b, synth
+    dev = torch.device("cuda", 0)
+    torch.cuda.set_device(0)
+    cases = {
+        # two ratio-1 rounds in one pass: 4 layers x 8 heads x 131072 tokens (2 GiB in)
+        "two_rounds_128k": ("llama8b_128k", dict(chunk=64, n_sink=0, n_recent=0, n_rounds_max=2, r_init=1.0, r_decay=0.0, r_min=1.0)),
+        # one ratio-1 round at chunk 64 / 128 / 256: 4 layers x 8 heads x 32768 tokens (512 MiB in)
+        "one_round_32k_chunk64": ("llama8b_32k", dict(chunk=64, n_sink=0, n_recent=0, n_rounds_max=1, r_init=1.0, r_decay=0.0, r_min=1.0)),
+        "one_round_32k_chunk128": ("llama8b_32k", dict(chunk=128, n_sink=0, n_recent=0, n_rounds_max=1, r_init=1.0, r_decay=0.0, r_min=1.0)),
+        "one_round_32k_chunk256": ("llama8b_32k", dict(chunk=256, n_sink=0, n_recent=0, n_rounds_max=1, r_init=1.0, r_decay=0.0, r_min=1.0)),
+        "ranked_round_32k_chunk256": ("llama8b_32k", dict(chunk=256, n_sink=16, n_recent=64, n_rounds_max=1, r_init=0.8, r_decay=0.0, r_min=0.8)),
+    }
+    if name not in cases:
+        raise SystemExit(f"unknown profile case {name!r}; known: {sorted(cases)}")
+    workload, kw = cases[name]
+    cfg = synth.CONFIGS[workload]
+    L, H, s, D = 4, cfg["H"], cfg["s"], cfg["d"]
+    K = synth.ar1_keys(L, H, s, D, cfg["rho"], cfg["mean_std"], seed=cfg["seed"], dtype="bf16", device=dev)
+    V = synth.normal_values(L, H, s, D, seed=cfg["seed"], dtype="bf16", device=dev)
+    p = b.Params(**kw)
+    src = b.Cache(K, V, None, None, s)
+    out_len, rounds, cap = b.compress_plan(s, p)
+    dst = b.Cache.empty(L, H, cap, D, K.dtype, dev)
+    ws = torch.empty(b.workspace_bytes(src, p), dtype=torch.uint8, device=dev)
+    for _ in range(3):
+        b.compress_prefill(src, dst, p, ws)
+    print(json.dumps({"profile_case": name, "layers": L, "seq": s, "out_len": out_len, "rounds": rounds, "status": b.workspace_status(ws)}))
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -939,7 +973,11 @@ def main():
     ap.add_argument("--skip-variants", action="store_true")
     ap.add_argument("--skip-serving", action="store_true")
     ap.add_argument("--serving-steps", type=int, default=1024, help="lock-step decode steps of the serving-mix workload (its stated size: 1024)")
+    ap.add_argument("--profile-case", default=None, help="run one small named case three times and exit (for ncu captures)")
     args = ap.parse_args()
+    if args.profile_case:
+        run_profile_case(args.profile_case)
+        return
     if args.steps is None:
         args.steps = 3 if args.impl == "reference" else 200
     if args.impl == "reference":
