@@ -220,11 +220,12 @@ cudaError_t run_round(const RoundPlan& rp, const Buf& src, const Buf& dst, int L
   // bf16: the full chunks of chunk 64 go to the warp-per-chunk kernel, those of chunk 256 to the tcgen05 kernel, chunk 128
   // and every shorter last chunk to the tile kernel; everything else runs on the general kernel
   auto launch_pass = [&](RoundArgs x) -> cudaError_t {
-    const bool fast = round_fast_supported(x, dtype, D), umma = !fast && round_umma_supported(x, dtype, D);
-    if (fast || umma) {
+    const bool fast = round_fast_supported(x, dtype, D), group = !fast && round_group_supported(x, dtype, D);
+    const bool umma = !fast && !group && round_umma_supported(x, dtype, D);
+    if (fast || group || umma) {
       const int64_t n_full = (rp.hi - rp.lo) / chunk;
       if (!fast && first_chunk > 0) return cudaErrorInvalidValue;
-      cudaError_t err = fast ? launch_round_fast(x, n_full, st) : launch_round_umma(x, n_full, st);
+      cudaError_t err = fast ? launch_round_fast(x, n_full, st) : (group ? launch_round_group(x, n_full, st) : launch_round_umma(x, n_full, st));
       if (err != cudaSuccess || rp.n_chunks == n_full) return err;
       x.chunk_first = (int32_t)n_full;
       x.n_launch = 1;

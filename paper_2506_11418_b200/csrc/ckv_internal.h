@@ -209,6 +209,9 @@ cudaError_t launch_bsm_merge(const RoundArgs& a, void* scratch, cudaStream_t st)
 // 2 * units chunks of every slab; assign2 / stride2: the second round's slot map when a.assign is given
 bool round_fused2_supported(int dtype, int D, int chunk);
 cudaError_t launch_round_fused2(const RoundArgs& a, int64_t units, int32_t* assign2, int64_t stride2, cudaStream_t st);
+// chunk 128 / 256 in the modes that merge: groups of warps per chunk, warp-level tensor-core matching and merge
+bool round_group_supported(const RoundArgs& a, int dtype, int D);
+cudaError_t launch_round_group(const RoundArgs& a, int64_t n_full, cudaStream_t st);
 bool round_tile_supported(const RoundArgs& a, int dtype, int D);
 cudaError_t launch_round_tile(const RoundArgs& a, cudaStream_t st);
 
