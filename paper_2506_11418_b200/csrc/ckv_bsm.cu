@@ -51,7 +51,8 @@ constexpr int kBPart = kBSteps * 2 * kBHalf;  // bytes of one column half of the
 constexpr int oBInv = oBB + 2 * kBPart;
 constexpr int oBBar = oBInv + kBInvSlots * kBN * 4;
 constexpr int oBPart = oBBar + 256;
-constexpr int oBTmem = oBPart + kBM * 4 * 8;
+constexpr int oBRowMax = oBPart + kBM * 4 * 8;  // float [kBM]: every row's running maximum over all column quarters
+constexpr int oBTmem = oBRowMax + kBM * 4;
 constexpr int kBBytes = oBTmem + 16;
 
 struct BsmArgs {
@@ -149,16 +150,52 @@ __device__ __forceinline__ float max3(float a, float b, float c) {
   return d;
 }
 
+// Bounded wait for the consumer warps: sixteen warps polling one barrier back to back would take issue slots from the
+// warps that feed the tensor core, so a poll that fails is followed by a short sleep at once.
+__device__ __forceinline__ bool mbar_wait_sleeping(uint32_t bar, uint32_t parity) {
+  for (uint32_t i = 0; i < kSpinLimit; ++i) {
+    if (mbar_try_wait(bar, parity)) return true;
+    __nanosleep(i < 8 ? 100 : 400);
+  }
+  return false;
+}
+
+// max for floats in shared memory (order-preserving views of the bit pattern: as int for v >= 0, as unsigned for v < 0)
+__device__ __forceinline__ void atomic_max_float(float* addr, float v) {
+  if (v >= 0.f)
+    atomicMax(reinterpret_cast<int*>(addr), __float_as_int(v));
+  else
+    atomicMin(reinterpret_cast<unsigned*>(addr), __float_as_uint(v));
+}
+
 // Running row argmax over 64 accumulator columns of one tensor-memory lane per thread: dot products scaled by 1 / |b|.
-// The running maximum rarely moves once a few tiles are in, so the common path is one maximum per sixteen columns and
-// one warp vote; only when some lane has a new maximum does the warp look for its column (the lowest one that holds the
-// maximum: the lowest B position wins ties; an equal value later on never replaces the running one).
+// Four warps share a row (one per quarter of a step's columns); `shared_max` is the row's running maximum over all of
+// them, so that a warp whose columns never hold the row's good matches still knows what it has to beat.
+// Sixteen columns at a time.  First a bound that needs no scaling: the largest raw dot product of the sixteen times the
+// largest 1 / |b| among them (ginv) is at least every scaled value (fp32 multiplication is monotone), so if that stays
+// below the row's maximum in every lane of the warp, the group cannot hold the argmax and is skipped -- the common case
+// once the first step is in, because an A token's good matches sit in a few groups near it.  Otherwise: scale, one
+// maximum per sixteen columns and one warp vote; only when some lane reaches its row's maximum does the warp look for
+// the column (the lowest one that holds the group's maximum; the lowest B position wins ties, also against the
+// running one).  What a warp keeps is the argmax over its own columns that can still be the row's: the final
+// combination over the four quarters takes the highest value, lowest position.
 template <bool RAGGED>
-__device__ __forceinline__ void argmax_64(const uint32_t (&r)[2][32], const float* invb, int col0, int nB, float& bv, int& bi) {
+__device__ __forceinline__ void argmax_64(const uint32_t (&r)[2][32], const float* invb, const float (&ginv)[4], int col0, int nB,
+                                          float& bv, int& bi, float* shared_max) {
+  float thr = fmaxf(bv, *shared_max);  // (a stale value is only a weaker threshold)
 #pragma unroll
   for (int h = 0; h < 2; ++h) {
 #pragma unroll
     for (int g = 0; g < 32; g += 16) {
+      if (!RAGGED) {  // (the last step's columns past the end have no defined 1 / |b|: no shortcut there)
+        float d[16];
+#pragma unroll
+        for (int e = 0; e < 16; ++e) d[e] = __uint_as_float(r[h][g + e]);
+        const float rm = max3(max3(max3(d[0], d[1], d[2]), max3(d[3], d[4], d[5]), max3(d[6], d[7], d[8])),
+                              max3(max3(d[9], d[10], d[11]), max3(d[12], d[13], d[14]), d[15]), 0.f);
+        // rm >= 0 by the last operand: a group of negative dot products is bounded by 0
+        if (!__any_sync(0xffffffffu, rm * ginv[2 * h + (g >> 4)] >= thr)) continue;
+      }
       float sv[16];
 #pragma unroll
       for (int e4 = 0; e4 < 16; e4 += 4) {
@@ -173,13 +210,15 @@ __device__ __forceinline__ void argmax_64(const uint32_t (&r)[2][32], const floa
       }
       const float gm = max3(max3(max3(sv[0], sv[1], sv[2]), max3(sv[3], sv[4], sv[5]), max3(sv[6], sv[7], sv[8])),
                             max3(max3(sv[9], sv[10], sv[11]), max3(sv[12], sv[13], sv[14]), sv[15]), -INFINITY);
-      if (__any_sync(0xffffffffu, gm > bv)) {
+      if (__any_sync(0xffffffffu, gm >= thr)) {
         int idx = 15;
 #pragma unroll
         for (int e = 14; e >= 0; --e) idx = sv[e] == gm ? e : idx;
-        if (gm > bv) {
+        if (gm >= thr && (gm > bv || (gm == bv && col + idx < bi))) {  // the steps are not visited in order: ties by position
           bv = gm;
           bi = col + idx;
+          thr = gm;
+          atomic_max_float(shared_max, gm);
         }
       }
     }
@@ -219,6 +258,15 @@ __global__ void __launch_bounds__(kBThreads, 1) bsm_match_kernel(const __grid_co
   tc_fence_after();
   const uint32_t tmem = *reinterpret_cast<volatile uint32_t*>(smem + oBTmem);
   bool failed = false;
+  // The B steps are visited starting with the one that holds this tile's own neighbourhood (B tokens of the same
+  // positions as its A tokens) and wrapping around: key similarity decays with distance (the paper's Observations 1 and
+  // 2), so the running maxima are close to final after the first step and the bound test of the argmax skips nearly
+  // everything that follows.  The result does not depend on the order (ties go to the lowest B position explicitly).
+  const int t_first = min(atile * (kBM / kBN), n_steps - 1);
+  auto step_of = [&](int t) {
+    const int x = t_first + t;
+    return x >= n_steps ? x - n_steps : x;
+  };
 
   if (warp == kBConsumers) {
     // ------------------------------------------------------------------ TMA warp: the A blocks once, then the B steps
@@ -237,15 +285,15 @@ __global__ void __launch_bounds__(kBThreads, 1) bsm_match_kernel(const __grid_co
         for (int hf = 0; hf < 2; ++hf) {  // B tokens t * 256 + 128 hf .. + 127 (zero-filled past the end)
           const uint32_t dst = s_base + oBB + (uint32_t)(2 * slot + hf) * kBHalf;
           mbar_arrive_expect_tx(bar_full(2 * slot + hf), 2 * kBHalf);
-          tma_load_4d(dst, &tm_b, 0, 0, t * kBN + hf * kBT, lh, bar_full(2 * slot + hf));
-          tma_load_4d(dst + kBPart, &tm_b, 64, 0, t * kBN + hf * kBT, lh, bar_full(2 * slot + hf));
+          tma_load_4d(dst, &tm_b, 0, 0, step_of(t) * kBN + hf * kBT, lh, bar_full(2 * slot + hf));
+          tma_load_4d(dst + kBPart, &tm_b, 64, 0, step_of(t) * kBN + hf * kBT, lh, bar_full(2 * slot + hf));
         }
         // The slice slot of step t was last read for step t - 4; this fetch runs after the MMAs of step t - 2 completed,
         // which were issued after every consumer warp had copied the accumulators of step t - 3 to registers, and a warp
         // does that only after its argmax over step t - 4.
         const int is = t % kBInvSlots;
         mbar_arrive_expect_tx(bar_inv(is), kBN * 4);
-        bulk_load(s_base + oBInv + (uint32_t)is * kBN * 4, a.inv_b + (int64_t)lh * a.inv_stride + (int64_t)t * kBN, kBN * 4, bar_inv(is));
+        bulk_load(s_base + oBInv + (uint32_t)is * kBN * 4, a.inv_b + (int64_t)lh * a.inv_stride + (int64_t)step_of(t) * kBN, kBN * 4, bar_inv(is));
       }
     }
   } else if (warp == kBConsumers + 1) {
@@ -285,17 +333,30 @@ __global__ void __launch_bounds__(kBThreads, 1) bsm_match_kernel(const __grid_co
     const int q = warp & 3, cq = warp >> 2;
     float bv[2] = {-INFINITY, -INFINITY};
     int bi[2] = {INT_MAX, INT_MAX};
+    float* row_max = reinterpret_cast<float*>(smem + oBRowMax);
+    if (tid < kBM) row_max[tid] = -INFINITY;
+    asm volatile("bar.sync 1, %0;" ::"n"(kBConsumers * 32) : "memory");
     for (int t = 0; t < n_steps && !failed; ++t) {
       const int is = t % kBInvSlots;
-      if (!mbar_wait(bar_inv(is), (uint32_t)((t / kBInvSlots) & 1))) {
+      if (!mbar_wait_sleeping(bar_inv(is), (uint32_t)((t / kBInvSlots) & 1))) {
         failed = true;
         break;
       }
       const float* invb = reinterpret_cast<const float*>(smem + oBInv + is * kBN * 4) + 64 * cq;
-      const int col0 = t * kBN + 64 * cq;
+      const int col0 = step_of(t) * kBN + 64 * cq;
+      // the largest 1 / |b| of each of this warp's four groups of sixteen columns (eight lanes x two values per group)
+      float ginv[4];
+      {
+        const float2 iv = *reinterpret_cast<const float2*>(invb + 2 * lane);
+        float gx = fmaxf(iv.x, iv.y);
+#pragma unroll
+        for (int o = 1; o <= 4; o <<= 1) gx = fmaxf(gx, __shfl_xor_sync(0xffffffffu, gx, o));
+#pragma unroll
+        for (int k = 0; k < 4; ++k) ginv[k] = __shfl_sync(0xffffffffu, gx, 8 * k);
+      }
 #pragma unroll
       for (int m = 0; m < 2; ++m) {
-        if (!mbar_wait(bar_tfull(m), (uint32_t)(t & 1))) {
+        if (!mbar_wait_sleeping(bar_tfull(m), (uint32_t)(t & 1))) {
           failed = true;
           break;
         }
@@ -310,9 +371,9 @@ __global__ void __launch_bounds__(kBThreads, 1) bsm_match_kernel(const __grid_co
         __syncwarp();
         if (lane == 0) mbar_arrive(bar_tempty(m));
         if (col0 + 64 <= a.nB) {  // only the last step can hold columns that are not B tokens
-          argmax_64<false>(r, invb, col0, a.nB, bv[m], bi[m]);
+          argmax_64<false>(r, invb, ginv, col0, a.nB, bv[m], bi[m], row_max + kBT * m + 32 * q + lane);
         } else {
-          argmax_64<true>(r, invb, col0, a.nB, bv[m], bi[m]);
+          argmax_64<true>(r, invb, ginv, col0, a.nB, bv[m], bi[m], row_max + kBT * m + 32 * q + lane);
         }
       }
     }
