@@ -8,8 +8,10 @@
 //                       warp issues tcgen05.mma 128 x 256 x 16 (the widest shape of one CTA: the least shared-memory
 //                       operand traffic per flop) for row block 0, then row block 1, each into its own 256 columns of
 //                       tensor memory; sixteen consumer warps copy an accumulator to registers (tcgen05.ld), hand it back
-//                       to the tensor core at once, scale by 1 / |b| and keep a running row argmax (lowest B position on
-//                       ties); the edge (cosine, target) is written at the end
+//                       to the tensor core at once and keep a running row argmax of dot / |b| (lowest B position on
+//                       ties).  The steps are visited from the tile's own neighbourhood outwards, the four warps of a row
+//                       share its running maximum, and groups of sixteen columns whose unscaled bound stays below it are
+//                       skipped; the edge (cosine, target) is written at the end
 //   select_kernel       the M best edges of the head (shared with the chunked path)
 //   bsm_prepare_kernel  prefix counts of the selected edges (output slots) and the number of members per B token
 //   bsm_prepare_kernel  also lists the members of every B token
