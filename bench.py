@@ -386,7 +386,13 @@ def run_gpu(args):
         extra["paged_compress"] = bench_paged_compress(b, synth, dev, K, V, peak)
         targets["paged_compress_ratio1"] = {k: extra["paged_compress"]["chunk64 ratio1"][k] for k in ("ms", "frac_of_peak", "pages_freed")}
         cv = extra["compress_variants"]
-        pick = lambda name: {k: cv[name][k] for k in ("ms", "frac_of_peak", "gbs", "moved_gb", "frac_on_moved_bytes")} if name in cv else None
+        def pick(name):
+            if name not in cv:
+                return None
+            row = {k: cv[name][k] for k in ("ms", "frac_of_peak", "gbs", "moved_gb", "frac_on_moved_bytes")}
+            row["frac_of_nominal_8tbs"] = row["gbs"] / 8000.0
+            return row
+        targets["chunk128_ratio1"] = pick("chunk128 ratio1")
         targets["chunk256_ratio1"] = pick("chunk256 ratio1")
         targets["chunk256_ratio0.8_ranked_per_head"] = pick("chunk256 ratio0.8 ranked per head")
         targets["chunk256_paper_schedule_to_25pct"] = pick("chunk256 paper schedule to 25%")
@@ -408,6 +414,7 @@ def run_gpu(args):
         d4 = extra["decode_cfg4"]
         targets["cfg4_decode_batch32"] = {"compressed_us_per_layer_step": d4["compressed"]["us_per_layer_step"],
                                           "compressed_frac_of_peak": d4["compressed"]["frac_of_peak"],
+                                          "compressed_frac_of_nominal_8tbs": d4["compressed"]["gbs"] / 8000.0,
                                           "uncompressed_us_per_layer_step": d4["uncompressed"]["us_per_layer_step"],
                                           "speedup_vs_uncompressed": d4["speedup"], "steps": d4["compressed"]["steps"],
                                           "paged_frac_of_peak": extra["decode_cfg4_paged"]["frac_of_peak"]}
