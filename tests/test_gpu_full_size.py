@@ -387,3 +387,54 @@ def test_no_chunking_128k_sampled_rows():
         counts = np.bincount(asg[0::2], minlength=s // 2) + 1
         np.testing.assert_array_equal(dst.deg[0, h, :s // 2].cpu().numpy(), counts)
     torch.cuda.empty_cache()
+
+
+def window_matches_full_run(K, V, p, dst, assign, t0, t1, out0, dtype="bf16"):
+    """With every edge merged (or ranked per chunk) a chunk's clusters depend on that chunk alone, so source tokens
+    [t0, t1) (t0 on a boundary of every round's chunks) clustered on their own must reproduce rows out0 ... of the full
+    run bit for bit; the window's own run is checked against the oracle round by round."""
+    Kw, Vw = K[:, :, t0:t1].contiguous(), V[:, :, t0:t1].contiguous()
+    st = TC.multi_round_check(Kw, Vw, dtype, p)
+    d1 = st["dst"]
+    n = d1.len
+    assert torch.equal(d1.k[0, 0, :n], dst.k[0, 0, out0:out0 + n]) and torch.equal(d1.v[0, 0, :n], dst.v[0, 0, out0:out0 + n])
+    assert torch.equal(d1.deg[0, 0, :n], dst.deg[0, 0, out0:out0 + n])
+    assert torch.equal(st["assign"][0, 0] + out0, assign[0, 0, t0:t1])
+    return n
+
+
+def test_one_head_longer_than_four_gib():
+    """Maximum sizes: one (layer, head) of 2^24 + 202 tokens, whose keys alone take more than 4 GiB, so that row offsets
+    inside a single slab pass 2^31 and 2^32 bytes.  Windows around both marks and the ragged end are compared with the
+    same windows clustered alone (and those with the oracle); the degrees of the whole slab must sum to its length."""
+    need_free(40)
+    b = B()
+    s = (1 << 24) + 202
+    K = synth.ar1_keys(1, 1, s, 128, (0.9, 0.9), 0.5, seed=5, dtype="bf16", device=DEV)
+    V = synth.normal_values(1, 1, s, 128, seed=5, dtype="bf16", device=DEV)
+    marks = [(0, 2048), ((1 << 23) - 1024, (1 << 23) + 1024), ((1 << 24) - 2048, s)]
+    cases = [
+        (b.Params(chunk=64, n_sink=0, n_recent=0, n_rounds_max=1, r_init=1.0, r_decay=0.0, r_min=1.0), lambda t: t // 2),
+        (b.Params(chunk=64, n_sink=0, n_recent=0, n_rounds_max=2, r_init=1.0, r_decay=0.0, r_min=1.0), lambda t: t // 4),
+        (b.Params(chunk=256, n_sink=0, n_recent=0, n_rounds_max=1, r_init=1.0, r_decay=0.0, r_min=1.0), lambda t: t // 2),
+        (b.Params(chunk=64, n_sink=0, n_recent=0, n_rounds_max=1, r_init=0.5, r_decay=0.0, r_min=0.5, select=b.SELECT_CHUNK),
+         lambda t: t // 64 * 48),
+    ]
+    for p, out_of in cases:
+        dst, assign, rounds = TC.run_gpu_prefill(K, V, None, p, want_assign=True, cap_extra=0)
+        n = dst.len
+        assert int(dst.deg[0, 0, :n].sum(dtype=torch.int64)) == s and int(dst.deg[0, 0, :n].min()) >= 1
+        end = 0
+        for t0, t1 in marks:
+            end = out_of(t0) + window_matches_full_run(K, V, p, dst, assign, t0, t1, out_of(t0))
+        assert end == n  # the last window ends where the compressed slab ends
+        del dst, assign
+        torch.cuda.empty_cache()
+    # ranked over the whole head: nothing local to compare with, the invariants must still hold
+    p = b.Params(chunk=64, n_sink=16, n_recent=64, n_rounds_max=2, r_init=0.8, r_decay=0.2, r_min=0.2)
+    dst, assign, rounds = TC.run_gpu_prefill(K, V, None, p, want_assign=True, cap_extra=0)
+    n = dst.len
+    assert int(dst.deg[0, 0, :n].sum(dtype=torch.int64)) == s and int(dst.deg[0, 0, :n].min()) >= 1
+    assert int(assign[0, 0].min()) == 0 and int(assign[0, 0].max()) == n - 1
+    del dst, assign
+    torch.cuda.empty_cache()
