@@ -180,10 +180,17 @@ cudaError_t run_round(const RoundPlan& rp, const Buf& src, const Buf& dst, int L
     c.src_off = 0; c.dst_off = 0; c.count = rp.s_in;
     return launch_copy(c, dtype, D, st);
   }
-  c.src_off = 0; c.dst_off = 0; c.count = rp.lo;
-  if ((e = launch_copy(c, dtype, D, st)) != cudaSuccess) return e;
-  c.src_off = rp.hi; c.dst_off = rp.hi - rp.M; c.count = rp.s_in - rp.hi;
-  if ((e = launch_copy(c, dtype, D, st)) != cudaSuccess) return e;
+  // Sinks and recent tokens.  After an ordered kernel of this round they may run beside the kernels of the round (they
+  // touch rows no chunk owns, and every earlier round has completed by then); on their own they are ordered launches.
+  auto copy_edges = [&](bool beside) -> cudaError_t {
+    c.overlap = beside ? 1 : 0;
+    c.src_off = 0; c.dst_off = 0; c.count = rp.lo;
+    cudaError_t ce = launch_copy(c, dtype, D, st);
+    if (ce != cudaSuccess) return ce;
+    c.src_off = rp.hi; c.dst_off = rp.hi - rp.M; c.count = rp.s_in - rp.hi;
+    return launch_copy(c, dtype, D, st);
+  };
+  if (chunk == 0 && (e = copy_edges(false)) != cudaSuccess) return e;
 
   RoundArgs a{};
   a.k_src = src.k; a.v_src = src.v; a.deg_src = src.deg;
@@ -210,7 +217,7 @@ cudaError_t run_round(const RoundPlan& rp, const Buf& src, const Buf& dst, int L
   }
   a.chunk = chunk; a.n_chunks = rp.n_chunks;
   a.chunk_first = first_chunk; a.n_launch = rp.n_chunks - first_chunk;
-  if (a.n_launch <= 0) return cudaSuccess;
+  if (a.n_launch <= 0) return copy_edges(false);
   a.m_full = rp.m_full; a.m_tail = rp.m_tail;
   a.out_stride = chunk - rp.m_full;
   a.out_lo = rp.lo;
@@ -225,10 +232,14 @@ cudaError_t run_round(const RoundPlan& rp, const Buf& src, const Buf& dst, int L
     if (fast || group || umma) {
       const int64_t n_full = (rp.hi - rp.lo) / chunk;
       if (!fast && first_chunk > 0) return cudaErrorInvalidValue;
-      cudaError_t err = fast ? launch_round_fast(x, n_full, st) : (group ? launch_round_group(x, n_full, st) : launch_round_umma(x, n_full, st));
-      if (err != cudaSuccess || rp.n_chunks == n_full) return err;
-      x.chunk_first = (int32_t)n_full;
-      x.n_launch = 1;
+      if (n_full > first_chunk) {
+        cudaError_t err = fast ? launch_round_fast(x, n_full, st) : (group ? launch_round_group(x, n_full, st) : launch_round_umma(x, n_full, st));
+        if (err != cudaSuccess) return err;
+        x.overlap = 1;  // the shorter last chunk is nobody else's: it may run beside the full chunks just launched
+      }
+      if (rp.n_chunks == n_full) return cudaSuccess;
+      x.chunk_first = (int32_t)std::max<int64_t>(n_full, first_chunk);
+      x.n_launch = rp.n_chunks - x.chunk_first;
     }
     return round_tile_supported(x, dtype, D) ? launch_round_tile(x, st) : launch_round(x, dtype, D, st);
   };
@@ -245,7 +256,8 @@ cudaError_t run_round(const RoundPlan& rp, const Buf& src, const Buf& dst, int L
     if ((e = launch_select(s, st)) != cudaSuccess) return e;
   }
   a.mode = rp.mode;
-  return launch_pass(a);
+  if ((e = launch_pass(a)) != cudaSuccess) return e;
+  return copy_edges(true);  // (the pass above began with an ordered launch)
 }
 
 // Runs the planned rounds from `src` into `dst` (ping-pong through the workspace's tmp cache).

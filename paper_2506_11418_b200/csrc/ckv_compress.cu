@@ -245,6 +245,8 @@ __global__ void __launch_bounds__(kRoundThreads) round_kernel(const RoundArgs a)
 template <typename T, int D>
 __global__ void __launch_bounds__(256) copy_rows_kernel(const CopyArgs a) {
   constexpr int kVecPerRow = D * (int)sizeof(T) / 16;
+  if (!a.overlap) griddep_wait();
+  griddep_launch();
   const int lh = blockIdx.y;
   const int64_t nvec = a.count * kVecPerRow;
   const uint4* ks = reinterpret_cast<const uint4*>(reinterpret_cast<const T*>(a.k_src) + ((int64_t)lh * a.src_cap + a.src_off) * D);
@@ -263,6 +265,7 @@ __global__ void __launch_bounds__(256) copy_rows_kernel(const CopyArgs a) {
     if (a.logdeg_dst) a.logdeg_dst[di] = logf((float)dg);
     if (a.assign) a.assign[(int64_t)lh * a.assign_stride + a.src_off + i] = (int32_t)(a.dst_off + i);
   }
+  if (a.overlap) griddep_wait();
 }
 
 // Algorithm 1, decoding branch, K = [K, k], V = [V, v], N = [N, 1] for a batch of sequences in one launch: block
@@ -328,6 +331,8 @@ __global__ void __launch_bounds__(kSelThreads, 2) select_kernel(const SelectArgs
   __shared__ uint32_t hist[256];
   __shared__ uint32_t s_prefix, s_rem;
   __shared__ int warp_tot[kSelThreads / 32];
+  griddep_wait();
+  griddep_launch();
   const int tid = threadIdx.x, lane = tid & 31;
   const int lh = blockIdx.x;
   const int64_t n = a.edge_stride;
@@ -438,6 +443,8 @@ __global__ void __launch_bounds__(kSelThreads, 2) select_kernel(const SelectArgs
 
 __global__ void __launch_bounds__(256) compose_assign_kernel(int32_t* total, const int32_t* step, int64_t n_src,
                                                              int64_t step_stride) {
+  griddep_wait();
+  griddep_launch();
   const int lh = blockIdx.y;
   const int64_t stride = (int64_t)gridDim.x * blockDim.x;
   for (int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; i < n_src; i += stride) {
@@ -477,11 +484,8 @@ cudaError_t launch_copy(const CopyArgs& a, int dtype, int D, cudaStream_t st) {
   const int64_t nvec = a.count * (D * (dtype == 0 ? 4 : 2) / 16);
   const unsigned gx = (unsigned)std::min<int64_t>((nvec + 255) / 256, 1184);
   const dim3 grid(gx, (unsigned)a.LH);
-  if (dtype == 0)
-    copy_rows_kernel<float, 128><<<grid, 256, 0, st>>>(a);
-  else
-    copy_rows_kernel<__nv_bfloat16, 128><<<grid, 256, 0, st>>>(a);
-  return cudaGetLastError();
+  return dtype == 0 ? launch_dependent(copy_rows_kernel<float, 128>, grid, dim3(256), 0, st, a)
+                    : launch_dependent(copy_rows_kernel<__nv_bfloat16, 128>, grid, dim3(256), 0, st, a);
 }
 
 cudaError_t launch_append_batch(const AppendBatchArgs& a, int dtype, int D, cudaStream_t st) {
@@ -497,16 +501,14 @@ cudaError_t launch_append_batch(const AppendBatchArgs& a, int dtype, int D, cuda
 }
 
 cudaError_t launch_select(const SelectArgs& a, cudaStream_t st) {
-  select_kernel<<<(unsigned)a.LH, kSelThreads, 0, st>>>(a);
-  return cudaGetLastError();
+  return launch_dependent(select_kernel, dim3((unsigned)a.LH), dim3(kSelThreads), 0, st, a);
 }
 
 cudaError_t launch_compose_assign(int32_t* total, const int32_t* step, int64_t n_src, int64_t step_stride, int32_t LH,
                                   cudaStream_t st) {
   if (n_src <= 0) return cudaSuccess;
   const dim3 grid((unsigned)std::min<int64_t>((n_src + 255) / 256, 592), (unsigned)LH);
-  compose_assign_kernel<<<grid, 256, 0, st>>>(total, step, n_src, step_stride);
-  return cudaGetLastError();
+  return launch_dependent(compose_assign_kernel, grid, dim3(256), 0, st, total, step, n_src, step_stride);
 }
 
 }  // namespace ckv

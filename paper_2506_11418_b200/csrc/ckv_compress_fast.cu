@@ -89,6 +89,8 @@ template <int NW, bool HAS_DEG, int KIND, bool PAGED>
 __global__ void __launch_bounds__(NW * 32, 1)
 round_fast_kernel(const FastArgs a, const __grid_constant__ typename std::conditional<PAGED, PagedArgs, NoPages>::type pg) {
   extern __shared__ __align__(128) unsigned char smem[];
+  griddep_wait();    // ordered launch: everything ahead in the stream has completed
+  griddep_launch();  // the next launch may become resident as this grid's CTAs leave
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
   const int g = lane >> 2, t = lane & 3;
   constexpr int kStage = KIND == kFastMatch ? kTileBytes : kStageBytes;  // the matching alone stages no V tile
@@ -443,8 +445,7 @@ cudaError_t launch_fast_inst(const FastArgs& a, const PG& pg, cudaStream_t st) {
   const int64_t ctas = std::min<int64_t>(sm_count(), (a.n_items + NW - 1) / NW);
   cudaError_t e = cudaFuncSetAttribute(round_fast_kernel<NW, HAS_DEG, KIND, PAGED>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
   if (e != cudaSuccess) return e;
-  round_fast_kernel<NW, HAS_DEG, KIND, PAGED><<<(unsigned)ctas, NW * 32, smem, st>>>(a, pg);
-  return cudaGetLastError();
+  return launch_dependent(round_fast_kernel<NW, HAS_DEG, KIND, PAGED>, dim3((unsigned)ctas), dim3(NW * 32), smem, st, a, pg);
 }
 
 template <int NW, int KIND, bool PAGED, typename PG>

@@ -405,6 +405,8 @@ __global__ void __launch_bounds__(kFThreads, 1)
 round_fused2_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__ CUtensorMap tm_v,
                     const __grid_constant__ CUtensorMap tm_ko, const __grid_constant__ CUtensorMap tm_vo, const FusedArgs a) {
   extern __shared__ __align__(1024) unsigned char smem[];
+  griddep_wait();    // ordered launch: everything ahead in the stream has completed
+  griddep_launch();  // the next launch may become resident as this grid's CTAs leave
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
   const int grp = warp >> 1, w = warp & 1, gtid = 32 * w + lane, bar_id = 1 + grp;
   if ((smem_u32(smem) & 1023u) != 0u) {  // the swizzle pattern needs 1024-byte aligned tiles
@@ -582,8 +584,7 @@ cudaError_t launch_round_fused2(const RoundArgs& r, int64_t units, int32_t* assi
   cudaError_t e = cudaFuncSetAttribute(round_fused2_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
   if (e != cudaSuccess) return e;
   const int64_t ctas = std::min<int64_t>(sm_count(), (a.n_items + kFGroups - 1) / kFGroups);
-  round_fused2_kernel<<<(unsigned)ctas, kFThreads, smem, st>>>(tm_k, tm_v, tm_ko, tm_vo, a);
-  return cudaGetLastError();
+  return launch_dependent(round_fused2_kernel, dim3((unsigned)ctas), dim3(kFThreads), smem, st, tm_k, tm_v, tm_ko, tm_vo, a);
 }
 
 }  // namespace ckv

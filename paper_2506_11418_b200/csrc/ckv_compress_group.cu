@@ -311,6 +311,8 @@ round_group_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_consta
   using Cfg = GroupCfg<C>;
   constexpr int NA = Cfg::kNA, GW = Cfg::kGW, GT = GW * 32;
   extern __shared__ __align__(1024) unsigned char smem[];
+  griddep_wait();    // ordered launch: everything ahead in the stream has completed
+  griddep_launch();  // the next launch may become resident as this grid's CTAs leave
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
   const int grp = warp / GW, w = warp % GW, gtid = w * 32 + lane, bar_id = 1 + grp;
   if ((smem_u32(smem) & 1023u) != 0u) {  // the swizzle pattern needs 1024-byte aligned tiles
@@ -567,8 +569,7 @@ cudaError_t launch_group_c(const RoundArgs& a, int64_t n_full, cudaStream_t st) 
   auto kern = a.deg_src ? round_group_kernel<C, true> : round_group_kernel<C, false>;
   cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)Cfg::kSmem);
   if (e != cudaSuccess) return e;
-  kern<<<(unsigned)ctas, Cfg::kThreads, Cfg::kSmem, st>>>(tm_k, tm_v, tm_ko, tm_vo, a, (int)n_full);
-  return cudaGetLastError();
+  return launch_dependent(kern, dim3((unsigned)ctas), dim3(Cfg::kThreads), Cfg::kSmem, st, tm_k, tm_v, tm_ko, tm_vo, a, (int)n_full);
 }
 
 }  // namespace

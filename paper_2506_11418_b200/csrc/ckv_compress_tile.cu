@@ -113,6 +113,8 @@ __global__ void __launch_bounds__(TileCfg<C>::T, TileCfg<C>::kCtasPerSm) round_t
   constexpr int NK = Cfg::NK, NV = Cfg::NV, PK = Cfg::PK, PV = Cfg::PV;
   static_assert(PV == PK || PV == 0, "the V tile is fetched together with the K tile or at the start of its own item");
   extern __shared__ __align__(128) unsigned char smem[];
+  if (!a.overlap) griddep_wait();  // (an overlap launch waits at its end instead)
+  griddep_launch();
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const int g = lane >> 2, t = lane & 3;
   const int mt = warp % MT, ng = warp / MT;  // this warp's m tile and its column group / slice
@@ -479,6 +481,7 @@ __global__ void __launch_bounds__(TileCfg<C>::T, TileCfg<C>::kCtasPerSm) round_t
     }
     __syncthreads();  // S5: the tiles are free
   }
+  if (a.overlap) griddep_wait();  // this grid must not complete before the one it ran beside has
 }
 
 template <int C>
@@ -490,8 +493,7 @@ cudaError_t launch_tile_c(const RoundArgs& a, cudaStream_t st) {
   cudaError_t e = cudaFuncSetAttribute(round_tile_kernel<C>, cudaFuncAttributeMaxDynamicSharedMemorySize, Cfg::kBytes);
   if (e != cudaSuccess) return e;
   const int64_t ctas = std::min<int64_t>((int64_t)sm_count() * Cfg::kCtasPerSm, n_items);
-  round_tile_kernel<C><<<(unsigned)ctas, Cfg::T, Cfg::kBytes, st>>>(a);
-  return cudaGetLastError();
+  return launch_dependent(round_tile_kernel<C>, dim3((unsigned)ctas), dim3(Cfg::T), Cfg::kBytes, st, a);
 }
 
 }  // namespace

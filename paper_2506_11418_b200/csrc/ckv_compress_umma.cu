@@ -65,6 +65,8 @@ template <int C>
 __global__ void __launch_bounds__(kMThreads, 1)
 match_umma_kernel(const __grid_constant__ CUtensorMap tm_k, const RoundArgs a, const int n_full) {
   static_assert(C == 256 || C == 128, "chunk 256, or pairs of chunks of 128");
+  griddep_wait();    // ordered launch: everything ahead in the stream has completed
+  griddep_launch();  // the next launch may become resident as this grid's CTAs leave
   const int n_blk = C == 256 ? n_full : (n_full + 1) / 2;  // items per slab
   extern __shared__ unsigned char smem_raw[];
   unsigned char* smem = reinterpret_cast<unsigned char*>((reinterpret_cast<uintptr_t>(smem_raw) + kUAlign - 1) & ~(uintptr_t)(kUAlign - 1));
@@ -317,8 +319,7 @@ cudaError_t launch_round_umma(const RoundArgs& a, int64_t n_full, cudaStream_t s
   cudaError_t em = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)msmem);
   if (em != cudaSuccess) return em;
   const int64_t items = (a.chunk == kUC ? n_full : (n_full + 1) / 2) * a.LH;
-  kern<<<(unsigned)std::min<int64_t>(sm_count(), items), kMThreads, msmem, st>>>(tm_k, a, (int)n_full);
-  return cudaGetLastError();
+  return launch_dependent(kern, dim3((unsigned)std::min<int64_t>(sm_count(), items)), dim3(kMThreads), msmem, st, tm_k, a, (int)n_full);
 }
 
 }  // namespace ckv

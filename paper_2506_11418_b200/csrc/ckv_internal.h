@@ -43,6 +43,7 @@ struct RoundArgs {
   int64_t edge_stride;     // n_chunks * chunk / 2
   int32_t LH;
   int32_t* status;         // device word in the workspace: nonzero after a bounded wait gave up
+  int32_t overlap;         // 1: this launch depends on nothing the kernels since the last ordered launch write (see below)
 };
 
 // Copy `count` token rows (K, V, degree) of every slab from src_off to dst_off.
@@ -58,6 +59,7 @@ struct CopyArgs {
   int64_t assign_stride;
   int64_t src_cap, dst_cap, src_off, dst_off, count;
   int32_t LH;
+  int32_t overlap;         // 1: see RoundArgs::overlap
 };
 
 // One new token (degree 1) for each of up to kAppendBatchMax sequences: token b of k_new / v_new [LH, n_total, D] goes
@@ -165,6 +167,15 @@ inline int sm_count() {
 
 // Launch with programmatic stream serialization: the kernel may become resident while the kernel ahead of it
 // in the stream drains; it must call griddep_wait() before it touches anything that kernel produced.
+//
+// How the kernels of a clustering round use it.  An ORDERED kernel calls griddep_wait() and then griddep_launch() before
+// anything else: it starts after everything ahead of it has completed, and lets the next launch become resident as its
+// own CTAs leave.  A kernel launched with `overlap` = 1 (the shorter last chunk of a pass, the copies of sinks and recent
+// tokens) skips the wait at its start and calls griddep_wait() as its last statement instead: it runs beside the ordered
+// kernel ahead of it and beside other overlap launches in between, so it may neither read what those write nor write
+// what they read; because it cannot complete before its predecessor has, "the kernel ahead has completed" still means
+// "everything before it has completed" for whatever comes next.  The host sets overlap only after an ordered kernel
+// of the same round has been launched.
 template <typename... KArgs, typename... Args>
 inline cudaError_t launch_dependent(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t st,
                                     Args&&... args) {
