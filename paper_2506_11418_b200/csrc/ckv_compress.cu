@@ -326,8 +326,13 @@ __device__ __forceinline__ int block_exscan(int x, int* total, int* warp_tot) {
   return before + inc - x;
 }
 
+// STAGED: the head's keys are read from global memory once, into shared memory (one pad word per 32, so that both the
+// strided sweeps of the radix passes and the per-thread runs of the position pass are free of bank conflicts); otherwise
+// every pass reads them again.
+template <bool STAGED>
 __global__ void __launch_bounds__(kSelThreads, 2) select_kernel(const SelectArgs a) {
   static_assert(kSelThreads == 1024, "one warp total per lane in block_exscan");
+  extern __shared__ uint32_t s_keys[];
   __shared__ uint32_t hist[256];
   __shared__ uint32_t s_prefix, s_rem;
   __shared__ int warp_tot[kSelThreads / 32];
@@ -339,6 +344,16 @@ __global__ void __launch_bounds__(kSelThreads, 2) select_kernel(const SelectArgs
   const float* sim = a.edge_sim + (int64_t)lh * n;
   const int hc = a.chunk >> 1;
   const bool none = a.M <= 0;
+  if (STAGED) {
+    const int nn = (int)n;
+#pragma unroll 8
+    for (int i = tid; i < nn; i += kSelThreads) s_keys[i + (i >> 5)] = sim_key(sim[i]);
+    __syncthreads();
+  }
+  auto key_at = [&](int64_t i) -> uint32_t {
+    if (STAGED) return s_keys[(int)i + ((int)i >> 5)];
+    return sim_key(sim[i]);
+  };
 
   // ---- the key of the M-th best edge: 4 x 8-bit radix select from the top byte down
   uint32_t prefix = 0, mask = 0, rem = (uint32_t)a.M;
@@ -349,7 +364,7 @@ __global__ void __launch_bounds__(kSelThreads, 2) select_kernel(const SelectArgs
       for (int i = tid; i < 256; i += kSelThreads) hist[i] = 0;
       __syncthreads();
       for (int64_t i = tid; i < n_up; i += kSelThreads) {
-        const uint32_t key = i < n ? sim_key(sim[i]) : 0u;
+        const uint32_t key = i < n ? key_at(i) : 0u;
         const bool in = i < n && (key & mask) == prefix;
         const uint32_t bin = in ? ((key >> shift) & 255u) : 256u;
         if (pass == 3) {
@@ -407,7 +422,7 @@ __global__ void __launch_bounds__(kSelThreads, 2) select_kernel(const SelectArgs
     const int len = (int)max((int64_t)0, min((int64_t)run, n - first));
     unsigned long long gt_bits = 0ull, eq_bits = 0ull;
     for (int j = 0; j < len; ++j) {
-      const uint32_t key = sim_key(sim[first + j]);
+      const uint32_t key = key_at(first + j);
       if (!none && key > T) gt_bits |= 1ull << j;
       if (!none && key == T) eq_bits |= 1ull << j;
     }
@@ -501,7 +516,15 @@ cudaError_t launch_append_batch(const AppendBatchArgs& a, int dtype, int D, cuda
 }
 
 cudaError_t launch_select(const SelectArgs& a, cudaStream_t st) {
-  return launch_dependent(select_kernel, dim3((unsigned)a.LH), dim3(kSelThreads), 0, st, a);
+  // keys of up to 24576 edges per head stay in shared memory (two CTAs of 99 KiB per SM)
+  constexpr int64_t kStageMax = 24576;
+  if (a.edge_stride <= kStageMax) {
+    const size_t smem = (size_t)(a.edge_stride + a.edge_stride / 32 + 1) * 4;
+    cudaError_t e = set_smem(select_kernel<true>, (kStageMax + kStageMax / 32 + 1) * 4);
+    if (e != cudaSuccess) return e;
+    return launch_dependent(select_kernel<true>, dim3((unsigned)a.LH), dim3(kSelThreads), smem, st, a);
+  }
+  return launch_dependent(select_kernel<false>, dim3((unsigned)a.LH), dim3(kSelThreads), 0, st, a);
 }
 
 cudaError_t launch_compose_assign(int32_t* total, const int32_t* step, int64_t n_src, int64_t step_stride, int32_t LH,
