@@ -273,6 +273,8 @@ __global__ void __launch_bounds__(256) copy_rows_kernel(const CopyArgs a) {
 template <typename T, int D>
 __global__ void __launch_bounds__(256) append_batch_kernel(const __grid_constant__ AppendBatchArgs a) {
   constexpr int kVecPerRow = D * (int)sizeof(T) / 16;
+  griddep_wait();    // ordered launch: the kernel ahead may still be reading the slots this one fills
+  griddep_launch();
   const int lh = blockIdx.y;
   const int nvec = a.n * kVecPerRow;
   for (int i = blockIdx.x * blockDim.x + threadIdx.x; i < nvec; i += gridDim.x * blockDim.x) {
@@ -508,11 +510,8 @@ cudaError_t launch_append_batch(const AppendBatchArgs& a, int dtype, int D, cuda
   if (a.n <= 0) return cudaSuccess;
   const int nvec = a.n * (D * (dtype == 0 ? 4 : 2) / 16);
   const dim3 grid((unsigned)((nvec + 255) / 256), (unsigned)a.LH);
-  if (dtype == 0)
-    append_batch_kernel<float, 128><<<grid, 256, 0, st>>>(a);
-  else
-    append_batch_kernel<__nv_bfloat16, 128><<<grid, 256, 0, st>>>(a);
-  return cudaGetLastError();
+  return dtype == 0 ? launch_dependent(append_batch_kernel<float, 128>, grid, dim3(256), 0, st, a)
+                    : launch_dependent(append_batch_kernel<__nv_bfloat16, 128>, grid, dim3(256), 0, st, a);
 }
 
 cudaError_t launch_select(const SelectArgs& a, cudaStream_t st) {
