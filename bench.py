@@ -937,9 +937,10 @@ def bench_decode_cfg4(b, synth, dev, peak_gbs, steps=256):
     return res
 
 
-def run_profile_case(name):
+def run_profile_case(name, layers=0):
     """A small stand-alone case for a profiler capture (a few launches of one kernel on a 4-layer cut of a workload,
-    inputs larger than L2, a few GB on the device at most).  Prints nothing that is a benchmark number."""
+    inputs larger than L2, a few GB on the device at most; --layers 32 for a one-pass launch list of the whole
+    workload).  Prints nothing that is a benchmark number."""
     import torch
 
     from paper_2506_11418_b200 import binding as b, synth
@@ -953,12 +954,15 @@ def run_profile_case(name):
         "one_round_32k_chunk128": ("llama8b_32k", dict(chunk=128, n_sink=0, n_recent=0, n_rounds_max=1, r_init=1.0, r_decay=0.0, r_min=1.0)),
         "one_round_32k_chunk256": ("llama8b_32k", dict(chunk=256, n_sink=0, n_recent=0, n_rounds_max=1, r_init=1.0, r_decay=0.0, r_min=1.0)),
         "ranked_round_32k_chunk256": ("llama8b_32k", dict(chunk=256, n_sink=16, n_recent=64, n_rounds_max=1, r_init=0.8, r_decay=0.0, r_min=0.8)),
+        # the paper's schedule (ratios 0.8, 0.6, 0.4, 0.2, ... ranked per head, 16 sinks, 64 recent) to a 25 % budget
+        "paper_schedule_32k_chunk64": ("llama8b_32k", dict(chunk=64, n_sink=16, n_recent=64, n_rounds_max=16, r_init=0.8, r_decay=0.2, r_min=0.2, budget=8192)),
+        "paper_schedule_32k_chunk256": ("llama8b_32k", dict(chunk=256, n_sink=16, n_recent=64, n_rounds_max=16, r_init=0.8, r_decay=0.2, r_min=0.2, budget=8192)),
     }
     if name not in cases:
         raise SystemExit(f"unknown profile case {name!r}; known: {sorted(cases)}")
     workload, kw = cases[name]
     cfg = synth.CONFIGS[workload]
-    L, H, s, D = 4, cfg["H"], cfg["s"], cfg["d"]
+    L, H, s, D = layers or 4, cfg["H"], cfg["s"], cfg["d"]
     K = synth.ar1_keys(L, H, s, D, cfg["rho"], cfg["mean_std"], seed=cfg["seed"], dtype="bf16", device=dev)
     V = synth.normal_values(L, H, s, D, seed=cfg["seed"], dtype="bf16", device=dev)
     p = b.Params(**kw)
@@ -987,7 +991,7 @@ def main():
     ap.add_argument("--profile-case", default=None, help="run one small named case three times and exit (for ncu captures)")
     args = ap.parse_args()
     if args.profile_case:
-        run_profile_case(args.profile_case)
+        run_profile_case(args.profile_case, args.layers)
         return
     if args.steps is None:
         args.steps = 3 if args.impl == "reference" else 200
