@@ -56,9 +56,20 @@ struct GroupCfg {
   static constexpr int oMask = oTgt + kNA;
   static constexpr int oFlags = oMask + 16;     // int: largest degree of the chunk
   static constexpr int oBar = oFlags + 8;
-  static constexpr int kExtra = (oBar + 8 + 127) / 128 * 128;
-  static constexpr size_t kSmem = (size_t)kGroups * (kStage + kExtra);
+  static constexpr int oBar2 = oBar + 8;        // chunk 256: the matching MMAs have completed
+  static constexpr int oBlkInv = oBar2 + 8;     // chunk 256: float [4], largest 1 / |b| of every 32 B tokens
+  static constexpr int kExtra = (oBlkInv + 16 + 127) / 128 * 128;
+  static constexpr int oTmem = kGroups * (kStage + kExtra);  // chunk 256: the CTA's tensor-memory base address
+  static constexpr size_t kSmem = (size_t)oTmem + 16;
+  // Chunk 256: the 128 x 128 x 128 dot products of a chunk run on the 5th-generation tensor core (tcgen05.mma from the
+  // TMA-delivered tile into 128 columns of tensor memory per group); the warps only read the scores back.
+  static constexpr bool kUmma = C == 256;
 };
+
+// instruction descriptor: bf16 x bf16 -> fp32, both operands K-major, M = 128, N = 128
+__host__ __device__ constexpr uint32_t group_idesc() {
+  return (1u << 4) | (1u << 7) | (1u << 10) | ((128u >> 3) << 17) | ((128u >> 4) << 24);
+}
 
 // byte address of 16-byte piece c16 (0..15) of row `row` of a swizzled tile whose halves are `half` bytes apart
 template <int C>
@@ -183,6 +194,46 @@ __device__ __forceinline__ void match_rows(uint32_t tile, int a0, const float* i
       if (which == 2 * mt + hi) { best = vb; best_v = vv; }
     }
   best = min(best, NA - 1);  // a row of NaNs has no maximum: stay inside the chunk
+}
+
+// The same for chunk 256 from tensor memory: lane i of warp w reads row 32 w + i of the 128 x 128 accumulator (raw dot
+// products), 32 columns at a time.  The 32 B tokens around the row's own position come first: with keys that resemble
+// their neighbours they set a high mark, and another block of 32 is only examined when its largest dot product times its
+// largest 1 / |b| (blk_inv) could reach some lane's mark.  (x <= max and 1/|b| <= blk_inv, all non-negative where it
+// matters, and rounding is monotonic: a skipped block holds no better candidate; ties go to the lowest B index.)
+__device__ __forceinline__ void match_rows_tmem(uint32_t taddr, int w, const float* inv_b, const float* blk_inv, int& best,
+                                                float& best_v) {
+  float bv = -INFINITY;
+  int bi = 0x7fffffff;
+#pragma unroll 1
+  for (int k = 0; k < 4; ++k) {
+    const int blk = k == 0 ? w : (k <= w ? k - 1 : k);  // own block first, then the others in increasing order
+    float v[32];
+    tmem_ld32(taddr + (uint32_t)(32 * blk), v);
+    if (k > 0) {
+      float m0 = fmaxf(v[0], v[1]), m1 = fmaxf(v[2], v[3]);
+#pragma unroll
+      for (int j = 4; j < 32; j += 4) {
+        m0 = fmaxf(m0, fmaxf(v[j], v[j + 1]));
+        m1 = fmaxf(m1, fmaxf(v[j + 2], v[j + 3]));
+      }
+      const float bound = fmaxf(fmaxf(m0, m1), 0.f) * blk_inv[blk];
+      if (!__any_sync(0xffffffffu, bound >= bv)) continue;
+    }
+#pragma unroll
+    for (int j = 0; j < 32; j += 4) {
+      const float4 ib = *reinterpret_cast<const float4*>(inv_b + 32 * blk + j);
+      const float ibs[4] = {ib.x, ib.y, ib.z, ib.w};
+#pragma unroll
+      for (int e = 0; e < 4; ++e) {
+        const float sc = v[j + e] * ibs[e] + 0.f;  // -0 -> +0
+        const int idx = 32 * blk + j + e;
+        if (sc > bv || (sc == bv && idx < bi)) { bv = sc; bi = idx; }
+      }
+    }
+  }
+  best = min(bi, 127);  // a row of NaNs has no maximum: stay inside the chunk
+  best_v = bi == 0x7fffffff ? 0.f : bv;
 }
 
 // bf16 bit pattern of one exact 8-bit piece of a degree (piece 0: bits 0-7, 1: bits 8-15, 2: bits 16-23)
@@ -329,15 +380,23 @@ round_group_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_consta
   unsigned short* row_of = reinterpret_cast<unsigned short*>(extra + Cfg::oRowOf);
   unsigned char* tgt = extra + Cfg::oTgt;
   uint32_t* selmask = reinterpret_cast<uint32_t*>(extra + Cfg::oMask);
-  const uint32_t bar = smem_u32(extra + Cfg::oBar);
+  const uint32_t bar = smem_u32(extra + Cfg::oBar), bar2 = smem_u32(extra + Cfg::oBar2);
+  float* blk_inv = reinterpret_cast<float*>(extra + Cfg::oBlkInv);
   const int mode = a.mode;
   const bool every = mode == kModeAll, external = mode == kModeExternal;
+  const bool umma = Cfg::kUmma && !external;  // (a pass that only merges computes no similarities)
 
   if (gtid == 0) {
     mbar_init(bar, 1);
+    mbar_init(bar2, 1);
     mbar_init_fence();
   }
+  if (umma && warp == 0) tmem_alloc(smem_u32(smem + Cfg::oTmem), 512);
+  tc_fence_before();
   __syncthreads();
+  tc_fence_after();
+  const uint32_t tmem = umma ? *reinterpret_cast<volatile uint32_t*>(smem + Cfg::oTmem) : 0u;
+  bool failed = false;
 
   const int64_t n_items = (int64_t)n_full * a.LH, stride = (int64_t)gridDim.x * Cfg::kGroups;
   int64_t item = (int64_t)blockIdx.x * Cfg::kGroups + grp;
@@ -362,7 +421,8 @@ round_group_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_consta
   if (item < n_items && gtid == 0) fetch(&tm_k, item);
 
   uint32_t parity = 0;
-  for (; item < n_items; item += stride) {
+  int n_done = 0;  // chunks this group has matched (the phase of bar2)
+  for (; item < n_items; item += stride, ++n_done) {
     const int lh = (int)(item / n_full), ch = (int)(item - (int64_t)lh * n_full);
     const int64_t beg = a.lo + (int64_t)ch * C;
     const int64_t eslot = (int64_t)lh * a.edge_stride + (int64_t)ch * NA;
@@ -385,9 +445,21 @@ round_group_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_consta
       if (group_or(bar_id, GT, !ok)) {
         if (gtid == 0) atomicExch(a.status, 1);
         mbar_wait(bar, parity);  // the copies may still land: one more bounded wait before leaving
-        return;
+        failed = true;
+        break;
       }
       parity ^= 1;
+    }
+    if (umma && gtid == 0) {
+      // S = A B^T for the whole chunk: eight k steps of 16 columns (four per 64-column half of the tile)
+      tc_fence_after();
+#pragma unroll
+      for (int ks = 0; ks < 8; ++ks) {
+        const uint32_t off = (uint32_t)(ks >> 2) * Cfg::kHalf + (uint32_t)(ks & 3) * 32u;
+        umma_bf16(tmem + (uint32_t)grp * 128u, umma_desc_sw128(tile + off, 16, 1024),
+                  umma_desc_sw128(tile + (uint32_t)NA * 128u + off, 16, 1024), group_idesc(), ks ? 1u : 0u);
+      }
+      umma_commit(bar2);
     }
     int n_pieces = 1;
     if (HAS_DEG) {
@@ -399,9 +471,28 @@ round_group_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_consta
     int best = -1;
     float sim = 0.f;
     if (!external) {
-      inv_b[gtid] = inv_norms32<C>(tile, NA + 32 * w, lane);
+      const float my_inv = inv_norms32<C>(tile, NA + 32 * w, lane);
+      inv_b[gtid] = my_inv;
+      if (Cfg::kUmma) {
+        float m = my_inv;
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) m = fmaxf(m, __shfl_xor_sync(0xffffffffu, m, o));
+        if (lane == 0) blk_inv[w] = m;
+      }
       group_sync(bar_id, GT);
-      match_rows<C>(tile, 32 * w, inv_b, lane, best, sim);
+      if (Cfg::kUmma) {
+        const bool ok = mbar_wait(bar2, (uint32_t)(n_done & 1));
+        if (group_or(bar_id, GT, !ok)) {
+          if (gtid == 0) atomicExch(a.status, 1);
+          failed = true;
+          break;
+        }
+        tc_fence_after();
+        match_rows_tmem(tmem + ((uint32_t)(32 * w) << 16) + (uint32_t)grp * 128u, w, inv_b, blk_inv, best, sim);
+        tc_fence_before();  // ordered before the group barriers below, behind which the next chunk's MMAs are issued
+      } else {
+        match_rows<C>(tile, 32 * w, inv_b, lane, best, sim);
+      }
       if (mode == kModeChunkTopM) {
         sim *= inv_norms32<C>(tile, 32 * w, lane);  // Eq. 2: the ranking compares cosines
         simv[gtid] = sim;
@@ -471,7 +562,8 @@ round_group_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_consta
         if (group_or(bar_id, GT, !ok)) {
           if (gtid == 0) atomicExch(a.status, 1);
           mbar_wait(bar, parity);
-          return;
+          failed = true;
+          break;
         }
         parity ^= 1;
       }
@@ -514,6 +606,16 @@ round_group_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_consta
           fetch(&tm_k, item + stride);
       }
     }
+    if (failed) break;
+  }
+  if (umma) {  // every group is done with tensor memory
+    tc_fence_before();
+    if (__syncthreads_or(failed)) {
+      // MMAs issued before the wait that gave up may still be running: they end on their own
+      for (int i = 0; i < 1000; ++i) __nanosleep(1000);
+      __syncthreads();
+    }
+    if (warp == 0) tmem_dealloc(tmem, 512);
   }
 }
 
