@@ -543,7 +543,7 @@ def bench_compress_variants(b, synth, dev, K, V, peak_gbs, with_128k):
         out_len, rounds, cap = b.compress_plan(n, p)
         dst = b.Cache.empty(L, H, cap, D, Kx.dtype, dev)
         ws = torch.empty(b.workspace_bytes(src, p), dtype=torch.uint8, device=dev)
-        for _ in range(2):
+        for _ in range(3):
             b.compress_prefill(src, dst, p, ws)
         torch.cuda.synchronize()
         t0, t1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
@@ -580,7 +580,7 @@ def bench_compress_variants(b, synth, dev, K, V, peak_gbs, with_128k):
         del dst, ws
 
     for name, p in variants:
-        time_one(name, K, V, p, 5)
+        time_one(name, K, V, p, 10)
     if with_128k:
         cfg = synth.CONFIGS["llama8b_128k"]
         K3 = synth.ar1_keys(L, H, cfg["s"], D, cfg["rho"], cfg["mean_std"], seed=cfg["seed"], dtype="bf16", device=dev)
