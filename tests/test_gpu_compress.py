@@ -420,3 +420,36 @@ def test_no_chunking_is_bf16_only():
     with pytest.raises(b.CkvError) as e:
         b.compress_prefill(src, dst, p, ws)
     assert e.value.status == 6
+
+
+@pytest.mark.parametrize("chunk,ranked", [(64, True), (128, True), (256, True), (64, False), (256, False)])
+def test_repeated_schedules_are_bit_identical(chunk, ranked):
+    """The launches of a round overlap where they are independent (the shorter last chunk and the copies of sinks and
+    recent tokens run beside the round's main kernel).  A missing ordering would show as a run that differs: the same
+    schedule (per-head ranking, sinks, recent tokens, shorter last chunks, six rounds) is repeated into fresh, poisoned
+    buffers and every run must reproduce the first bit for bit, slot map included."""
+    b = B()
+    L, H, s = 3, 8, 20000 + chunk // 2 + 7
+    K, V, _ = make_inputs(L, H, s, "bf16", seed=77)
+    if ranked:
+        p = b.Params(chunk=chunk, n_sink=16, n_recent=64, n_rounds_max=16, r_init=0.8, r_decay=0.2, r_min=0.2, budget=s // 4)
+    else:  # every edge, three rounds: at chunk 64 the first two run in one pass, with an odd chunk left over
+        p = b.Params(chunk=chunk, n_sink=16, n_recent=64, n_rounds_max=3, r_init=1.0, r_decay=0.0, r_min=1.0)
+    src = b.Cache(K, V, None, None, s)
+    out_len, rounds, cap = b.compress_plan(s, p)
+    first = None
+    for run in range(12):
+        dst = b.Cache.empty(L, H, cap, 128, K.dtype, DEV)
+        dst.k.fill_(float("nan")); dst.v.fill_(float("nan")); dst.deg.fill_(-1)
+        ws = torch.empty(b.workspace_bytes(src, p), dtype=torch.uint8, device=DEV)
+        ws.fill_(0xA5 if run % 2 else 0x00)
+        assign = torch.full((L, H, s), -7, dtype=torch.int32, device=DEV)
+        assert b.compress_prefill(src, dst, p, ws, assign) == rounds and dst.len == out_len
+        assert b.workspace_status(ws) == 0
+        got = (dst.k[:, :, :out_len].clone(), dst.v[:, :, :out_len].clone(), dst.deg[:, :, :out_len].clone(), assign)
+        if first is None:
+            first = got
+            assert int(got[2].sum()) == L * H * s
+        else:
+            for x, y in zip(first, got):
+                assert torch.equal(x.view(torch.int16) if x.dtype == torch.bfloat16 else x, y.view(torch.int16) if y.dtype == torch.bfloat16 else y)
