@@ -180,6 +180,28 @@ def _oracle_worker_pass(_):
     return oracle_pass(_WORKER_INPUT)
 
 
+def _oracle_parity_pass(job):
+    """One (layer, head) slab of the timed compression against the oracle: how many entries of the slot map differ, and
+    how many of those sit where the oracle's two best candidates are closer than 1e-5 relative (near ties)."""
+    import numpy as np
+    from threadpoolctl import threadpool_limits
+
+    from oracle import ckv_oracle as O
+
+    K, V, assign_gpu, deg_gpu, chunk = job
+    s = K.shape[0]
+    p = O.Params(chunk=chunk, n_sink=0, n_recent=0, n_rounds_max=1, r_init=1.0, r_decay=0.0, r_min=1.0)
+    with threadpool_limits(limits=1):
+        _, _, do, asg, log = O.csm_round(K[None, None].astype(np.float64), V[None, None].astype(np.float64),
+                                         np.ones((1, 1, s), dtype=np.int64), p, 1.0, storage=None)
+    e = log.edges[0]
+    gap_at = np.full(s, np.inf)
+    gap_at[e.a_pos] = e.argmax_gap
+    differ = np.nonzero(asg[0, 0] != assign_gpu)[0]
+    return {"edges": int(len(e.a_pos)), "differ": int(len(differ)), "near": int(np.sum(gap_at[differ] < 1e-5)),
+            "deg_equal": bool(np.array_equal(do[0, 0], deg_gpu)) if len(differ) == 0 else None}
+
+
 class OraclePool:
     """The oracle on the host's cores: one single-threaded NumPy process per core, each working through (layer, head)
     slabs (the method is independent per slab; the oracle itself is not changed or tuned for this).  Must be created
@@ -261,10 +283,10 @@ def run_gpu(args):
     rank, local, world = parallel.env_world()
     # the CPU baseline first: its worker processes are forked, which has to happen before this process touches CUDA
     cpu = None
+    pool = None
     if rank == 0 and world == 1 and not args.skip_cpu:
         pool = OraclePool()
-        cpu = cpu_baseline(pool)
-        pool.close()
+        cpu = cpu_baseline(pool)  # (the workers stay for the parity sample below; they never touch CUDA)
     if not torch.cuda.is_available():
         raise SystemExit("bench.py needs a CUDA device; there is no CPU fallback")
     torch.cuda.set_device(local)
@@ -292,6 +314,23 @@ def run_gpu(args):
     wsd = torch.empty(b.decode_workspace_bytes(1, H, G, D, cap + c), dtype=torch.uint8, device=dev)
     scale = 1.0 / math.sqrt(D)
     final_len = out_len + c // 2
+    if pool is not None:
+        # two slabs of the timed compression, clustered on their own with the slot map, against the oracle on the host
+        jobs = []
+        for l, h in ((0, 0), (L // 2, 5 % H)):
+            one = b.Cache(K[l:l + 1, h:h + 1].contiguous(), V[l:l + 1, h:h + 1].contiguous(), None, None, s)
+            d1 = b.Cache.empty(1, 1, cap, D, K.dtype, dev)
+            asg = torch.full((1, 1, s), -1, dtype=torch.int32, device=dev)
+            b.compress_prefill(one, d1, p, ws, asg)
+            jobs.append((one.k[0, 0].float().cpu().numpy(), one.v[0, 0].float().cpu().numpy(), asg[0, 0].cpu().numpy().astype("int64"),
+                         d1.deg[0, 0, :out_len].cpu().numpy().astype("int64"), c))
+        res = pool.pool.map(_oracle_parity_pass, jobs, chunksize=1)
+        pool.close()
+        cpu["parity_sample"] = {
+            "what": "the timed compression on 2 (layer, head) slabs against the oracle (fp64): entries of the slot map that differ",
+            "slabs": len(res), "edges": sum(r["edges"] for r in res), "slot_map_entries_that_differ": sum(r["differ"] for r in res),
+            "of_which_near_ties_below_1e-5": sum(r["near"] for r in res),
+            "degrees_equal_where_the_maps_agree": all(r["deg_equal"] for r in res if r["deg_equal"] is not None)}
     # the lengths a step produces are a function of shapes only, so the decode views can be built once
     dst.len = final_len
     views = [b.layer_views([dst], l, dev) for l in range(L)]
