@@ -153,22 +153,25 @@ round_fast_kernel(const FastArgs a, const __grid_constant__ typename std::condit
     out_row0 += out_pos0;
     // paged: the layer and head of this slab, and the (at most two) destination pages the chunk's output rows reach
     int pl = 0, ph = 0;
-    int64_t dst_pg0 = 0, dst_id0 = 0, dst_id1 = 0;
+    // output row `op` sits at pool row out_pos0 + op + pg_add0 while it is in the first page (op < pg_first), + pg_add1 behind
+    int64_t pg_add0 = 0, pg_add1 = 0;
+    int pg_first = 0;
     if constexpr (PAGED) {
       pl = (int)(lh / (uint32_t)pg.H);
       ph = (int)(lh - (uint32_t)pl * pg.H);
       if (KIND != kFastMatch) {
-        dst_pg0 = out_pos0 >> pg.shift;
-        dst_id0 = pg.dst_table[min(dst_pg0, pg.dst_last_page)];
-        dst_id1 = pg.dst_table[min((out_pos0 + kC - 1) >> pg.shift, pg.dst_last_page)];
+        const int64_t dst_pg0 = out_pos0 >> pg.shift;
+        const int64_t dst_id0 = pg.dst_table[min(dst_pg0, pg.dst_last_page)];
+        const int64_t dst_id1 = pg.dst_table[min((out_pos0 + kC - 1) >> pg.shift, pg.dst_last_page)];
+        pg_first = (int)(((dst_pg0 + 1) << pg.shift) - out_pos0);
+        pg_add0 = ((dst_id0 * pg.H + ph) << pg.shift) - (dst_pg0 << pg.shift);
+        pg_add1 = ((dst_id1 * pg.H + ph) << pg.shift) - ((dst_pg0 + 1) << pg.shift);
       }
     }
     // row of output row `op` of this chunk: in the destination slab array, or in the destination pool's page grid
     auto dst_row = [&](int op) -> int64_t {
       if constexpr (PAGED) {
-        const int64_t pos = out_pos0 + op;
-        const int64_t id = (pos >> pg.shift) == dst_pg0 ? dst_id0 : dst_id1;
-        return ((id * pg.H + ph) << pg.shift) + (pos & (((int64_t)1 << pg.shift) - 1));
+        return out_pos0 + op + (op < pg_first ? pg_add0 : pg_add1);
       } else {
         return out_row0 + op;
       }
