@@ -131,6 +131,27 @@ class ClockSampler:
                 "reasons": sorted(self.reasons), "samples": len(self.samples)}
 
 
+def timed_burst(torch, dev, fn, iters, warm=3, rest_s=0.3):
+    """Mean milliseconds of fn() over `iters` calls, after a rest and `warm` untimed calls, with the SM clock seen
+    meanwhile.  The rest lets the board's power average fall back so that every row is a kernel timed alone: after a
+    few hundred milliseconds of back-to-back launches the SM clock of these parts sinks from 1965 to 1.7-1.9 GHz, and
+    every kernel that is not purely bandwidth-bound slows down with it (a row would then depend on the rows before it)."""
+    torch.cuda.synchronize()
+    time.sleep(rest_s)
+    for _ in range(warm):
+        fn()
+    torch.cuda.synchronize()
+    sampler = ClockSampler(dev.index or 0, 0.002)
+    t0, t1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    t0.record()
+    for _ in range(iters):
+        fn()
+    t1.record()
+    torch.cuda.synchronize()
+    clk = sampler.stop()
+    return t0.elapsed_time(t1) / iters, {"sm_mhz": clk.get("sm_mhz"), "reasons": clk.get("reasons")}
+
+
 # --------------------------------------------------------------------------- CPU oracle leg
 
 def oracle_inputs(n_heads: int, seed: int = 0):
@@ -424,12 +445,14 @@ def run_gpu(args):
         extra["no_chunk"] = bench_no_chunk(b, synth, dev, K, V, peaks, args.layers == 0)
         extra["paged_compress"] = bench_paged_compress(b, synth, dev, K, V, peak)
         targets["paged_compress_ratio1"] = {k: extra["paged_compress"]["chunk64 ratio1"][k] for k in ("ms", "frac_of_peak", "pages_freed")}
+        targets["paged_compress_ratio1"]["sm_mhz"] = extra["paged_compress"]["chunk64 ratio1"]["clocks"]["sm_mhz"]
         cv = extra["compress_variants"]
         def pick(name):
             if name not in cv:
                 return None
             row = {k: cv[name][k] for k in ("ms", "frac_of_peak", "gbs", "moved_gb", "frac_on_moved_bytes")}
             row["frac_of_nominal_8tbs"] = row["gbs"] / 8000.0
+            row["sm_mhz"] = cv[name]["clocks"]["sm_mhz"]
             return row
         targets["chunk128_ratio1"] = pick("chunk128 ratio1")
         targets["chunk256_ratio1"] = pick("chunk256 ratio1")
@@ -456,7 +479,8 @@ def run_gpu(args):
                                           "compressed_frac_of_nominal_8tbs": d4["compressed"]["gbs"] / 8000.0,
                                           "uncompressed_us_per_layer_step": d4["uncompressed"]["us_per_layer_step"],
                                           "speedup_vs_uncompressed": d4["speedup"], "steps": d4["compressed"]["steps"],
-                                          "paged_frac_of_peak": extra["decode_cfg4_paged"]["frac_of_peak"]}
+                                          "paged_frac_of_peak": extra["decode_cfg4_paged"]["frac_of_peak"],
+                                          "sm_mhz": d4["compressed"]["clocks"]["sm_mhz"]}
     if rank == 0 and not args.skip_serving and args.layers == 0:
         extra["serving_mix"] = bench_serving_mix(b, synth, dev, peak, steps=args.serving_steps)
         sm = extra["serving_mix"]
@@ -582,16 +606,7 @@ def bench_compress_variants(b, synth, dev, K, V, peak_gbs, with_128k):
         out_len, rounds, cap = b.compress_plan(n, p)
         dst = b.Cache.empty(L, H, cap, D, Kx.dtype, dev)
         ws = torch.empty(b.workspace_bytes(src, p), dtype=torch.uint8, device=dev)
-        for _ in range(3):
-            b.compress_prefill(src, dst, p, ws)
-        torch.cuda.synchronize()
-        t0, t1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-        t0.record()
-        for _ in range(iters):
-            b.compress_prefill(src, dst, p, ws)
-        t1.record()
-        torch.cuda.synchronize()
-        ms = t0.elapsed_time(t1) / iters
+        ms, clk = timed_burst(torch, dev, lambda: b.compress_prefill(src, dst, p, ws), iters)
         lens, cur = [n], n
         for j in range(rounds):
             pj = P(chunk=p.chunk, n_sink=p.n_sink, n_recent=p.n_recent, n_rounds_max=j + 1, r_init=p.r_init, r_decay=p.r_decay,
@@ -615,7 +630,7 @@ def bench_compress_variants(b, synth, dev, K, V, peak_gbs, with_128k):
         res[name] = {"seq": n, "out_len": out_len, "rounds": rounds, "ms": ms, "tokens_per_s": n / (ms * 1e-3),
                      "gbs": nbytes / (ms * 1e-3) / 1e9, "frac_of_peak": nbytes / (ms * 1e-3) / 1e9 / peak_gbs,
                      "moved_gb": moved / 1e9, "frac_on_moved_bytes": moved / (ms * 1e-3) / 1e9 / peak_gbs,
-                     "status": b.workspace_status(ws)}
+                     "clocks": clk, "status": b.workspace_status(ws)}
         del dst, ws
 
     for name, p in variants:
@@ -757,19 +772,11 @@ def bench_no_chunk(b, synth, dev, K, V, peaks, with_128k):
         out_len, _, cap = b.compress_plan(n, p)
         dst = b.Cache.empty(L, H, cap, D, Ks.dtype, dev)
         ws = torch.empty(b.workspace_bytes(src, p), dtype=torch.uint8, device=dev)
-        b.compress_prefill(src, dst, p, ws)
-        torch.cuda.synchronize()
-        t0, t1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-        t0.record()
-        for _ in range(iters):
-            b.compress_prefill(src, dst, p, ws)
-        t1.record()
-        torch.cuda.synchronize()
-        ms = t0.elapsed_time(t1) / iters
+        ms, clk = timed_burst(torch, dev, lambda: b.compress_prefill(src, dst, p, ws), iters, warm=1)
         tf = 2.0 * L * H * (n / 2) * (n / 2) * D / (ms * 1e-3) / 1e12
         return {"layers": L, "seq": n, "out_len": out_len, "ms": ms, "similarity_tflops": tf, "bound": "tensor",
                 "frac_of_bf16_peak": tf / peaks["bf16_tflops"], "workspace_mib": ws.numel() / 2**20,
-                "status": b.workspace_status(ws)}
+                "clocks": clk, "status": b.workspace_status(ws)}
 
     L, n = min(4, K.shape[0]), 16384
     res = {"16k_4_layers": time_one(K[:L, :, :n].contiguous(), V[:L, :, :n].contiguous(), 3)}
@@ -897,21 +904,11 @@ def bench_paged_compress(b, synth, dev, K, V, peak_gbs, page_tokens=64):
             pools.append((kp, vp, dp, lp))
         ws = torch.empty(b.paged_workspace_bytes(L, H, D, torch.bfloat16, s, p), dtype=torch.uint8, device=dev)
         # the call overwrites its source pages, which does not change what a repeated call costs
-        for _ in range(2):
-            b.compress_paged(pools, table, s, False, scratch, p, ws)
-        torch.cuda.synchronize()
-        iters = 5
-        t0, t1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-        t0.record()
-        for _ in range(iters):
-            b.compress_paged(pools, table, s, False, scratch, p, ws)
-        t1.record()
-        torch.cuda.synchronize()
-        ms = t0.elapsed_time(t1) / iters
+        ms, clk = timed_burst(torch, dev, lambda: b.compress_paged(pools, table, s, False, scratch, p, ws), 5, warm=2)
         nbytes = schedule_bytes(L, H, s, out_len, D, 2)
         res[name] = {"page_tokens": P, "seq": s, "out_len": out_len, "rounds": rounds, "ms": ms, "gbs": nbytes / (ms * 1e-3) / 1e9,
                      "frac_of_peak": nbytes / (ms * 1e-3) / 1e9 / peak_gbs, "pages_kept": kept, "pages_freed": own - kept,
-                     "status": b.workspace_status(ws)}
+                     "clocks": clk, "status": b.workspace_status(ws)}
         del pools, ws
         torch.cuda.empty_cache()
     return res
@@ -946,6 +943,8 @@ def bench_decode_cfg4(b, synth, dev, peak_gbs, steps=256):
         out = torch.empty_like(qs[0])
         ws = torch.empty(b.decode_workspace_bytes(Bz, H, G, D, cap), dtype=torch.uint8, device=dev)
         wsa = torch.empty(b.workspace_bytes(caches[0], no_trigger), dtype=torch.uint8, device=dev)
+        torch.cuda.synchronize()
+        time.sleep(0.3)      # each arm timed alone (see timed_burst)
         for i in range(5):   # warm-up on the initial length
             b.decode_attn(b.layer_views(caches, 0, dev), H, G, qs[i], out, scale, slots, ws)
         # the view arrays of all steps are laid out on the device beforehand (only the lengths differ), so that the loop
@@ -953,6 +952,7 @@ def bench_decode_cfg4(b, synth, dev, peak_gbs, steps=256):
         views_all = b.layer_views(caches, 0, dev).unsqueeze(0).repeat(steps, 1, 1)
         views_all[:, :, 3] += torch.arange(1, steps + 1, device=dev, dtype=torch.int64).view(steps, 1)
         torch.cuda.synchronize()
+        sampler = ClockSampler(dev.index or 0, 0.002)
         evs, rows = [], 0
         for i in range(steps):
             b.compress_append_batch(caches, kn[i], vn[i], no_trigger, wsa)
@@ -965,11 +965,13 @@ def bench_decode_cfg4(b, synth, dev, peak_gbs, steps=256):
             evs.append((e0, e1))
             rows += Bz * H * n
         torch.cuda.synchronize()
+        clk = sampler.stop()
         assert caches[0].len == slots + steps
         us = 1e3 * statistics.mean(x.elapsed_time(y) for x, y in evs)
         nbytes = (decode_bytes(rows, D, 2) if with_deg else rows * 2 * D * 2) / steps
         res[name] = {"slots": f"{slots} -> {slots + steps}", "steps": steps, "us_per_layer_step": us, "gbs": nbytes / (us * 1e-6) / 1e9,
-                     "frac_of_peak": nbytes / (us * 1e-6) / 1e9 / peak_gbs, "decode_tok_s_per_layer": Bz / (us * 1e-6)}
+                     "frac_of_peak": nbytes / (us * 1e-6) / 1e9 / peak_gbs, "decode_tok_s_per_layer": Bz / (us * 1e-6),
+                     "clocks": {"sm_mhz": clk.get("sm_mhz"), "reasons": clk.get("reasons")}}
         del caches
         torch.cuda.empty_cache()
     res["speedup"] = res["uncompressed"]["us_per_layer_step"] / res["compressed"]["us_per_layer_step"]
