@@ -1019,7 +1019,7 @@ def run_profile_case(name, layers=0):
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=None, help="timed steps (default: 200; 3 for --impl reference, whose step is seconds of CPU work)")
+    ap.add_argument("--steps", type=int, default=None, help="timed steps (default: 50; 3 for --impl reference, whose step is seconds of CPU work)")
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="ckv", choices=["ckv", "reference"])
     ap.add_argument("--layers", type=int, default=0, help="use only this many layers of the workload (profiling a small case)")
@@ -1035,7 +1035,7 @@ def main():
         run_profile_case(args.profile_case, args.layers)
         return
     if args.steps is None:
-        args.steps = 3 if args.impl == "reference" else 200
+        args.steps = 3 if args.impl == "reference" else 50
     if args.impl == "reference":
         run_reference(args)
     else:
