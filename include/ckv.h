@@ -8,7 +8,11 @@
  *    The library allocates and frees nothing and keeps no global state that a call could observe (the one
  *    exception is ckv_decode_attn_static, whose scratch array is shared by every call: see its comment).
  *  - All work is enqueued on `cuda_stream` (a cudaStream_t passed as void*; NULL = the
- *    default stream) and the calls return without synchronising.
+ *    default stream) and the calls return without synchronising.  The kernels are launched with programmatic
+ *    stream serialization among themselves; towards the caller they behave like ordinary stream work (a call's results are
+ *    complete when the last of its kernels is).  Only a caller kernel that is itself launched with the programmatic
+ *    serialization attribute directly behind a call has to execute griddepcontrol.wait (cudaGridDependencySynchronize)
+ *    before it reads the call's results, as that attribute always requires.
  *  - The return value is a ckv_status.  Argument errors are found on the host before any
  *    launch and leave every output untouched.
  *  - Tensors are row-major.  K and V of one sequence: [L, H, cap, D] (layers, KV heads,
